@@ -1,0 +1,171 @@
+"""CPU fp64 oracle for the per-matrix Muon optimizer step.
+
+TEST INFRASTRUCTURE ONLY.  This module defines what "correct" means for the
+CUDA path; it is imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg, and by nothing else.  It shares no code with the
+CUDA path and never imports it.  Everything is plain NumPy in float64; the only
+library primitive used as a step is the dense matrix product ``@``.  There is
+no blocking, no fusion, no use of symmetry and no reordering beyond what the
+paper's equations state, so each function can be checked against the paper by
+eye.
+
+All functions take float64 arrays.  Callers widen bf16 / fp32 storage to
+float64 exactly (every bf16 and fp32 value is representable) before calling.
+
+Every function here is pinned by tests that do not call back into it (closed
+forms, an SVD from LAPACK, hand-derived 2x2 cases, brute-force expansion,
+symmetries); no function is "parity unpinned".
+
+Passages followed (paper = "Muon is Scalable for LLM Training"):
+  * Sec. 2.1 "The Muon Optimizer": the three-line update rule (momentum,
+    Newton-Schulz, weight step) and its footnote 1 (Nesterov-style input).
+  * Sec. 2.1 "Newton-Schulz Iterations for Matrix Orthogonalization":
+    X_0 = M / ||M||_F and the quintic iteration (Eq. 2) with the coefficients
+    a = 3.4445, b = -4.7750, c = 2.0315.
+  * Sec. 2.2 "Weight Decay" (Eq. 3) and "Matching update RMS of AdamW"
+    (the unnumbered equation with 0.2 * sqrt(max(A, B))).
+  * Algorithm 1, last line: the update RMS returned for logging.
+"""
+
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+
+import numpy as np
+
+# Sec. 2.1: coefficients of the quintic Newton-Schulz polynomial.
+NS_A = 3.4445
+NS_B = -4.7750
+NS_C = 2.0315
+
+
+@dataclass
+class Hyper:
+    """Hyper-parameters of one step.  Defaults are the paper's choices:
+    mu = 0.95 and N = 5 (Sec. 2.2 "Other Hyper-parameters"), Nesterov-style
+    input (Sec. 2.1 footnote 1), update-RMS factor 0.2 (Sec. 2.2)."""
+
+    lr: float = 2e-2
+    wd: float = 0.1
+    mu: float = 0.95
+    nesterov: bool = True
+    ns_steps: int = 5
+    a: float = NS_A
+    b: float = NS_B
+    c: float = NS_C
+    eps: float = 1e-7
+    rms_scale: float = 0.2
+
+
+def _f64(x):
+    x = np.asarray(x)
+    if x.dtype != np.float64:
+        raise TypeError("oracle inputs must already be widened to float64")
+    return x
+
+
+def momentum_update(M_prev, G, mu):
+    """M_t = mu * M_{t-1} + grad  (Sec. 2.1, first line of the update rule).
+    No dampening factor appears in the paper's rule."""
+    return mu * _f64(M_prev) + _f64(G)
+
+
+def newton_schulz_input(M_new, G, mu, nesterov):
+    """What is fed to Newton-Schulz.  Sec. 2.1 footnote 1: with the
+    Nesterov-style momentum the input is mu * M_t + grad (M_t is the freshly
+    updated momentum); otherwise it is M_t itself."""
+    if nesterov:
+        return mu * _f64(M_new) + _f64(G)
+    return _f64(M_new).copy()
+
+
+def frobenius_normalise(U, eps):
+    """X_0 = U / ||U||_F  (Sec. 2.1, Newton-Schulz paragraph).  The paper has
+    no epsilon; the reading taken here is X_0 = U / (||U||_F + eps) so that a
+    zero input gives X_0 = 0 instead of NaN.  Returns (norm, X_0)."""
+    U = _f64(U)
+    nu = math.sqrt(float(np.sum(U * U)))
+    return nu, U / (nu + eps)
+
+
+def newton_schulz(X0, steps, a=NS_A, b=NS_B, c=NS_C, trace=None):
+    """N steps of Eq. 2:  X_k = a X + b (X X^T) X + c (X X^T)^2 X.
+
+    When the matrix has more rows than columns the iteration runs on the
+    transpose and the result is transposed back; the polynomial is odd, so in
+    exact arithmetic this changes nothing and only makes X X^T the smaller of
+    the two possible Gram matrices.  If ``trace`` is a list, the per-iteration
+    (A, B, X) triples are appended to it in the orientation the iteration ran
+    in (short side first)."""
+    X = _f64(X0)
+    transposed = X.shape[0] > X.shape[1]
+    if transposed:
+        X = X.T
+    X = X.copy()
+    for _ in range(int(steps)):
+        A = X @ X.T
+        B = b * A + c * (A @ A)
+        X = a * X + B @ X
+        if trace is not None:
+            trace.append((A, B, X.copy()))
+    if transposed:
+        X = X.T
+    return np.ascontiguousarray(X)
+
+
+def apply_update(W, O, lr, wd, rms_scale=0.2):
+    """W_t = W_{t-1} - lr * (rms_scale * sqrt(max(A, B)) * O + wd * W_{t-1})
+    for a parameter of shape [A, B]  (Sec. 2.2, "Matching update RMS of
+    AdamW"; rms_scale is the paper's 0.2).  The decay term uses W_{t-1} and is
+    multiplied by the learning rate, as in Eq. 3."""
+    W = _f64(W)
+    O = _f64(O)
+    rows, cols = W.shape
+    scale = rms_scale * math.sqrt(max(rows, cols))
+    return W - lr * (scale * O + wd * W)
+
+
+def update_rms(O, rms_scale=0.2):
+    """sqrt(mean(u^2)) of the scaled update u = rms_scale*sqrt(max(A,B))*O
+    (Algorithm 1, returned value; the reading taken is that u carries the
+    scale factor, so the value sits near 0.2 as Sec. 2.2 intends)."""
+    O = _f64(O)
+    rows, cols = O.shape
+    u = rms_scale * math.sqrt(max(rows, cols)) * O
+    return math.sqrt(float(np.mean(u * u)))
+
+
+def muon_step(W, G, M, hp: Hyper, trace=False):
+    """One full Muon step for one matrix.  Returns a dict with the new weight
+    ``W``, the new momentum ``M``, the Frobenius norm ``nu`` of the
+    Newton-Schulz input, ``X0``, the orthogonalised update ``O``, the logged
+    ``rms`` and, when ``trace`` is set, the per-iteration (A, B, X) list.
+
+    Non-finite input (a NaN or Inf anywhere in the Newton-Schulz input): the
+    paper is silent.  The reading taken: the weight is left unchanged, the
+    momentum is still M_t as the first line of the rule defines it, and the
+    result carries ``nonfinite = True``."""
+    W = _f64(W)
+    G = _f64(G)
+    M = _f64(M)
+    if not (W.shape == G.shape == M.shape and W.ndim == 2):
+        raise ValueError("W, G, M must be 2-D and of one shape")
+    M_new = momentum_update(M, G, hp.mu)
+    U = newton_schulz_input(M_new, G, hp.mu, hp.nesterov)
+    nu, X0 = frobenius_normalise(U, hp.eps)
+    out = {"M": M_new, "nu": nu, "nonfinite": False}
+    if not math.isfinite(nu):
+        out.update(W=W.copy(), X0=None, O=None, rms=float("nan"), nonfinite=True)
+        return out
+    stages = [] if trace else None
+    O = newton_schulz(X0, hp.ns_steps, hp.a, hp.b, hp.c, trace=stages)
+    out.update(
+        W=apply_update(W, O, hp.lr, hp.wd, hp.rms_scale),
+        X0=X0,
+        O=O,
+        rms=update_rms(O, hp.rms_scale),
+    )
+    if trace:
+        out["stages"] = stages
+    return out
