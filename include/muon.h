@@ -1,0 +1,204 @@
+/*
+ * muon.h - C ABI of the B200 (sm_100a) Muon optimizer-step library.
+ *
+ * The library performs, for every 2-D parameter matrix it is given, the
+ * per-matrix Muon step of "Muon is Scalable for LLM Training":
+ *
+ *   M <- mu*M + G                                   (Sec. 2.1, update rule)
+ *   U  = mu*M + G  (Nesterov-style) or  U = M       (Sec. 2.1, footnote 1)
+ *   X0 = U / (||U||_F + eps)                        (Sec. 2.1, Newton-Schulz paragraph)
+ *   repeat ns_steps:  A = X X^T;  B = b*A + c*A^2;  X = a*X + B X      (Eq. 2)
+ *   W <- W - lr*(rms_scale*sqrt(max(rows,cols))*X + wd*W)
+ *                                                   (Sec. 2.2, Eq. 3 and the
+ *                                                    "Matching update RMS" equation)
+ *
+ * Newton-Schulz runs in bf16 with fp32 accumulation on the matrix in its
+ * short-side-first orientation (transposed when rows > cols); everything
+ * element-wise is fp32.  Every step runs in hand-written CUDA kernels; there is
+ * no CPU fallback.  All pointers in param-group descriptors are DEVICE pointers
+ * unless a comment says "host".  All entry points return 0 on success and a
+ * negative MUON_ERR_* code on failure; on a host-side failure nothing has been
+ * launched.  muon_last_error() gives a thread-local message for the last
+ * failure.
+ *
+ * Which parameters: 2-D weight matrices only.  Embeddings, the LM head and
+ * norm gains stay with AdamW (Sec. 2.2 "Matching update RMS of AdamW"); the
+ * caller also decides matrix granularity (Sec. 2.2 warns that splitting e.g.
+ * each KV head into its own matrix makes max(rows, cols) too small).
+ */
+#ifndef MUON_H_
+#define MUON_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  MUON_OK = 0,
+  MUON_ERR_INVALID_ARG = -1,  /* null pointer, non-positive size, bad enum */
+  MUON_ERR_UNSUPPORTED = -2,  /* dtype / size the kernels do not handle */
+  MUON_ERR_ALIGNMENT = -3,    /* pointer or leading dimension not aligned as required */
+  MUON_ERR_WORKSPACE = -4,    /* workspace too small or misaligned */
+  MUON_ERR_CUDA = -5,         /* a CUDA runtime / driver call failed */
+  MUON_ERR_TIMEOUT = -6,      /* a bounded device-side wait expired (device status) */
+  MUON_ERR_NONFINITE = -7     /* a matrix had a NaN/Inf Newton-Schulz input (device status) */
+};
+
+enum { MUON_DTYPE_BF16 = 0, MUON_DTYPE_FP32 = 1 };
+
+/*
+ * One group = `count` matrices of one shape [rows, cols] and one dtype pair.
+ * Groups of equal (min(rows,cols), max(rows,cols), dtypes) are merged into one
+ * shape bucket and processed by batched launches, whatever their orientation.
+ *
+ *   w, g, m : HOST arrays of `count` DEVICE pointers (weight, gradient,
+ *             momentum).  Row-major, `rows` rows of `cols` elements, row
+ *             stride ld_* elements.  The pointer arrays are copied at init;
+ *             the matrices themselves stay owned by the caller and must stay
+ *             allocated until muon_destroy.  W, G and M must not alias.
+ *   w_dtype : dtype of W (bf16 or fp32).  g_dtype: dtype of G.  M is always
+ *             fp32 and must be zero before the first step (M_0 = 0, Sec. 2.1).
+ *   Alignment: every pointer aligned to its element size; ld_w, ld_g, ld_m >=
+ *             cols.  The fast vector paths need 16-byte aligned pointers and
+ *             ld_* that are multiples of 8; anything else takes a slower
+ *             scalar path with the same results.
+ */
+typedef struct muon_group {
+  int32_t rows;
+  int32_t cols;
+  int32_t count;
+  int32_t w_dtype;
+  int32_t g_dtype;
+  int32_t reserved;
+  void* const* w;
+  const void* const* g;
+  float* const* m;
+  int64_t ld_w;
+  int64_t ld_g;
+  int64_t ld_m;
+} muon_group;
+
+/*
+ * Hyper-parameters of one step (passed per call, nothing is cached).
+ *   lr, wd    : eta and lambda of Eq. 3 (shared with AdamW, Sec. 2.2).
+ *   mu        : momentum, 0.95 in the paper.
+ *   nesterov  : non-zero selects the Nesterov-style input of footnote 1.
+ *   ns_steps  : N of Eq. 2 (5 in the paper; 0 skips the iteration, O = X0).
+ *   a, b, c   : quintic coefficients (3.4445, -4.7750, 2.0315).
+ *   eps       : added to the Frobenius norm (the paper has none; 1e-7 keeps a
+ *               zero input finite).
+ *   rms_scale : the 0.2 of Sec. 2.2.
+ */
+typedef struct muon_hparams {
+  float lr;
+  float wd;
+  float mu;
+  int32_t nesterov;
+  int32_t ns_steps;
+  float a;
+  float b;
+  float c;
+  float eps;
+  float rms_scale;
+} muon_hparams;
+
+typedef struct muon_ctx muon_ctx;
+
+/*
+ * Bytes of device workspace muon_init needs for these groups (pure host
+ * computation; only rows/cols/count/dtypes are read).  The workspace holds the
+ * bf16 Newton-Schulz operands X, A, B of one bucket chunk, pointer tables,
+ * per-matrix scalars and the status word.  Large buckets are processed in
+ * chunks so that the workspace stays bounded.
+ */
+int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_bytes);
+
+/*
+ * Build a context: validate the descriptors, form shape buckets, carve the
+ * caller's workspace (DEVICE memory, 1024-byte aligned, at least
+ * muon_workspace_bytes() long, owned by the caller, alive until destroy),
+ * upload pointer tables and encode the TMA descriptors.  `device` is the CUDA
+ * device ordinal all pointers live on.  Allocates no device memory itself.
+ */
+int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* workspace,
+              size_t workspace_bytes, int device);
+
+/*
+ * Enqueue one Muon step for every matrix of the context on `stream` (a
+ * cudaStream_t passed as void*; NULL = legacy default stream).  Reads G,
+ * updates W and M in place.  Asynchronous: returns after the launches are
+ * enqueued, performs no allocation and no host synchronisation.  Device-side
+ * problems (expired wait, non-finite input) are reported by muon_status.
+ * Calls on one context must be stream-ordered with respect to each other.
+ */
+int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream);
+
+/*
+ * Same step with HOST gradients and HOST weight read-back, for callers whose
+ * gradients arrive in (pinned) host memory: for every matrix i of every group
+ * j, g_host[j][i] (host, dense rows*cols of the group's g_dtype) is copied
+ * into the device G buffer, the step runs, and if w_host is non-NULL the
+ * updated W is copied to w_host[j][i] (host, dense rows*cols of w_dtype).
+ * All copies are cudaMemcpyAsync on `stream`; the call does not synchronise.
+ */
+int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* const* g_host,
+                   void* const* const* w_host, void* stream);
+
+/*
+ * Synchronise `stream` and read the device status word.  *device_status is 0,
+ * MUON_ERR_TIMEOUT or MUON_ERR_NONFINITE; *matrix_index (may be NULL) is the
+ * global index (groups in order, matrices in order) of the first matrix that
+ * reported it, or -1.  The status word is cleared.  A matrix with a non-finite
+ * Newton-Schulz input keeps its W; its M has been updated (and now holds the
+ * non-finite values).
+ */
+int muon_status(muon_ctx* ctx, void* stream, int* device_status, int* matrix_index);
+
+/*
+ * Per-matrix Frobenius norms ||U||_F of the last step's Newton-Schulz inputs:
+ * copies `n` floats (global matrix order) to the HOST array `out` after
+ * synchronising `stream`.
+ */
+int muon_get_norms(muon_ctx* ctx, void* stream, float* out, int n);
+
+/* Free the host-side context.  Never touches caller memory. */
+int muon_destroy(muon_ctx* ctx);
+
+/* Message for the last failure on this thread ("" if none). */
+const char* muon_last_error(void);
+
+/* Number of kernels the last muon_step on this context enqueued. */
+int muon_last_launch_count(const muon_ctx* ctx);
+
+/*
+ * Test taps.  muon_debug_keep(ctx, 1) makes the last Newton-Schulz iteration
+ * also store its X (= O) in the workspace.  muon_debug_read copies one stage
+ * of one matrix to a HOST buffer as dense bf16, short side first (m x n with
+ * m = min(rows, cols); m x m for A and B): `which` is MUON_TAP_X0 (bf16(U),
+ * NOT yet divided by the norm; valid while ns_steps <= 1), MUON_TAP_A, MUON_TAP_B (last iteration) or
+ * MUON_TAP_X (last iteration's X).  Only valid while the matrix's chunk is
+ * still resident (buckets that fit one chunk).  Synchronises the device.
+ */
+enum { MUON_TAP_X0 = 0, MUON_TAP_A = 1, MUON_TAP_B = 2, MUON_TAP_X = 3 };
+int muon_debug_keep(muon_ctx* ctx, int keep);
+int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, size_t dst_bytes);
+
+/*
+ * Test/bench knob: operand layout of the a*X + B*X product, process-wide, read
+ * by muon_workspace_bytes and muon_init (contexts keep the value they were
+ * created with).
+ *   0 = the X operand is read from X itself (MN-major shared-memory
+ *       descriptor); default,
+ *   1 = the X operand is read from a transposed copy X^T kept beside X
+ *       (K-major descriptor); costs extra workspace and traffic.
+ * Returns the previous value.
+ */
+int muon_debug_set_variant(int variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MUON_H_ */

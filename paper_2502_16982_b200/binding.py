@@ -1,0 +1,267 @@
+"""ctypes binding of the Muon C ABI (include/muon.h).
+
+Argument marshalling only: every step of the optimizer runs in the CUDA
+kernels of libmuon_b200.so.  PyTorch supplies device memory and streams.
+The functions carry the C names; :class:`MuonContext` bundles them for the
+usual init / step / status / destroy life cycle.
+"""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmuon_b200.so")
+
+MUON_OK = 0
+MUON_ERR_INVALID_ARG = -1
+MUON_ERR_UNSUPPORTED = -2
+MUON_ERR_ALIGNMENT = -3
+MUON_ERR_WORKSPACE = -4
+MUON_ERR_CUDA = -5
+MUON_ERR_TIMEOUT = -6
+MUON_ERR_NONFINITE = -7
+MUON_DTYPE_BF16 = 0
+MUON_DTYPE_FP32 = 1
+MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
+
+EXPORTED = [
+    "muon_workspace_bytes", "muon_init", "muon_step", "muon_step_host", "muon_status",
+    "muon_get_norms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
+    "muon_debug_keep", "muon_debug_read", "muon_debug_set_variant",
+]
+
+
+class muon_group(C.Structure):
+    _fields_ = [
+        ("rows", C.c_int32), ("cols", C.c_int32), ("count", C.c_int32),
+        ("w_dtype", C.c_int32), ("g_dtype", C.c_int32), ("reserved", C.c_int32),
+        ("w", C.POINTER(C.c_void_p)), ("g", C.POINTER(C.c_void_p)), ("m", C.POINTER(C.c_void_p)),
+        ("ld_w", C.c_int64), ("ld_g", C.c_int64), ("ld_m", C.c_int64),
+    ]
+
+
+class muon_hparams(C.Structure):
+    _fields_ = [
+        ("lr", C.c_float), ("wd", C.c_float), ("mu", C.c_float),
+        ("nesterov", C.c_int32), ("ns_steps", C.c_int32),
+        ("a", C.c_float), ("b", C.c_float), ("c", C.c_float),
+        ("eps", C.c_float), ("rms_scale", C.c_float),
+    ]
+
+
+class MuonError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__("muon error %d: %s" % (code, msg))
+        self.code = code
+
+
+_lib = None
+
+
+def lib():
+    """Load libmuon_b200.so (once).  There is no fallback: a missing library
+    is an error."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "libmuon_b200.so is not built (%s); run `python -m paper_2502_16982_b200.build`" % LIB_PATH)
+    L = C.CDLL(LIB_PATH)
+    L.muon_workspace_bytes.argtypes = [C.POINTER(muon_group), C.c_int, C.POINTER(C.c_size_t)]
+    L.muon_init.argtypes = [C.POINTER(C.c_void_p), C.POINTER(muon_group), C.c_int, C.c_void_p, C.c_size_t, C.c_int]
+    L.muon_step.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_void_p]
+    L.muon_step_host.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.POINTER(C.POINTER(C.c_void_p)),
+                                 C.POINTER(C.POINTER(C.c_void_p)), C.c_void_p]
+    L.muon_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+    L.muon_get_norms.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_float), C.c_int]
+    L.muon_destroy.argtypes = [C.c_void_p]
+    L.muon_last_error.restype = C.c_char_p
+    L.muon_last_launch_count.argtypes = [C.c_void_p]
+    L.muon_debug_keep.argtypes = [C.c_void_p, C.c_int]
+    L.muon_debug_read.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
+    L.muon_debug_set_variant.argtypes = [C.c_int]
+    for name in EXPORTED:
+        if name != "muon_last_error":
+            getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def _check(rc):
+    if rc != 0:
+        raise MuonError(rc, lib().muon_last_error().decode())
+
+
+def muon_last_error() -> str:
+    return lib().muon_last_error().decode()
+
+
+@dataclass
+class Hyper:
+    """Hyper-parameters of one step; defaults are the paper's."""
+    lr: float = 2e-2
+    wd: float = 0.1
+    mu: float = 0.95
+    nesterov: bool = True
+    ns_steps: int = 5
+    a: float = 3.4445
+    b: float = -4.7750
+    c: float = 2.0315
+    eps: float = 1e-7
+    rms_scale: float = 0.2
+
+    def to_c(self) -> muon_hparams:
+        return muon_hparams(self.lr, self.wd, self.mu, int(bool(self.nesterov)), int(self.ns_steps),
+                            self.a, self.b, self.c, self.eps, self.rms_scale)
+
+
+def _dtype_code(t):
+    import torch
+    if t.dtype == torch.bfloat16:
+        return MUON_DTYPE_BF16
+    if t.dtype == torch.float32:
+        return MUON_DTYPE_FP32
+    raise MuonError(MUON_ERR_UNSUPPORTED, "dtype %s" % t.dtype)
+
+
+class _GroupArrays:
+    """Keeps the ctypes arrays of one param group alive."""
+
+    def __init__(self, ws, gs, ms):
+        w0, g0, m0 = ws[0], gs[0], ms[0]
+        n = len(ws)
+        for t in list(ws) + list(gs) + list(ms):
+            if t.dim() != 2 or t.shape != w0.shape or t.stride(1) != 1:
+                raise MuonError(MUON_ERR_INVALID_ARG, "matrices of a group must be 2-D, equal-shaped, rows contiguous")
+        for seq, ref in ((ws, w0), (gs, g0), (ms, m0)):
+            for t in seq:
+                if t.dtype != ref.dtype or t.stride(0) != ref.stride(0):
+                    raise MuonError(MUON_ERR_INVALID_ARG, "dtype and row stride must be uniform within a group")
+        self.w = (C.c_void_p * n)(*[t.data_ptr() for t in ws])
+        self.g = (C.c_void_p * n)(*[t.data_ptr() for t in gs])
+        self.m = (C.c_void_p * n)(*[t.data_ptr() for t in ms])
+        self.desc = muon_group(
+            w0.shape[0], w0.shape[1], n, _dtype_code(w0), _dtype_code(g0), 0,
+            C.cast(self.w, C.POINTER(C.c_void_p)), C.cast(self.g, C.POINTER(C.c_void_p)),
+            C.cast(self.m, C.POINTER(C.c_void_p)),
+            w0.stride(0) if w0.shape[0] > 1 else max(w0.stride(0), w0.shape[1]),
+            g0.stride(0) if g0.shape[0] > 1 else max(g0.stride(0), g0.shape[1]),
+            m0.stride(0) if m0.shape[0] > 1 else max(m0.stride(0), m0.shape[1]))
+
+
+def shape_only_groups(shapes) -> "C.Array":
+    """muon_group array carrying only (rows, cols, count, w_dtype, g_dtype)
+    for muon_workspace_bytes."""
+    arr = (muon_group * len(shapes))()
+    for i, (rows, cols, count, wd, gd) in enumerate(shapes):
+        arr[i].rows, arr[i].cols, arr[i].count, arr[i].w_dtype, arr[i].g_dtype = rows, cols, count, wd, gd
+    return arr
+
+
+def muon_workspace_bytes(groups_c, n_groups) -> int:
+    out = C.c_size_t(0)
+    _check(lib().muon_workspace_bytes(groups_c, n_groups, C.byref(out)))
+    return out.value
+
+
+def muon_debug_set_variant(variant: int) -> int:
+    return lib().muon_debug_set_variant(int(variant))
+
+
+class MuonContext:
+    """One initialised set of param groups.
+
+    ``groups`` is a list of (weights, grads, momenta) triples; each entry of a
+    triple is a list of equal-shaped 2-D CUDA tensors (bf16 or fp32 weights and
+    gradients, fp32 momenta).  Tensors must outlive the context.
+    """
+
+    def __init__(self, groups: Sequence[Sequence[Sequence["torch.Tensor"]]], device: Optional[int] = None):
+        import torch
+        if not torch.cuda.is_available():
+            raise MuonError(MUON_ERR_CUDA, "no CUDA device: this library has no CPU path")
+        L = lib()
+        self._arrays: List[_GroupArrays] = [_GroupArrays(ws, gs, ms) for ws, gs, ms in groups]
+        self._tensors = groups
+        n = len(self._arrays)
+        self._groups_c = (muon_group * n)(*[a.desc for a in self._arrays])
+        self.n_groups = n
+        self.n_matrices = sum(a.desc.count for a in self._arrays)
+        dev = groups[0][0][0].device
+        self.device = dev.index if device is None else device
+        nbytes = muon_workspace_bytes(self._groups_c, n)
+        self.workspace_bytes = nbytes
+        self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 1023) // 1024 * 1024
+        ctx = C.c_void_p()
+        _check(L.muon_init(C.byref(ctx), self._groups_c, n, C.c_void_p(self._ws_ptr), nbytes, self.device))
+        self._ctx = ctx
+
+    # -- the C calls -------------------------------------------------------
+    def muon_step(self, hp: Hyper, stream=None):
+        import torch
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        c_hp = hp.to_c()
+        _check(lib().muon_step(self._ctx, C.byref(c_hp), C.c_void_p(s.cuda_stream)))
+
+    def muon_step_host(self, hp: Hyper, g_host, w_host=None, stream=None):
+        """g_host / w_host: per group, a list of pinned CPU tensors (dense)."""
+        import torch
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        c_hp = hp.to_c()
+
+        def table(host):
+            rows = [(C.c_void_p * len(ts))(*[t.data_ptr() for t in ts]) for ts in host]
+            tab = (C.POINTER(C.c_void_p) * len(rows))(*[C.cast(r, C.POINTER(C.c_void_p)) for r in rows])
+            return rows, tab
+
+        g_rows, g_tab = table(g_host)
+        w_tab = None
+        if w_host is not None:
+            w_rows, w_tab = table(w_host)
+        _check(lib().muon_step_host(self._ctx, C.byref(c_hp), g_tab, w_tab, C.c_void_p(s.cuda_stream)))
+
+    def muon_status(self, stream=None):
+        """Synchronises the stream; returns (status_code, matrix_index)."""
+        import torch
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        st, mi = C.c_int(0), C.c_int(-1)
+        _check(lib().muon_status(self._ctx, C.c_void_p(s.cuda_stream), C.byref(st), C.byref(mi)))
+        return st.value, mi.value
+
+    def muon_get_norms(self, stream=None):
+        import torch
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        out = (C.c_float * self.n_matrices)()
+        _check(lib().muon_get_norms(self._ctx, C.c_void_p(s.cuda_stream), out, self.n_matrices))
+        return list(out)
+
+    def muon_last_launch_count(self) -> int:
+        return lib().muon_last_launch_count(self._ctx)
+
+    def muon_debug_keep(self, keep: bool):
+        _check(lib().muon_debug_keep(self._ctx, int(keep)))
+
+    def muon_debug_read(self, matrix_index: int, which: int, rows: int, cols: int):
+        """Returns a CPU bf16 tensor rows x cols (short side first)."""
+        import torch
+        out = torch.empty((rows, cols), dtype=torch.bfloat16)
+        _check(lib().muon_debug_read(self._ctx, matrix_index, which, C.c_void_p(out.data_ptr()), out.numel() * 2))
+        return out
+
+    def muon_destroy(self):
+        if getattr(self, "_ctx", None) is not None and self._ctx:
+            lib().muon_destroy(self._ctx)
+            self._ctx = None
+
+    def __del__(self):
+        try:
+            self.muon_destroy()
+        except Exception:
+            pass

@@ -1,0 +1,644 @@
+// Host side of the Muon step library: descriptor validation, shape-bucket
+// planner, workspace carving, TMA descriptor encoding, launch sequencing and
+// the C ABI declared in include/muon.h.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "../../include/muon.h"
+#include "internal.h"
+
+namespace muon {
+
+cudaError_t launch_momentum_cast(const StreamParams& P, bool grad_fp32, cudaStream_t stream);
+cudaError_t launch_norm_finalise(const float* partials, int tiles_per_matrix, int count, float eps,
+                                 const MatDesc* descs, MatScal* scal, float* norms, DevStatus* status,
+                                 cudaStream_t stream);
+cudaError_t launch_update_noiter(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
+                                 long long x_stride, int ldx, int count, long long elems,
+                                 float upd_scale, float decay, bool w_fp32, cudaStream_t stream);
+cudaError_t gemm_configure();
+cudaError_t launch_ns_gemm(const GemmParams& P, int num_sms, cudaStream_t stream);
+
+namespace {
+
+thread_local std::string g_last_error;
+int g_default_variant = 0;  // 0: MN-major B operand, 1: transposed copy (K-major)
+
+int fail(int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  g_last_error = buf;
+  return code;
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Upper bound on the Newton-Schulz operand bytes of one chunk; larger buckets
+// are processed in several chunks that reuse the same workspace.
+constexpr size_t kChunkBytesMax = size_t(8) << 30;
+constexpr int kChunkCountMax = 4096;
+
+struct MatRef {
+  int group, index, global;
+};
+
+struct Bucket {
+  int m, n;  // short side, long side
+  int w_dtype, g_dtype;
+  std::vector<MatRef> mats;
+  int chunk;        // matrices per chunk
+  int ldx, ldxt, lda;
+  size_t x_stride, xt_stride, a_stride;  // elements per matrix
+  int stream_tiles;                      // CTAs per matrix of the streaming kernel
+  // workspace offsets (bytes) of the chunk buffers
+  size_t off_x[2], off_xt[2], off_a, off_b, off_partials, off_scal, off_descs;
+  // tensor maps over the chunk buffers
+  CUtensorMap x_op[2];    // X as K-major operand / tile input / tile output: box {64,128} swizzled
+  CUtensorMap x_mn[2];    // X as MN-major operand: box {64,64} swizzled
+  CUtensorMap xt_op[2];   // X^T as K-major operand: box {64,128} swizzled
+  CUtensorMap xt_out[2];  // X^T as transposed output: box {128,128} plain
+  CUtensorMap a_op, b_op;      // A, B: box {64,128} swizzled
+  CUtensorMap a_out_t, b_out_t;  // A, B mirrored output: box {128,128} plain
+};
+
+struct PlanSizes {
+  size_t total;
+  size_t off_status;
+  size_t off_norms;  // float per matrix (global order)
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess) {
+    return nullptr;
+  }
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+// 3-D bf16 map over [count][rows][cols] with row pitch `ld` elements.
+int encode_map(CUtensorMap* out, void* base, int cols, int rows, int count, int ld,
+               size_t mat_stride_elems, int box_x, int box_y, bool swizzle128) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return fail(MUON_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
+  cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows),
+                        static_cast<cuuint64_t>(count)};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld) * 2, static_cast<cuuint64_t>(mat_stride_elems) * 2};
+  cuuint32_t box[3] = {static_cast<cuuint32_t>(box_x), static_cast<cuuint32_t>(box_y), 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(MUON_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return MUON_OK;
+}
+
+int validate_groups(const muon_group* groups, int n_groups, bool need_ptrs) {
+  if (!groups || n_groups <= 0) return fail(MUON_ERR_INVALID_ARG, "groups is null or n_groups <= 0");
+  for (int g = 0; g < n_groups; ++g) {
+    const muon_group& G = groups[g];
+    if (G.rows <= 0 || G.cols <= 0 || G.count <= 0)
+      return fail(MUON_ERR_INVALID_ARG, "group %d: rows, cols and count must be positive", g);
+    if (G.rows > 65536 || G.cols > 65536)
+      return fail(MUON_ERR_UNSUPPORTED, "group %d: dimensions above 65536 are not supported", g);
+    if ((G.w_dtype != MUON_DTYPE_BF16 && G.w_dtype != MUON_DTYPE_FP32) ||
+        (G.g_dtype != MUON_DTYPE_BF16 && G.g_dtype != MUON_DTYPE_FP32))
+      return fail(MUON_ERR_UNSUPPORTED, "group %d: dtype must be bf16 or fp32", g);
+    if (!need_ptrs) continue;
+    if (!G.w || !G.g || !G.m) return fail(MUON_ERR_INVALID_ARG, "group %d: null pointer array", g);
+    if (G.ld_w < G.cols || G.ld_g < G.cols || G.ld_m < G.cols)
+      return fail(MUON_ERR_INVALID_ARG, "group %d: leading dimension smaller than cols", g);
+    for (int i = 0; i < G.count; ++i) {
+      if (!G.w[i] || !G.g[i] || !G.m[i])
+        return fail(MUON_ERR_INVALID_ARG, "group %d matrix %d: null device pointer", g, i);
+      const uintptr_t wa = G.w_dtype == MUON_DTYPE_FP32 ? 3 : 1, ga = G.g_dtype == MUON_DTYPE_FP32 ? 3 : 1;
+      if ((reinterpret_cast<uintptr_t>(G.w[i]) & wa) || (reinterpret_cast<uintptr_t>(G.g[i]) & ga) ||
+          (reinterpret_cast<uintptr_t>(G.m[i]) & 3))
+        return fail(MUON_ERR_ALIGNMENT, "group %d matrix %d: pointer not aligned to its element size", g, i);
+      if (G.w[i] == G.g[i] || G.w[i] == (void*)G.m[i] || G.g[i] == (const void*)G.m[i])
+        return fail(MUON_ERR_INVALID_ARG, "group %d matrix %d: W, G and M must not alias", g, i);
+    }
+  }
+  return MUON_OK;
+}
+
+// Forms the shape buckets and lays out the workspace.  Deterministic in the
+// group list, so muon_workspace_bytes and muon_init agree.
+int make_plan(const muon_group* groups, int n_groups, int variant, std::vector<Bucket>* buckets,
+              PlanSizes* sizes, int* total_mats) {
+  std::map<std::tuple<int, int, int, int>, int> index;
+  buckets->clear();
+  int global = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    const muon_group& G = groups[g];
+    const int m = std::min(G.rows, G.cols), n = std::max(G.rows, G.cols);
+    auto key = std::make_tuple(m, n, G.w_dtype, G.g_dtype);
+    auto it = index.find(key);
+    int b;
+    if (it == index.end()) {
+      b = static_cast<int>(buckets->size());
+      index[key] = b;
+      Bucket nb{};
+      nb.m = m;
+      nb.n = n;
+      nb.w_dtype = G.w_dtype;
+      nb.g_dtype = G.g_dtype;
+      buckets->push_back(nb);
+    } else {
+      b = it->second;
+    }
+    for (int i = 0; i < G.count; ++i) (*buckets)[b].mats.push_back(MatRef{g, i, global++});
+  }
+  *total_mats = global;
+
+  // Chunk buffers are shared by all buckets (they run one after another), so
+  // the workspace is the maximum over buckets, not the sum.
+  size_t chunk_region = 0;
+  for (Bucket& B : *buckets) {
+    B.ldx = static_cast<int>(align_up(B.n, 64));
+    B.ldxt = static_cast<int>(align_up(B.m, 64));
+    B.lda = static_cast<int>(align_up(B.m, 64));
+    B.x_stride = static_cast<size_t>(B.m) * B.ldx;
+    B.xt_stride = static_cast<size_t>(B.n) * B.ldxt;
+    B.a_stride = static_cast<size_t>(B.m) * B.lda;
+    // tile counts of the streaming kernel for both stored orientations
+    const int t1 = ceil_div(B.m, kSTR) * ceil_div(B.n, kSTC);
+    const int t2 = ceil_div(B.n, kSTR) * ceil_div(B.m, kSTC);
+    B.stream_tiles = std::max(t1, t2);
+    size_t per_mat = 2 * B.x_stride * 2 + 2 * B.a_stride * 2;
+    if (variant == 1) per_mat += 2 * B.xt_stride * 2;
+    size_t chunk = std::max<size_t>(1, kChunkBytesMax / per_mat);
+    chunk = std::min<size_t>(chunk, B.mats.size());
+    chunk = std::min<size_t>(chunk, kChunkCountMax);
+    // keep the streaming grid within 2^31 CTAs
+    while (chunk > 1 && chunk * static_cast<size_t>(B.stream_tiles) > (size_t(1) << 30)) chunk /= 2;
+    B.chunk = static_cast<int>(chunk);
+    size_t off = 0;
+    auto take = [&off](size_t bytes) {
+      size_t o = off;
+      off = align_up(off + bytes, 1024);
+      return o;
+    };
+    B.off_x[0] = take(chunk * B.x_stride * 2);
+    B.off_x[1] = take(chunk * B.x_stride * 2);
+    if (variant == 1) {
+      B.off_xt[0] = take(chunk * B.xt_stride * 2);
+      B.off_xt[1] = take(chunk * B.xt_stride * 2);
+    } else {
+      B.off_xt[0] = B.off_xt[1] = 0;
+    }
+    B.off_a = take(chunk * B.a_stride * 2);
+    B.off_b = take(chunk * B.a_stride * 2);
+    B.off_partials = take(chunk * static_cast<size_t>(B.stream_tiles) * sizeof(float));
+    B.off_scal = take(chunk * sizeof(MatScal));
+    chunk_region = std::max(chunk_region, off);
+  }
+  size_t off = align_up(chunk_region, 1024);
+  // persistent region: descriptors of every matrix (bucket by bucket), status, norms
+  for (Bucket& B : *buckets) {
+    B.off_descs = off;
+    off = align_up(off + B.mats.size() * sizeof(MatDesc), 1024);
+  }
+  sizes->off_status = off;
+  off = align_up(off + sizeof(DevStatus), 1024);
+  sizes->off_norms = off;
+  off = align_up(off + static_cast<size_t>(global) * sizeof(float), 1024);
+  sizes->total = off;
+  return MUON_OK;
+}
+
+}  // namespace
+}  // namespace muon
+
+using namespace muon;
+
+struct muon_ctx {
+  int device;
+  int num_sms;
+  int variant;
+  int keep_o;
+  int last_launches;
+  uint8_t* ws;
+  size_t ws_bytes;
+  std::vector<muon_group> groups;            // copies (pointer arrays re-owned below)
+  std::vector<std::vector<void*>> w_ptrs;    // per group
+  std::vector<std::vector<const void*>> g_ptrs;
+  std::vector<std::vector<float*>> m_ptrs;
+  std::vector<Bucket> buckets;
+  PlanSizes sizes;
+  int total_mats;
+  // where each global matrix lives: bucket and position
+  std::vector<std::pair<int, int>> where;
+  // debug taps: which X buffer holds X0 / the last X per bucket
+  std::vector<int> x0_buf, xlast_buf;
+};
+
+extern "C" {
+
+const char* muon_last_error(void) { return g_last_error.c_str(); }
+
+int muon_debug_set_variant(int variant) {
+  int prev = g_default_variant;
+  if (variant == 0 || variant == 1) g_default_variant = variant;
+  return prev;
+}
+
+int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_bytes) {
+  if (!out_bytes) return fail(MUON_ERR_INVALID_ARG, "out_bytes is null");
+  int rc = validate_groups(groups, n_groups, false);
+  if (rc) return rc;
+  std::vector<Bucket> buckets;
+  PlanSizes sizes;
+  int total;
+  rc = make_plan(groups, n_groups, g_default_variant, &buckets, &sizes, &total);
+  if (rc) return rc;
+  *out_bytes = sizes.total;
+  return MUON_OK;
+}
+
+int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* workspace,
+              size_t workspace_bytes, int device) {
+  if (!out_ctx) return fail(MUON_ERR_INVALID_ARG, "out_ctx is null");
+  *out_ctx = nullptr;
+  int rc = validate_groups(groups, n_groups, true);
+  if (rc) return rc;
+  if (!workspace) return fail(MUON_ERR_WORKSPACE, "workspace is null");
+  if (reinterpret_cast<uintptr_t>(workspace) & 1023)
+    return fail(MUON_ERR_WORKSPACE, "workspace must be 1024-byte aligned");
+
+  muon_ctx* ctx = new (std::nothrow) muon_ctx();
+  if (!ctx) return fail(MUON_ERR_INVALID_ARG, "out of host memory");
+  ctx->device = device;
+  ctx->variant = g_default_variant;
+  ctx->keep_o = 0;
+  ctx->last_launches = 0;
+  ctx->ws = static_cast<uint8_t*>(workspace);
+  ctx->ws_bytes = workspace_bytes;
+  rc = make_plan(groups, n_groups, ctx->variant, &ctx->buckets, &ctx->sizes, &ctx->total_mats);
+  if (rc) { delete ctx; return rc; }
+  if (workspace_bytes < ctx->sizes.total) {
+    const size_t need = ctx->sizes.total;
+    delete ctx;
+    return fail(MUON_ERR_WORKSPACE, "workspace too small: need %zu bytes, got %zu", need, workspace_bytes);
+  }
+
+  cudaError_t ce = cudaSetDevice(device);
+  if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce)); }
+  cudaDeviceProp prop;
+  ce = cudaGetDeviceProperties(&prop, device);
+  if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "cudaGetDeviceProperties: %s", cudaGetErrorString(ce)); }
+  if (prop.major != 10) {
+    delete ctx;
+    return fail(MUON_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a only", device,
+                prop.major, prop.minor);
+  }
+  ctx->num_sms = prop.multiProcessorCount;
+  ce = gemm_configure();
+  if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ce)); }
+
+  // own copies of the descriptor arrays
+  ctx->groups.assign(groups, groups + n_groups);
+  ctx->w_ptrs.resize(n_groups);
+  ctx->g_ptrs.resize(n_groups);
+  ctx->m_ptrs.resize(n_groups);
+  for (int g = 0; g < n_groups; ++g) {
+    ctx->w_ptrs[g].assign(groups[g].w, groups[g].w + groups[g].count);
+    ctx->g_ptrs[g].assign(groups[g].g, groups[g].g + groups[g].count);
+    ctx->m_ptrs[g].assign(groups[g].m, groups[g].m + groups[g].count);
+    ctx->groups[g].w = ctx->w_ptrs[g].data();
+    ctx->groups[g].g = ctx->g_ptrs[g].data();
+    ctx->groups[g].m = ctx->m_ptrs[g].data();
+  }
+  ctx->where.assign(ctx->total_mats, std::make_pair(-1, -1));
+  ctx->x0_buf.assign(ctx->buckets.size(), 0);
+  ctx->xlast_buf.assign(ctx->buckets.size(), 0);
+
+  // per-bucket: upload matrix descriptors, encode tensor maps
+  for (size_t b = 0; b < ctx->buckets.size(); ++b) {
+    Bucket& B = ctx->buckets[b];
+    std::vector<MatDesc> descs(B.mats.size());
+    for (size_t i = 0; i < B.mats.size(); ++i) {
+      const MatRef& r = B.mats[i];
+      const muon_group& G = ctx->groups[r.group];
+      MatDesc d{};
+      d.w = G.w[r.index];
+      d.g = G.g[r.index];
+      d.m = G.m[r.index];
+      d.ld_w = G.ld_w;
+      d.ld_g = G.ld_g;
+      d.ld_m = G.ld_m;
+      d.rows = G.rows;
+      d.cols = G.cols;
+      d.transposed = G.rows > G.cols ? 1 : 0;
+      d.global_index = r.global;
+      const bool ptr16 = ((reinterpret_cast<uintptr_t>(d.w) | reinterpret_cast<uintptr_t>(d.g) |
+                           reinterpret_cast<uintptr_t>(d.m)) & 15) == 0;
+      d.vec_ok = (ptr16 && G.ld_w % 8 == 0 && G.ld_g % 8 == 0 && G.ld_m % 8 == 0) ? 1 : 0;
+      descs[i] = d;
+      ctx->where[r.global] = std::make_pair(static_cast<int>(b), static_cast<int>(i));
+    }
+    ce = cudaMemcpy(ctx->ws + B.off_descs, descs.data(), descs.size() * sizeof(MatDesc), cudaMemcpyHostToDevice);
+    if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "descriptor upload: %s", cudaGetErrorString(ce)); }
+
+    for (int p = 0; p < 2 && rc == MUON_OK; ++p) {
+      void* xb = ctx->ws + B.off_x[p];
+      rc = encode_map(&B.x_op[p], xb, B.n, B.m, B.chunk, B.ldx, B.x_stride, 64, 128, true);
+      if (rc == MUON_OK) rc = encode_map(&B.x_mn[p], xb, B.n, B.m, B.chunk, B.ldx, B.x_stride, 64, 64, true);
+      if (ctx->variant == 1 && rc == MUON_OK) {
+        void* xtb = ctx->ws + B.off_xt[p];
+        rc = encode_map(&B.xt_op[p], xtb, B.m, B.n, B.chunk, B.ldxt, B.xt_stride, 64, 128, true);
+        if (rc == MUON_OK) rc = encode_map(&B.xt_out[p], xtb, B.m, B.n, B.chunk, B.ldxt, B.xt_stride, 128, 128, false);
+      }
+    }
+    void* ab = ctx->ws + B.off_a;
+    void* bb = ctx->ws + B.off_b;
+    if (rc == MUON_OK) rc = encode_map(&B.a_op, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 128, true);
+    if (rc == MUON_OK) rc = encode_map(&B.a_out_t, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 128, false);
+    if (rc == MUON_OK) rc = encode_map(&B.b_op, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 128, true);
+    if (rc == MUON_OK) rc = encode_map(&B.b_out_t, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 128, false);
+    if (rc != MUON_OK) { delete ctx; return rc; }
+  }
+  ce = cudaMemset(ctx->ws + ctx->sizes.off_status, 0, sizeof(DevStatus));
+  if (ce == cudaSuccess) {
+    DevStatus init{0, -1};
+    ce = cudaMemcpy(ctx->ws + ctx->sizes.off_status, &init, sizeof(init), cudaMemcpyHostToDevice);
+  }
+  if (ce == cudaSuccess) ce = cudaMemset(ctx->ws + ctx->sizes.off_norms, 0, ctx->total_mats * sizeof(float));
+  if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "workspace init: %s", cudaGetErrorString(ce)); }
+  *out_ctx = ctx;
+  return MUON_OK;
+}
+
+static int check_hparams(const muon_hparams* hp) {
+  if (!hp) return fail(MUON_ERR_INVALID_ARG, "hparams is null");
+  if (hp->ns_steps < 0 || hp->ns_steps > 64) return fail(MUON_ERR_INVALID_ARG, "ns_steps must be in [0, 64]");
+  if (!(hp->eps >= 0.f)) return fail(MUON_ERR_INVALID_ARG, "eps must be >= 0");
+  if (!std::isfinite(hp->lr) || !std::isfinite(hp->wd) || !std::isfinite(hp->mu) || !std::isfinite(hp->a) ||
+      !std::isfinite(hp->b) || !std::isfinite(hp->c) || !std::isfinite(hp->rms_scale))
+    return fail(MUON_ERR_INVALID_ARG, "hyper-parameters must be finite");
+  return MUON_OK;
+}
+
+int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
+  if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
+  int rc = check_hparams(hp);
+  if (rc) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  int launches = 0;
+  cudaError_t ce = cudaSuccess;
+  DevStatus* status = reinterpret_cast<DevStatus*>(ctx->ws + ctx->sizes.off_status);
+  float* norms = reinterpret_cast<float*>(ctx->ws + ctx->sizes.off_norms);
+
+  for (size_t b = 0; b < ctx->buckets.size(); ++b) {
+    Bucket& B = ctx->buckets[b];
+    const int total = static_cast<int>(B.mats.size());
+    const float upd_scale = -hp->lr * hp->rms_scale * std::sqrt(static_cast<float>(B.n));
+    const float decay = 1.0f - hp->lr * hp->wd;
+    for (int first = 0; first < total; first += B.chunk) {
+      const int count = std::min(B.chunk, total - first);
+      const MatDesc* descs = reinterpret_cast<const MatDesc*>(ctx->ws + B.off_descs) + first;
+      MatScal* scal = reinterpret_cast<MatScal*>(ctx->ws + B.off_scal);
+      float* partials = reinterpret_cast<float*>(ctx->ws + B.off_partials);
+
+      StreamParams S{};
+      S.descs = descs;
+      S.partials = partials;
+      S.x = reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_x[0]);
+      S.xt = ctx->variant == 1 ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_xt[0]) : nullptr;
+      S.x_stride = static_cast<long long>(B.x_stride);
+      S.xt_stride = static_cast<long long>(B.xt_stride);
+      S.ldx = B.ldx;
+      S.ldxt = B.ldxt;
+      S.count = count;
+      S.tiles_per_matrix = B.stream_tiles;
+      S.mu = hp->mu;
+      S.nesterov = hp->nesterov ? 1 : 0;
+      ce = launch_momentum_cast(S, B.g_dtype == MUON_DTYPE_FP32, stream);
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "momentum kernel launch: %s", cudaGetErrorString(ce));
+      ++launches;
+      ce = launch_norm_finalise(partials, B.stream_tiles, count, hp->eps, descs, scal, norms, status, stream);
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "norm kernel launch: %s", cudaGetErrorString(ce));
+      ++launches;
+
+      int cur = 0;
+      if (hp->ns_steps == 0) {
+        ce = launch_update_noiter(descs, scal, S.x, S.x_stride, B.ldx, count,
+                                  static_cast<long long>(B.m) * B.n, upd_scale, decay,
+                                  B.w_dtype == MUON_DTYPE_FP32, stream);
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "update kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
+      }
+      const int nb = ceil_div(B.m, kBM);
+      for (int it = 0; it < hp->ns_steps; ++it) {
+        const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
+        const int nxt = cur ^ 1;
+        GemmParams P{};
+        P.descs = descs;
+        P.scal = scal;
+        P.status = status;
+        P.count = count;
+        P.upd_scale = upd_scale;
+        P.decay = decay;
+        P.w_fp32 = B.w_dtype == MUON_DTYPE_FP32;
+
+        // A = X X^T (first iteration: times s^2, the deferred normalisation)
+        P.mode = kGram;
+        P.map_a = B.x_op[cur];
+        P.map_b = B.x_op[cur];
+        P.map_in = B.a_op;
+        P.map_out = B.a_op;
+        P.map_out_t = B.a_out_t;
+        P.out_rows = B.m; P.out_cols = B.m; P.k = B.n;
+        P.nb_i = nb; P.nb_j = nb; P.tiles_per_matrix = nb * (nb + 1) / 2;
+        P.symmetric = 1; P.has_in = 0; P.write_direct = 1; P.write_t = 1;
+        P.scale_kind = first_it ? 1 : 0;
+        P.last = 0; P.b_mn_major = 0;
+        P.c_acc = 1.f; P.c_in = 0.f;
+        ce = launch_ns_gemm(P, ctx->num_sms, stream);
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
+
+        // B = b*A + c*A*A^T
+        P.mode = kPoly;
+        P.map_a = B.a_op;
+        P.map_b = B.a_op;
+        P.map_in = B.a_op;
+        P.map_out = B.b_op;
+        P.map_out_t = B.b_out_t;
+        P.k = B.m;
+        P.has_in = 1;
+        P.scale_kind = 0;
+        P.c_acc = hp->c; P.c_in = hp->b;
+        ce = launch_ns_gemm(P, ctx->num_sms, stream);
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
+
+        // X' = a*X + B*X (first iteration: times s); last iteration updates W
+        P.mode = kComb;
+        P.map_a = B.b_op;
+        if (ctx->variant == 1) {
+          P.map_b = B.xt_op[cur];
+          P.b_mn_major = 0;
+        } else {
+          P.map_b = B.x_mn[cur];
+          P.b_mn_major = 1;
+        }
+        P.map_in = B.x_op[cur];
+        P.map_out = B.x_op[nxt];
+        P.map_out_t = ctx->variant == 1 ? B.xt_out[nxt] : B.x_op[nxt];
+        P.out_rows = B.m; P.out_cols = B.n; P.k = B.m;
+        P.nb_i = nb; P.nb_j = ceil_div(B.n, kBN); P.tiles_per_matrix = P.nb_i * P.nb_j;
+        P.symmetric = 0; P.has_in = 1;
+        P.write_direct = last_it ? (ctx->keep_o ? 1 : 0) : 1;
+        P.write_t = (!last_it && ctx->variant == 1) ? 1 : 0;
+        P.scale_kind = first_it ? 2 : 0;
+        P.last = last_it ? 1 : 0;
+        P.c_acc = 1.f; P.c_in = hp->a;
+        ce = launch_ns_gemm(P, ctx->num_sms, stream);
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
+        cur = nxt;
+      }
+      ctx->x0_buf[b] = 0;
+      ctx->xlast_buf[b] = cur;
+    }
+  }
+  ctx->last_launches = launches;
+  return MUON_OK;
+}
+
+int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* const* g_host,
+                   void* const* const* w_host, void* stream_v) {
+  if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
+  if (!g_host) return fail(MUON_ERR_INVALID_ARG, "g_host is null");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  for (size_t g = 0; g < ctx->groups.size(); ++g) {
+    const muon_group& G = ctx->groups[g];
+    const size_t es = G.g_dtype == MUON_DTYPE_FP32 ? 4 : 2;
+    for (int i = 0; i < G.count; ++i) {
+      cudaError_t ce = cudaMemcpy2DAsync(const_cast<void*>(G.g[i]), G.ld_g * es, g_host[g][i], G.cols * es,
+                                         G.cols * es, G.rows, cudaMemcpyHostToDevice, stream);
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gradient upload: %s", cudaGetErrorString(ce));
+    }
+  }
+  int rc = muon_step(ctx, hp, stream_v);
+  if (rc) return rc;
+  if (w_host) {
+    for (size_t g = 0; g < ctx->groups.size(); ++g) {
+      const muon_group& G = ctx->groups[g];
+      const size_t es = G.w_dtype == MUON_DTYPE_FP32 ? 4 : 2;
+      for (int i = 0; i < G.count; ++i) {
+        cudaError_t ce = cudaMemcpy2DAsync(w_host[g][i], G.cols * es, G.w[i], G.ld_w * es, G.cols * es, G.rows,
+                                           cudaMemcpyDeviceToHost, stream);
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "weight download: %s", cudaGetErrorString(ce));
+      }
+    }
+  }
+  return MUON_OK;
+}
+
+int muon_status(muon_ctx* ctx, void* stream_v, int* device_status, int* matrix_index) {
+  if (!ctx || !device_status) return fail(MUON_ERR_INVALID_ARG, "ctx or device_status is null");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  DevStatus st{0, -1};
+  cudaError_t ce = cudaMemcpyAsync(&st, ctx->ws + ctx->sizes.off_status, sizeof(st), cudaMemcpyDeviceToHost, stream);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "status read: %s", cudaGetErrorString(ce));
+  *device_status = st.code;
+  if (matrix_index) *matrix_index = st.code ? st.matrix : -1;
+  if (st.code) {
+    DevStatus init{0, -1};
+    ce = cudaMemcpyAsync(ctx->ws + ctx->sizes.off_status, &init, sizeof(init), cudaMemcpyHostToDevice, stream);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "status clear: %s", cudaGetErrorString(ce));
+  }
+  return MUON_OK;
+}
+
+int muon_get_norms(muon_ctx* ctx, void* stream_v, float* out, int n) {
+  if (!ctx || !out || n < 0 || n > ctx->total_mats) return fail(MUON_ERR_INVALID_ARG, "bad arguments");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  cudaError_t ce = cudaMemcpyAsync(out, ctx->ws + ctx->sizes.off_norms, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "norm read: %s", cudaGetErrorString(ce));
+  return MUON_OK;
+}
+
+int muon_destroy(muon_ctx* ctx) {
+  delete ctx;
+  return MUON_OK;
+}
+
+int muon_last_launch_count(const muon_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+
+int muon_debug_keep(muon_ctx* ctx, int keep) {
+  if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
+  ctx->keep_o = keep ? 1 : 0;
+  return MUON_OK;
+}
+
+int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, size_t dst_bytes) {
+  if (!ctx || !dst_host) return fail(MUON_ERR_INVALID_ARG, "ctx or dst is null");
+  if (matrix_index < 0 || matrix_index >= ctx->total_mats) return fail(MUON_ERR_INVALID_ARG, "matrix index out of range");
+  const int b = ctx->where[matrix_index].first, pos = ctx->where[matrix_index].second;
+  const Bucket& B = ctx->buckets[b];
+  if (static_cast<int>(B.mats.size()) > B.chunk)
+    return fail(MUON_ERR_UNSUPPORTED, "taps need a bucket that fits one chunk");
+  const uint8_t* src;
+  int rows, cols, ld;
+  switch (which) {
+    case MUON_TAP_X0:
+      src = ctx->ws + B.off_x[ctx->x0_buf[b]] + static_cast<size_t>(pos) * B.x_stride * 2;
+      rows = B.m; cols = B.n; ld = B.ldx;
+      break;
+    case MUON_TAP_X:
+      src = ctx->ws + B.off_x[ctx->xlast_buf[b]] + static_cast<size_t>(pos) * B.x_stride * 2;
+      rows = B.m; cols = B.n; ld = B.ldx;
+      break;
+    case MUON_TAP_A:
+      src = ctx->ws + B.off_a + static_cast<size_t>(pos) * B.a_stride * 2;
+      rows = B.m; cols = B.m; ld = B.lda;
+      break;
+    case MUON_TAP_B:
+      src = ctx->ws + B.off_b + static_cast<size_t>(pos) * B.a_stride * 2;
+      rows = B.m; cols = B.m; ld = B.lda;
+      break;
+    default:
+      return fail(MUON_ERR_INVALID_ARG, "unknown tap");
+  }
+  if (dst_bytes < static_cast<size_t>(rows) * cols * 2) return fail(MUON_ERR_INVALID_ARG, "destination too small");
+  cudaError_t ce = cudaDeviceSynchronize();
+  if (ce == cudaSuccess)
+    ce = cudaMemcpy2D(dst_host, static_cast<size_t>(cols) * 2, src, static_cast<size_t>(ld) * 2,
+                      static_cast<size_t>(cols) * 2, rows, cudaMemcpyDeviceToHost);
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "tap read: %s", cudaGetErrorString(ce));
+  return MUON_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,287 @@
+// HBM-streaming kernels of the Muon step:
+//   momentum_cast_kernel : M <- mu*M + G, U = Nesterov blend or M, per-tile sum
+//                          of U^2, bf16(U) stored short side first (and, when
+//                          asked, a transposed copy)            (Sec. 2.1 rule
+//                          line 1, footnote 1, Newton-Schulz paragraph)
+//   norm_finalise_kernel : fixed-order sum of the per-tile partials ->
+//                          ||U||_F, 1/(||U||_F + eps), non-finite flag
+//   update_noiter_kernel : the weight update when ns_steps == 0 (O = X0)
+// The division by the norm is deferred: bf16(U) is stored un-normalised and the
+// scalar 1/(||U||_F+eps) is applied in fp32 by the first iteration's epilogues.
+#include <cuda_bf16.h>
+
+#include "internal.h"
+
+namespace muon {
+
+namespace {
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) {
+  return __uint_as_float(bits16 << 16);
+}
+
+template <bool kGradFp32>
+__device__ __forceinline__ void load_g8(const void* g, long long off, bool vec, int valid,
+                                        float (&out)[8]) {
+  if (kGradFp32) {
+    const float* p = reinterpret_cast<const float*>(g) + off;
+    if (vec && valid == 8) {
+      float4 a = __ldcs(reinterpret_cast<const float4*>(p));
+      float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+      out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+      out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) out[e] = e < valid ? p[e] : 0.f;
+    }
+  } else {
+    const __nv_bfloat16* p = reinterpret_cast<const __nv_bfloat16*>(g) + off;
+    if (vec && valid == 8) {
+      uint4 a = __ldcs(reinterpret_cast<const uint4*>(p));
+      out[0] = bf16_bits_to_float(a.x & 0xFFFFu); out[1] = bf16_bits_to_float(a.x >> 16);
+      out[2] = bf16_bits_to_float(a.y & 0xFFFFu); out[3] = bf16_bits_to_float(a.y >> 16);
+      out[4] = bf16_bits_to_float(a.z & 0xFFFFu); out[5] = bf16_bits_to_float(a.z >> 16);
+      out[6] = bf16_bits_to_float(a.w & 0xFFFFu); out[7] = bf16_bits_to_float(a.w >> 16);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) out[e] = e < valid ? __bfloat162float(p[e]) : 0.f;
+    }
+  }
+}
+
+// One CTA = one kSTR x kSTC (64 x 128) tile of one matrix in its stored
+// orientation.  Thread t owns 8 consecutive columns (t % 16) of rows
+// (t / 16) + 16*p, p = 0..3.
+template <bool kGradFp32>
+__global__ void __launch_bounds__(kStreamThreads)
+momentum_cast_kernel(const StreamParams P) {
+  // bf16 tile for the transposed store; +2 elements of row padding keeps the
+  // column reads off a single bank.
+  __shared__ __nv_bfloat16 tile[kSTR][kSTC + 2];
+  __shared__ float warp_sums[kStreamThreads / 32];
+
+  const int mat = blockIdx.x / P.tiles_per_matrix;
+  const int t_in = blockIdx.x - mat * P.tiles_per_matrix;
+  const MatDesc d = P.descs[mat];
+  const int tiles_c = (d.cols + kSTC - 1) / kSTC;
+  const int tiles_r = (d.rows + kSTR - 1) / kSTR;
+  float* partial = P.partials + static_cast<long long>(mat) * P.tiles_per_matrix + t_in;
+  if (t_in >= tiles_c * tiles_r) {  // padding CTA (orientations differ in tile count)
+    if (threadIdx.x == 0) *partial = 0.f;
+    return;
+  }
+  const int tr = t_in / tiles_c, tc = t_in - tr * tiles_c;
+  const int row0 = tr * kSTR, col0 = tc * kSTC;
+  const int cgrp = threadIdx.x & 15, rsub = threadIdx.x >> 4;
+  const int col = col0 + cgrp * 8;
+  const int valid = min(8, max(0, d.cols - col));
+  const bool vec = d.vec_ok != 0;
+
+  float g[4][8], m[4][8];
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    const int row = row0 + rsub + 16 * p;
+    const bool in = row < d.rows && valid > 0;
+    if (in) {
+      load_g8<kGradFp32>(d.g, static_cast<long long>(row) * d.ld_g + col, vec, valid, g[p]);
+      const float* mp = d.m + static_cast<long long>(row) * d.ld_m + col;
+      if (vec && valid == 8) {
+        float4 a = __ldcs(reinterpret_cast<const float4*>(mp));
+        float4 b = __ldcs(reinterpret_cast<const float4*>(mp) + 1);
+        m[p][0] = a.x; m[p][1] = a.y; m[p][2] = a.z; m[p][3] = a.w;
+        m[p][4] = b.x; m[p][5] = b.y; m[p][6] = b.z; m[p][7] = b.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) m[p][e] = e < valid ? mp[e] : 0.f;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { g[p][e] = 0.f; m[p][e] = 0.f; }
+    }
+  }
+
+  // Which of the two outputs is the row-major copy of the stored orientation.
+  __nv_bfloat16* direct = d.transposed ? P.xt : P.x;
+  __nv_bfloat16* transp = d.transposed ? P.x : P.xt;
+  const long long direct_stride = d.transposed ? P.xt_stride : P.x_stride;
+  const long long transp_stride = d.transposed ? P.x_stride : P.xt_stride;
+  const int ld_direct = d.transposed ? P.ldxt : P.ldx;
+  const int ld_transp = d.transposed ? P.ldx : P.ldxt;
+
+  float sumsq = 0.f;
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    const int row = row0 + rsub + 16 * p;
+    const bool in = row < d.rows && valid > 0;
+    float u[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float mn = fmaf(P.mu, m[p][e], g[p][e]);  // M_t = mu*M_{t-1} + G
+      m[p][e] = mn;
+      u[e] = P.nesterov ? fmaf(P.mu, mn, g[p][e]) : mn;  // footnote 1
+      sumsq = fmaf(u[e], u[e], sumsq);
+    }
+    __nv_bfloat162 h[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(u[2 * e], u[2 * e + 1]);
+    if (in) {
+      float* mp = d.m + static_cast<long long>(row) * d.ld_m + col;
+      if (vec && valid == 8) {
+        __stcs(reinterpret_cast<float4*>(mp), make_float4(m[p][0], m[p][1], m[p][2], m[p][3]));
+        __stcs(reinterpret_cast<float4*>(mp) + 1, make_float4(m[p][4], m[p][5], m[p][6], m[p][7]));
+      } else {
+        for (int e = 0; e < valid; ++e) mp[e] = m[p][e];
+      }
+      if (direct != nullptr) {
+        __nv_bfloat16* xp = direct + mat * direct_stride + static_cast<long long>(row) * ld_direct + col;
+        if (valid == 8) {  // workspace rows are 16-byte aligned by construction
+          *reinterpret_cast<uint4*>(xp) = *reinterpret_cast<const uint4*>(h);
+        } else {
+          const __nv_bfloat16* hs = reinterpret_cast<const __nv_bfloat16*>(h);
+          for (int e = 0; e < valid; ++e) xp[e] = hs[e];
+        }
+      }
+    }
+    if (transp != nullptr) {
+      const int lr = rsub + 16 * p;
+      __nv_bfloat162* trow = reinterpret_cast<__nv_bfloat162*>(&tile[lr][cgrp * 8]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) trow[e] = h[e];
+    }
+  }
+
+  // Block reduction of the sum of squares in a fixed order.
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sumsq += __shfl_xor_sync(0xFFFFFFFFu, sumsq, o);
+  if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = sumsq;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < kStreamThreads / 32; ++w) s += warp_sums[w];
+    *partial = s;
+  }
+
+  if (transp != nullptr) {
+    // Transposed store: output row = source column.  Each thread gathers 8
+    // source rows of one column and writes 16 bytes; 8 threads cover the 64
+    // source rows (128 bytes) of one output row.
+    __nv_bfloat16* base = transp + mat * transp_stride;
+    const int rgrp = threadIdx.x & 7;
+    for (int c = threadIdx.x >> 3; c < kSTC; c += kStreamThreads / 8) {
+      const int gcol = col0 + c;
+      if (gcol >= d.cols) break;
+      const int grow = row0 + rgrp * 8;
+      if (grow >= d.rows) continue;
+      __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = tile[rgrp * 8 + e][c];
+      __nv_bfloat16* op = base + static_cast<long long>(gcol) * ld_transp + grow;
+      const int nv = min(8, d.rows - grow);
+      if (nv == 8) {
+        *reinterpret_cast<uint4*>(op) = *reinterpret_cast<const uint4*>(v);
+      } else {
+        for (int e = 0; e < nv; ++e) op[e] = v[e];
+      }
+    }
+  }
+}
+
+// One warp per matrix: sums the per-tile partials in a fixed order (lane-strided
+// sequential accumulation, then a fixed butterfly), so the result is
+// reproducible bit for bit.
+__global__ void norm_finalise_kernel(const float* __restrict__ partials, int tiles_per_matrix,
+                                     int count, float eps, const MatDesc* __restrict__ descs,
+                                     MatScal* __restrict__ scal, float* __restrict__ norms,
+                                     DevStatus* status) {
+  const int mat = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (mat >= count) return;
+  const int lane = threadIdx.x & 31;
+  const float* p = partials + static_cast<long long>(mat) * tiles_per_matrix;
+  float s = 0.f;
+  for (int i = lane; i < tiles_per_matrix; i += 32) s += p[i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  if (lane == 0) {
+    const float nu = sqrtf(s);
+    MatScal r;
+    r.norm = nu;
+    r.nonfinite = isfinite(nu) ? 0 : 1;
+    const float inv = 1.0f / (nu + eps);
+    r.inv_norm = r.nonfinite ? 0.f : inv;
+    r.inv_norm_sq = r.nonfinite ? 0.f : inv * inv;
+    scal[mat] = r;
+    const int gidx = descs[mat].global_index;
+    norms[gidx] = nu;
+    if (r.nonfinite) {
+      if (atomicCAS(&status->code, 0, -7 /* MUON_ERR_NONFINITE */) == 0) {
+        status->matrix = gidx;
+      }
+    }
+  }
+}
+
+// ns_steps == 0: O = X0 = s * bf16(U).  W <- decay*W + upd_scale*s*X0.
+template <bool kWFp32>
+__global__ void update_noiter_kernel(const MatDesc* __restrict__ descs,
+                                     const MatScal* __restrict__ scal,
+                                     const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx,
+                                     float upd_scale, float decay) {
+  const int mat = blockIdx.y;
+  const MatDesc d = descs[mat];
+  const MatScal sc = scal[mat];
+  if (sc.nonfinite) return;
+  const long long total = static_cast<long long>(d.rows) * d.cols;
+  const __nv_bfloat16* xm = x + mat * x_stride;
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const int r = static_cast<int>(i / d.cols), c = static_cast<int>(i - static_cast<long long>(r) * d.cols);
+    const float o = sc.inv_norm * __bfloat162float(d.transposed ? xm[static_cast<long long>(c) * ldx + r]
+                                                                : xm[static_cast<long long>(r) * ldx + c]);
+    if (kWFp32) {
+      float* w = reinterpret_cast<float*>(d.w) + static_cast<long long>(r) * d.ld_w + c;
+      *w = fmaf(decay, *w, upd_scale * o);
+    } else {
+      __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(d.w) + static_cast<long long>(r) * d.ld_w + c;
+      *w = __float2bfloat16_rn(fmaf(decay, __bfloat162float(*w), upd_scale * o));
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_momentum_cast(const StreamParams& P, bool grad_fp32, cudaStream_t stream) {
+  const unsigned grid = static_cast<unsigned>(P.count) * static_cast<unsigned>(P.tiles_per_matrix);
+  if (grid == 0) return cudaSuccess;
+  if (grad_fp32) momentum_cast_kernel<true><<<grid, kStreamThreads, 0, stream>>>(P);
+  else momentum_cast_kernel<false><<<grid, kStreamThreads, 0, stream>>>(P);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_norm_finalise(const float* partials, int tiles_per_matrix, int count, float eps,
+                                 const MatDesc* descs, MatScal* scal, float* norms,
+                                 DevStatus* status, cudaStream_t stream) {
+  if (count == 0) return cudaSuccess;
+  const int warps = 4;
+  norm_finalise_kernel<<<(count + warps - 1) / warps, warps * 32, 0, stream>>>(
+      partials, tiles_per_matrix, count, eps, descs, scal, norms, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_update_noiter(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
+                                 long long x_stride, int ldx, int count, long long elems,
+                                 float upd_scale, float decay, bool w_fp32, cudaStream_t stream) {
+  if (count == 0) return cudaSuccess;
+  const int threads = 256;
+  long long bx = (elems + threads - 1) / threads;
+  if (bx > 1024) bx = 1024;
+  if (bx < 1) bx = 1;
+  dim3 grid(static_cast<unsigned>(bx), static_cast<unsigned>(count));
+  if (w_fp32)
+    update_noiter_kernel<true><<<grid, threads, 0, stream>>>(descs, scal, x, x_stride, ldx, upd_scale, decay);
+  else
+    update_noiter_kernel<false><<<grid, threads, 0, stream>>>(descs, scal, x, x_stride, ldx, upd_scale, decay);
+  return cudaGetLastError();
+}
+
+}  // namespace muon

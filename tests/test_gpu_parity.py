@@ -1,0 +1,332 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU fp64
+oracle on the same seeded inputs.
+
+Tolerances (relative Frobenius error):
+  * fp32 element-wise parts (momentum, norm):            <= 1e-5
+  * bf16 Newton-Schulz path (A, B, X stages, O, delta W): <= 2e-2
+For bf16 weights the per-step change is about one bf16 ulp of the weight, so
+the weight itself is compared with the oracle's result rounded to bf16:
+>= 99.9 % of elements within one ulp.
+"""
+
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import muon_oracle as orc
+from paper_2502_16982_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-5
+TOL_NS = 2e-2
+
+
+def _binding():
+    from paper_2502_16982_b200 import binding
+    return binding
+
+
+def rel(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    d = np.linalg.norm(a - b)
+    n = np.linalg.norm(b)
+    return d / n if n > 0 else d
+
+
+def f64(t):
+    return t.detach().cpu().to(torch.float64).numpy()
+
+
+def to_orc(hp):
+    return orc.Hyper(lr=hp.lr, wd=hp.wd, mu=hp.mu, nesterov=hp.nesterov, ns_steps=hp.ns_steps,
+                     a=hp.a, b=hp.b, c=hp.c, eps=hp.eps, rms_scale=hp.rms_scale)
+
+
+def bf16_ulp_ok_fraction(got_bf16, expect_f64):
+    """Fraction of elements of a bf16 tensor within one bf16 ulp of the
+    float64 expectation."""
+    exp_t = torch.from_numpy(expect_f64).to(torch.float32)
+    got = got_bf16.detach().cpu().to(torch.float32)
+    ulp = torch.clamp(exp_t.abs(), min=1e-30).log2().floor().exp2() * 2.0 ** -7
+    return float(((got - exp_t).abs() <= ulp * 1.0001).double().mean())
+
+
+class Case:
+    """Device tensors of some groups plus host snapshots for the oracle."""
+
+    def __init__(self, specs, seed, variant=0, zero_momentum=True):
+        b = _binding()
+        self.b = b
+        self.prev_variant = b.muon_debug_set_variant(variant)
+        self.specs = specs
+        self.dev = []
+        for gi, sp in enumerate(specs):
+            W, G, M = wl.make_group(sp, seed + gi, "cpu", zero_momentum=zero_momentum)
+            self.dev.append((W.cuda(), G.cuda(), M.cuda()))
+        self.ctx = b.MuonContext([(wl.views(W), wl.views(G), wl.views(M)) for (W, G, M) in self.dev])
+        b.muon_debug_set_variant(self.prev_variant)
+
+    def snapshot(self):
+        return [(f64(W), f64(G), f64(M)) for (W, G, M) in self.dev]
+
+    def step(self, hp):
+        self.ctx.muon_step(hp)
+        return self.ctx.muon_status()
+
+    def close(self):
+        self.ctx.muon_destroy()
+
+
+def check_step(case, hp, check_w=True, check_o=False):
+    """Runs one step and compares every matrix with the oracle.  With
+    ``check_o`` the last iteration also stores O (test tap) and O itself is
+    compared."""
+    before = case.snapshot()
+    case.ctx.muon_debug_keep(bool(check_o))
+    status, which = case.step(hp)
+    assert status == 0, (status, which)
+    norms = case.ctx.muon_get_norms()
+    gidx = 0
+    ohp = to_orc(hp)
+    for gi, sp in enumerate(case.specs):
+        W, G, M = case.dev[gi]
+        W0, G0, M0 = before[gi]
+        for i in range(sp.count):
+            ref = orc.muon_step(W0[i], G0[i], M0[i], ohp)
+            assert rel(f64(M[i]), ref["M"]) <= TOL_FP32, ("M", gi, i)
+            assert abs(norms[gidx] - ref["nu"]) <= TOL_FP32 * ref["nu"] + 1e-30, ("nu", gi, i)
+            if check_o and hp.ns_steps > 0:
+                m, n = min(sp.rows, sp.cols), max(sp.rows, sp.cols)
+                o_gpu = f64(case.ctx.muon_debug_read(gidx, case.b.MUON_TAP_X, m, n))
+                o_ref = ref["O"].T if sp.rows > sp.cols else ref["O"]
+                assert rel(o_gpu, o_ref) <= TOL_NS, ("O", gi, i, rel(o_gpu, o_ref))
+            if check_w:
+                dW_ref = ref["W"] - W0[i]
+                if sp.w_dtype == torch.float32:
+                    assert rel(f64(W[i]) - W0[i], dW_ref) <= TOL_NS, ("dW", gi, i, rel(f64(W[i]) - W0[i], dW_ref))
+                else:
+                    frac = bf16_ulp_ok_fraction(W[i], ref["W"])
+                    assert frac >= 0.999, ("W ulp", gi, i, frac)
+            gidx += 1
+
+
+HP = None
+
+
+def default_hp(**kw):
+    b = _binding()
+    return b.Hyper(**kw)
+
+
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("variant", [0, 1])
+def test_config1_full_step(variant):
+    specs = wl.config_groups(1)
+    case = Case(specs, seed=0, variant=variant)
+    try:
+        check_step(case, default_hp(lr=2e-2, wd=0.1, mu=0.95, nesterov=True, ns_steps=5))
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("rows,cols", [(128, 256), (256, 128), (320, 704), (576, 200)])
+def test_stagewise_one_iteration(rows, cols, variant):
+    """X0, A, B, X of a single Newton-Schulz iteration against the oracle's."""
+    sp = wl.GroupSpec(rows, cols, 2, torch.float32, torch.float32, 0.02, 1.0)
+    case = Case([sp], seed=42, variant=variant)
+    try:
+        case.ctx.muon_debug_keep(True)
+        hp = default_hp(ns_steps=1)
+        before = case.snapshot()
+        assert case.step(hp)[0] == 0
+        m, n = min(rows, cols), max(rows, cols)
+        for i in range(sp.count):
+            W0, G0, M0 = (x[i] for x in before[0])
+            ref = orc.muon_step(W0, G0, M0, to_orc(hp), trace=True)
+            A, B, X1 = ref["stages"][0]
+            U = ref["X0"] * (ref["nu"] + hp.eps)
+            U = U.T if rows > cols else U
+            b = case.b
+            x0 = f64(case.ctx.muon_debug_read(i, b.MUON_TAP_X0, m, n))
+            assert rel(x0, U) <= 4e-3  # one bf16 rounding of U
+            a_gpu = f64(case.ctx.muon_debug_read(i, b.MUON_TAP_A, m, m))
+            b_gpu = f64(case.ctx.muon_debug_read(i, b.MUON_TAP_B, m, m))
+            x_gpu = f64(case.ctx.muon_debug_read(i, b.MUON_TAP_X, m, n))
+            assert rel(a_gpu, A) <= TOL_NS, rel(a_gpu, A)
+            assert rel(b_gpu, B) <= TOL_NS, rel(b_gpu, B)
+            assert rel(x_gpu, X1) <= TOL_NS, rel(x_gpu, X1)
+            # mirrored tiles: A and B symmetric bit for bit
+            assert np.array_equal(a_gpu, a_gpu.T)
+            assert np.array_equal(b_gpu, b_gpu.T)
+    finally:
+        case.close()
+
+
+RAGGED = [(1, 300), (300, 1), (129, 257), (257, 129), (8, 8), (130, 130), (64, 1000), (1000, 72), (333, 515)]
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("rows,cols", RAGGED)
+@pytest.mark.parametrize("wdt", [torch.float32, torch.bfloat16])
+def test_ragged_shapes(rows, cols, wdt, variant):
+    sp = wl.GroupSpec(rows, cols, 3, wdt, wdt, 0.02, 1.0)
+    case = Case([sp], seed=rows * 7 + cols, variant=variant)
+    try:
+        check_step(case, default_hp(lr=4.2e-4, wd=0.05), check_o=True)
+        check_step(case, default_hp(lr=4.2e-4, wd=0.05))
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+def test_mixed_orientation_bucket_and_multi_step(variant):
+    """Two orientations of one (m, n) share a bucket; three steps with fresh
+    gradients exercise non-zero momentum."""
+    specs = [wl.GroupSpec(384, 200, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
+             wl.GroupSpec(200, 384, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
+             wl.GroupSpec(256, 256, 2, torch.float32, torch.bfloat16, 0.02, 1e-3)]
+    case = Case(specs, seed=5, variant=variant)
+    try:
+        hp = default_hp(lr=4.2e-4, wd=0.1)
+        gen = torch.Generator().manual_seed(99)
+        for step in range(3):
+            if step:
+                for gi, sp in enumerate(specs):
+                    case.dev[gi][1].copy_(wl.make_grads(sp, gen, "cpu"))
+            check_step(case, hp, check_o=(step == 2))
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("ns_steps", [0, 1, 2, 10])
+def test_ns_step_counts(ns_steps):
+    sp = wl.GroupSpec(192, 320, 2, torch.float32, torch.float32, 0.02, 1.0)
+    case = Case([sp], seed=3)
+    try:
+        check_step(case, default_hp(ns_steps=ns_steps, nesterov=(ns_steps != 2)))
+    finally:
+        case.close()
+
+
+def test_bitwise_reproducible():
+    specs = [wl.GroupSpec(448, 640, 4, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
+    outs = []
+    for _ in range(2):
+        case = Case(specs, seed=17)
+        try:
+            hp = default_hp(lr=1e-2)
+            for _ in range(2):
+                assert case.step(hp)[0] == 0
+            W, G, M = case.dev[0]
+            outs.append((W.cpu().view(torch.int16).clone(), M.cpu().view(torch.int32).clone()))
+        finally:
+            case.close()
+    assert torch.equal(outs[0][0], outs[1][0])
+    assert torch.equal(outs[0][1], outs[1][1])
+
+
+def test_zero_gradient_only_decays():
+    sp = wl.GroupSpec(128, 192, 1, torch.float32, torch.float32, 0.02, 1.0)
+    case = Case([sp], seed=1)
+    try:
+        W, G, M = case.dev[0]
+        G.zero_()
+        W0 = W.clone()
+        hp = default_hp(lr=0.1, wd=0.5)
+        assert case.step(hp)[0] == 0
+        assert torch.allclose(W, W0 * (1 - 0.05), rtol=1e-6, atol=0)
+        assert torch.count_nonzero(M) == 0
+    finally:
+        case.close()
+
+
+def test_nonfinite_gradient_reports_and_keeps_weight():
+    b = _binding()
+    sp = wl.GroupSpec(128, 256, 3, torch.float32, torch.float32, 0.02, 1.0)
+    case = Case([sp], seed=2)
+    try:
+        W, G, M = case.dev[0]
+        G[1, 5, 7] = float("inf")
+        W0 = W.clone()
+        status, which = case.step(default_hp())
+        assert status == b.MUON_ERR_NONFINITE and which == 1
+        assert torch.equal(W[1], W0[1])
+        assert not torch.equal(W[0], W0[0]) and not torch.equal(W[2], W0[2])
+        # the status word was cleared by the read
+        assert case.ctx.muon_status()[0] == 0
+    finally:
+        case.close()
+
+
+def test_closed_form_medium_size_on_gpu():
+    """G = U diag(s) V^T with chosen singular values: the result must equal
+    U diag(f^5(s/||s||)) V^T (Sec. 2.1: the iteration is an odd polynomial, so
+    it acts on singular values only).  Pins the CUDA path without the oracle."""
+    rows, cols = 512, 768
+    rng = np.random.default_rng(0)
+    Q1, _ = np.linalg.qr(rng.standard_normal((rows, rows)))
+    Q2, _ = np.linalg.qr(rng.standard_normal((cols, rows)))
+    s = rng.uniform(0.5, 1.5, size=rows)
+    G = (Q1 * s) @ Q2.T
+    sp = wl.GroupSpec(rows, cols, 1, torch.float32, torch.float32, 0.02, 1.0)
+    case = Case([sp], seed=8)
+    try:
+        W, Gd, M = case.dev[0]
+        Gd[0].copy_(torch.from_numpy(G).to(torch.float32))
+        W0 = f64(W[0])
+        hp = default_hp(lr=1e-2, wd=0.0)
+        assert case.step(hp)[0] == 0
+
+        def f(x):
+            return 3.4445 * x - 4.7750 * x ** 3 + 2.0315 * x ** 5
+
+        x = s / np.linalg.norm(s)
+        for _ in range(5):
+            x = f(x)
+        O = (Q1 * x) @ Q2.T
+        dW = -hp.lr * 0.2 * math.sqrt(cols) * O
+        assert rel(f64(W[0]) - W0, dW) <= TOL_NS
+    finally:
+        case.close()
+
+
+def test_host_buffer_entry_point():
+    """muon_step_host: gradients from pinned host memory, weights read back."""
+    specs = [wl.GroupSpec(256, 384, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
+    case = Case(specs, seed=23)
+    ref = Case(specs, seed=23)
+    try:
+        gen = torch.Generator().manual_seed(5)
+        g_new = wl.make_grads(specs[0], gen, "cpu")
+        g_host = [[g_new[i].contiguous().pin_memory() for i in range(2)]]
+        w_host = [[torch.empty(256, 384, dtype=torch.bfloat16).pin_memory() for _ in range(2)]]
+        hp = default_hp(lr=1e-2)
+        case.ctx.muon_step_host(hp, g_host, w_host)
+        assert case.ctx.muon_status()[0] == 0
+        ref.dev[0][1].copy_(g_new)
+        assert ref.step(hp)[0] == 0
+        for i in range(2):
+            assert torch.equal(w_host[0][i], ref.dev[0][0][i].cpu())
+            assert torch.equal(case.dev[0][0][i], ref.dev[0][0][i])
+    finally:
+        case.close()
+        ref.close()
+
+
+def test_invalid_descriptors_are_rejected_on_the_host():
+    b = _binding()
+    W = torch.zeros(2, 64, 64, device="cuda")
+    G = torch.zeros(2, 64, 64, device="cuda")
+    M = torch.zeros(2, 64, 64, device="cuda")
+    with pytest.raises(b.MuonError) as e:
+        b.MuonContext([([W[0]], [W[0]], [M[0]])])  # W aliases G
+    assert e.value.code == b.MUON_ERR_INVALID_ARG
+    ctx = b.MuonContext([([W[0]], [G[0]], [M[0]])])
+    with pytest.raises(b.MuonError):
+        ctx.muon_step(b.Hyper(ns_steps=-1))
+    ctx.muon_destroy()
