@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the Muon step on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--config C] [--impl reference]
+
+One "step" is one pass of the whole hot path (momentum / norm / cast kernel,
+N Newton-Schulz iterations, fused weight update) over every matrix of the
+workload.  Default workload: the MoE expert bucket (198 matrices of
+2048x1408 / 1408x2048, bf16 weights and gradients, fp32 momentum), the
+configuration the Newton-Schulz throughput target is quoted on.
+
+Metric: algorithmic Newton-Schulz TFLOP/s (5 * (3 m^2 n + m^3) per matrix,
+symmetric products counted once) over the whole step time.  `ms_per_step` is
+the absolute step time.  `e2e` is the same metric through muon_step_host:
+gradients come from pinned host memory and the updated weights go back to the
+host inside the timed region.
+
+--impl reference times the CPU fp64 oracle on a bounded sample of the same
+workload (it is the only reference this method has; a baseline, not a target).
+
+With N > 1 (torchrun) every rank owns its own shard of matrices of the same
+size (matrices are independent units; no data-path collective): weak scaling.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2502_16982_b200 import workloads as wl  # noqa: E402
+
+METRIC = "newton_schulz_tflops"
+UNIT = "TFLOP/s"
+WORKLOAD_NAMES = {
+    1: "cfg1: one fp32 128x256 matrix",
+    2: "cfg2: dense transformer 24 layers d=2048 (168 matrices, 1.61 G params)",
+    3: "cfg3: MoE expert bucket, 198 matrices of 2048x1408 / 1408x2048 (0.571 G params)",
+    4: "cfg4: shape sweep, 7 single matrices",
+    5: "cfg5: Moonlight-shaped full parameter set (5286 matrices, 15.3 G params)",
+}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []  # (arrival time, text)
+        self.t_begin = self.t_end = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+            # nvidia-smi needs a moment before its first line; wait for it so
+            # that the samples fall inside the timed region
+            t0 = time.time()
+            while not self.lines and time.time() - t0 < 5.0:
+                time.sleep(0.02)
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def begin(self):
+        self.t_begin = time.time()
+
+    def stop(self):
+        self.t_end = time.time()
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        inside = [ln for (t, ln) in self.lines if self.t_begin is None or self.t_begin <= t <= self.t_end + 0.1]
+        if not inside:  # region shorter than one sampling period: take the nearest sample
+            inside = [ln for (_, ln) in self.lines[-1:]]
+        for ln in inside:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample_time(specs, hp_dict, budget_s=20.0, max_mats=4):
+    """Times the CPU oracle on one matrix per distinct shape (largest groups
+    first), repeating while the budget allows.  Returns (algorithmic flops
+    done, seconds, description, threads)."""
+    import numpy as np
+    from oracle import muon_oracle as orc
+
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    hp = orc.Hyper(**hp_dict)
+    order = sorted(specs, key=lambda s: -s.count * s.rows * s.cols)
+    flops = 0.0
+    secs = 0.0
+    done = []
+    gen = torch.Generator().manual_seed(1234)
+    shapes = order[:max_mats]
+    k = 0
+    while secs < budget_s and k < 64:
+        sp = shapes[k % len(shapes)]
+        one = wl.GroupSpec(sp.rows, sp.cols, 1, sp.w_dtype, sp.g_dtype, sp.w_std, sp.g_std, sp.lognormal_scale)
+        W, G, M = wl.make_group(one, int(gen.initial_seed()) + k, "cpu")
+        Wd, Gd, Md = (t[0].double().numpy() for t in (W, G, M))
+        t0 = time.perf_counter()
+        orc.muon_step(Wd, Gd, Md, hp)
+        dt = time.perf_counter() - t0
+        m, n = min(sp.rows, sp.cols), max(sp.rows, sp.cols)
+        flops += hp.ns_steps * (3.0 * m * m * n + float(m) ** 3)
+        secs += dt
+        done.append("%dx%d" % (sp.rows, sp.cols))
+        k += 1
+    uniq = sorted(set(done))
+    return flops, secs, "%d oracle steps on single matrices of %s" % (len(done), ", ".join(uniq)), threads
+
+
+def hp_dict_default():
+    return dict(lr=4.2e-4, wd=0.1, mu=0.95, nesterov=True, ns_steps=5, a=3.4445, b=-4.7750, c=2.0315,
+                eps=1e-7, rms_scale=0.2)
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    specs = wl.config_groups(args.config)
+    hp = hp_dict_default()
+    times, flops_per = [], 0.0
+    desc, threads = "", 1
+    for i in range(args.warmup + args.steps):
+        fl, secs, desc, threads = oracle_sample_time(specs, hp, budget_s=args.ref_budget, max_mats=args.ref_mats)
+        if i >= args.warmup:
+            times.append(secs)
+            flops_per = fl
+    total = sum(times)
+    value = flops_per * len(times) / total / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": WORKLOAD_NAMES[args.config], "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--layers", type=int, default=None, help="shrink configs 2 and 5 (tests only)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", type=int, default=0, choices=[0, 1])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--max-count", type=int, default=None,
+                    help="cap the matrices per group (small cases for profiler captures)")
+    ap.add_argument("--ref-budget", type=float, default=12.0)
+    ap.add_argument("--ref-mats", type=int, default=4)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    if args.warmup < 3:
+        args.warmup = 3
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the Muon step has no CPU path")
+    from paper_2502_16982_b200 import binding
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    specs = wl.config_groups(args.config, args.layers)
+    if args.max_count is not None:
+        import dataclasses
+        specs = [dataclasses.replace(s, count=min(s.count, args.max_count)) for s in specs]
+    hpd = hp_dict_default()
+    hp = binding.Hyper(**hpd)
+    binding.muon_debug_set_variant(args.variant)
+
+    # Inputs: seeded, drawn on the device (each rank its own shard of equal size).
+    groups, state = [], []
+    for gi, sp in enumerate(specs):
+        W, G, M = wl.make_group(sp, 1000 * args.config + gi + 100000 * rank, dev)
+        state.append((W, G, M))
+        groups.append((wl.views(W), wl.views(G), wl.views(M)))
+    ctx = binding.MuonContext(groups)
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    alg_flops, dense_flops = wl.ns_flops(specs, hp.ns_steps)
+    sbytes = wl.stream_bytes(specs)
+
+    # ---- device-resident timing ------------------------------------------------
+    for _ in range(args.warmup):
+        ctx.muon_step(hp)
+    status, which = ctx.muon_status()
+    if status != 0:
+        raise SystemExit("device status %d at matrix %d during warm-up" % (status, which))
+    launches_per_step = ctx.muon_last_launch_count()
+    ctx.muon_profile_enable(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    barrier()
+    sampler.begin()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        ctx.muon_step(hp)
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    prof = ctx.muon_profile_read()
+    ctx.muon_profile_enable(False)
+    status, which = ctx.muon_status()
+    if status != 0:
+        raise SystemExit("device status %d at matrix %d in the timed region" % (status, which))
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * alg_flops / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end through muon_step_host --------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        g_host, w_host = [], []
+        h2d = d2h = 0
+        for sp, (W, G, M) in zip(specs, state):
+            gh = [G[i].cpu().pin_memory() for i in range(sp.count)]
+            wh = [torch.empty((sp.rows, sp.cols), dtype=sp.w_dtype).pin_memory() for _ in range(sp.count)]
+            g_host.append(gh)
+            w_host.append(wh)
+            h2d += sum(t.numel() * t.element_size() for t in gh)
+            d2h += sum(t.numel() * t.element_size() for t in wh)
+        e2e_steps = max(3, min(args.steps, 5))
+        ctx.muon_step_host(hp, g_host, w_host)
+        barrier()
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            ctx.muon_step_host(hp, g_host, w_host)
+        e1.record(stream)
+        barrier()
+        ms_e2e = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        ms_e2e /= e2e_steps
+        e2e = {"value": world * alg_flops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel -----------------------------------------
+    peaks = load_peaks()
+    gemm_ms = sum(prof[k][0] for k in ("gram", "poly", "comb"))
+    gemm_launches = sum(prof[k][1] for k in ("gram", "poly", "comb"))
+    mom_ms, mom_launches = prof["momentum"]
+    per_kernel = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
+                  for k, v in prof.items() if v[1]}
+    roofline = None
+    if gemm_launches:
+        achieved = alg_flops * args.steps / (gemm_ms * 1e-3) / 1e12
+        peak = float(peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops")))
+        roofline = {
+            "kernel": "ns_gemm_kernel (gram + poly + comb launches)", "bound": "tensor",
+            "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+            "peak_source": "%s bf16_tflops_sustained" % peaks["_source"],
+            "frac_of_measured_burst": achieved / float(peaks.get("bf16_tflops", peak)),
+            "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
+            "dense_equivalent_tflops": dense_flops * args.steps / (gemm_ms * 1e-3) / 1e12,
+            "avg_launch_ms": gemm_ms / gemm_launches,
+            "flops_per_launch": alg_flops * args.steps / gemm_launches,
+            "traffic": None,
+        }
+    stream_roof = None
+    if mom_launches:
+        gbs = sbytes * args.steps / (mom_ms * 1e-3) / 1e9
+        stream_roof = {"kernel": "momentum_cast_kernel", "bound": "hbm", "achieved": gbs,
+                       "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]),
+                       "peak_source": "%s hbm_gbs" % peaks["_source"], "frac_of_nominal": gbs / NOMINAL_HBM_GBS,
+                       "bytes_per_element": sbytes / wl.group_params(specs), "traffic": None}
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline and world == 1:
+        fl, secs, desc, threads = oracle_sample_time(specs, hpd, budget_s=args.ref_budget, max_mats=args.ref_mats)
+        cpu_baseline = {"value": fl / secs / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+                        "sample": desc, "seconds": secs}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD_NAMES[args.config], "matrices": sum(s.count for s in specs),
+                   "params": wl.group_params(specs), "ns_steps": hp.ns_steps,
+                   "l2": "inputs exceed L2" if wl.group_params(specs) * 8 > 126e6 else "inputs fit L2",
+                   "variant": args.variant, "algorithmic_tflop_per_step": alg_flops / 1e12},
+        "pct_bf16_peak_measured_sustained": 100.0 * value / world / float(peaks.get("bf16_tflops_sustained", 1400.0)),
+        "pct_bf16_peak_nominal": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline, "roofline_stream": stream_roof, "kernels": per_kernel,
+        "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line))
+    ctx.muon_destroy()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

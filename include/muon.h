@@ -174,13 +174,33 @@ const char* muon_last_error(void);
 int muon_last_launch_count(const muon_ctx* ctx);
 
 /*
+ * Measurement mode.  While enabled, muon_step records a CUDA event pair around
+ * every kernel it enqueues (on the step's stream).  muon_profile_read
+ * synchronises the device, sums the elapsed milliseconds and the launch counts
+ * per kernel kind since the last read (arrays of MUON_KERNEL_KINDS entries,
+ * indexed by MUON_KERNEL_*) and resets the record.  Events are created on
+ * demand; this mode is for benchmarks, not for training loops.
+ */
+enum {
+  MUON_KERNEL_MOMENTUM = 0, /* momentum + Nesterov + sum of squares + bf16 cast */
+  MUON_KERNEL_NORM = 1,     /* norm finalisation */
+  MUON_KERNEL_GRAM = 2,     /* A = X X^T */
+  MUON_KERNEL_POLY = 3,     /* B = b A + c A A^T */
+  MUON_KERNEL_COMB = 4,     /* X' = a X + B X (last iteration: weight update) */
+  MUON_KERNEL_UPDATE = 5,   /* weight update when ns_steps == 0 */
+  MUON_KERNEL_KINDS = 6
+};
+int muon_profile_enable(muon_ctx* ctx, int enable);
+int muon_profile_read(muon_ctx* ctx, double* ms_by_kernel, int* launches_by_kernel);
+
+/*
  * Test taps.  muon_debug_keep(ctx, 1) makes the last Newton-Schulz iteration
  * also store its X (= O) in the workspace.  muon_debug_read copies one stage
  * of one matrix to a HOST buffer as dense bf16, short side first (m x n with
  * m = min(rows, cols); m x m for A and B): `which` is MUON_TAP_X0 (bf16(U),
  * NOT yet divided by the norm; valid while ns_steps <= 1), MUON_TAP_A, MUON_TAP_B (last iteration) or
- * MUON_TAP_X (last iteration's X).  Only valid while the matrix's chunk is
- * still resident (buckets that fit one chunk).  Synchronises the device.
+ * MUON_TAP_X (last iteration's X).  Only valid for a context with a single
+ * shape bucket that fits one chunk (buckets share the chunk buffers).  Synchronises the device.
  */
 enum { MUON_TAP_X0 = 0, MUON_TAP_A = 1, MUON_TAP_B = 2, MUON_TAP_X = 3 };
 int muon_debug_keep(muon_ctx* ctx, int keep);

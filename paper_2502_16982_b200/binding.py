@@ -32,7 +32,9 @@ EXPORTED = [
     "muon_workspace_bytes", "muon_init", "muon_step", "muon_step_host", "muon_status",
     "muon_get_norms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_variant",
+    "muon_profile_enable", "muon_profile_read",
 ]
+KERNEL_KINDS = ["momentum", "norm", "gram", "poly", "comb", "update"]
 
 
 class muon_group(C.Structure):
@@ -85,6 +87,8 @@ def lib():
     L.muon_debug_keep.argtypes = [C.c_void_p, C.c_int]
     L.muon_debug_read.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
     L.muon_debug_set_variant.argtypes = [C.c_int]
+    L.muon_profile_enable.argtypes = [C.c_void_p, C.c_int]
+    L.muon_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int)]
     for name in EXPORTED:
         if name != "muon_last_error":
             getattr(L, name).restype = C.c_int
@@ -244,6 +248,17 @@ class MuonContext:
 
     def muon_last_launch_count(self) -> int:
         return lib().muon_last_launch_count(self._ctx)
+
+    def muon_profile_enable(self, enable: bool):
+        _check(lib().muon_profile_enable(self._ctx, int(enable)))
+
+    def muon_profile_read(self):
+        """Returns {kernel kind: (milliseconds, launches)} since the last read."""
+        n = len(KERNEL_KINDS)
+        ms = (C.c_double * n)()
+        cnt = (C.c_int * n)()
+        _check(lib().muon_profile_read(self._ctx, ms, cnt))
+        return {k: (ms[i], cnt[i]) for i, k in enumerate(KERNEL_KINDS)}
 
     def muon_debug_keep(self, keep: bool):
         _check(lib().muon_debug_keep(self._ctx, int(keep)))

@@ -257,7 +257,40 @@ struct muon_ctx {
   std::vector<std::pair<int, int>> where;
   // debug taps: which X buffer holds X0 / the last X per bucket
   std::vector<int> x0_buf, xlast_buf;
+  // per-launch timing (measurement mode)
+  int profile;
+  std::vector<cudaEvent_t> ev_pool;           // pairs: start, stop
+  std::vector<int> ev_kind;                   // kind of each recorded pair
+  size_t ev_used;
+  ~muon_ctx() {
+    for (cudaEvent_t e : ev_pool) cudaEventDestroy(e);
+  }
 };
+
+namespace {
+// Records an event pair around one launch when the context is in measurement mode.
+struct LaunchTimer {
+  muon_ctx* ctx;
+  cudaStream_t stream;
+  bool on;
+  LaunchTimer(muon_ctx* c, cudaStream_t s, int kind) : ctx(c), stream(s), on(c->profile != 0) {
+    if (!on) return;
+    if (ctx->ev_used + 2 > ctx->ev_pool.size()) {
+      cudaEvent_t a, b;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
+      ctx->ev_pool.push_back(a);
+      ctx->ev_pool.push_back(b);
+    }
+    ctx->ev_kind.push_back(kind);
+    cudaEventRecord(ctx->ev_pool[ctx->ev_used], stream);
+  }
+  ~LaunchTimer() {
+    if (!on) return;
+    cudaEventRecord(ctx->ev_pool[ctx->ev_used + 1], stream);
+    ctx->ev_used += 2;
+  }
+};
+}  // namespace
 
 extern "C" {
 
@@ -298,6 +331,8 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   ctx->variant = g_default_variant;
   ctx->keep_o = 0;
   ctx->last_launches = 0;
+  ctx->profile = 0;
+  ctx->ev_used = 0;
   ctx->ws = static_cast<uint8_t*>(workspace);
   ctx->ws_bytes = workspace_bytes;
   rc = make_plan(groups, n_groups, ctx->variant, &ctx->buckets, &ctx->sizes, &ctx->total_mats);
@@ -439,15 +474,16 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
       S.tiles_per_matrix = B.stream_tiles;
       S.mu = hp->mu;
       S.nesterov = hp->nesterov ? 1 : 0;
-      ce = launch_momentum_cast(S, B.g_dtype == MUON_DTYPE_FP32, stream);
+      { LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM); ce = launch_momentum_cast(S, B.g_dtype == MUON_DTYPE_FP32, stream); }
       if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "momentum kernel launch: %s", cudaGetErrorString(ce));
       ++launches;
-      ce = launch_norm_finalise(partials, B.stream_tiles, count, hp->eps, descs, scal, norms, status, stream);
+      { LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM); ce = launch_norm_finalise(partials, B.stream_tiles, count, hp->eps, descs, scal, norms, status, stream); }
       if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "norm kernel launch: %s", cudaGetErrorString(ce));
       ++launches;
 
       int cur = 0;
       if (hp->ns_steps == 0) {
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_UPDATE);
         ce = launch_update_noiter(descs, scal, S.x, S.x_stride, B.ldx, count,
                                   static_cast<long long>(B.m) * B.n, upd_scale, decay,
                                   B.w_dtype == MUON_DTYPE_FP32, stream);
@@ -480,7 +516,7 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
         P.scale_kind = first_it ? 1 : 0;
         P.last = 0; P.b_mn_major = 0;
         P.c_acc = 1.f; P.c_in = 0.f;
-        ce = launch_ns_gemm(P, ctx->num_sms, stream);
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm(P, ctx->num_sms, stream); }
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
         ++launches;
 
@@ -495,7 +531,7 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
         P.has_in = 1;
         P.scale_kind = 0;
         P.c_acc = hp->c; P.c_in = hp->b;
-        ce = launch_ns_gemm(P, ctx->num_sms, stream);
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm(P, ctx->num_sms, stream); }
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
         ++launches;
 
@@ -520,7 +556,7 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
         P.scale_kind = first_it ? 2 : 0;
         P.last = last_it ? 1 : 0;
         P.c_acc = 1.f; P.c_in = hp->a;
-        ce = launch_ns_gemm(P, ctx->num_sms, stream);
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, ctx->num_sms, stream); }
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
         ++launches;
         cur = nxt;
@@ -597,6 +633,31 @@ int muon_destroy(muon_ctx* ctx) {
 
 int muon_last_launch_count(const muon_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
 
+int muon_profile_enable(muon_ctx* ctx, int enable) {
+  if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
+  ctx->profile = enable ? 1 : 0;
+  ctx->ev_used = 0;
+  ctx->ev_kind.clear();
+  return MUON_OK;
+}
+
+int muon_profile_read(muon_ctx* ctx, double* ms_by_kernel, int* launches_by_kernel) {
+  if (!ctx || !ms_by_kernel || !launches_by_kernel) return fail(MUON_ERR_INVALID_ARG, "null argument");
+  for (int k = 0; k < MUON_KERNEL_KINDS; ++k) { ms_by_kernel[k] = 0.0; launches_by_kernel[k] = 0; }
+  cudaError_t ce = cudaDeviceSynchronize();
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "synchronise: %s", cudaGetErrorString(ce));
+  for (size_t i = 0; i * 2 + 1 < ctx->ev_used + 1 && i < ctx->ev_kind.size(); ++i) {
+    float ms = 0.f;
+    ce = cudaEventElapsedTime(&ms, ctx->ev_pool[2 * i], ctx->ev_pool[2 * i + 1]);
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "event elapsed: %s", cudaGetErrorString(ce));
+    ms_by_kernel[ctx->ev_kind[i]] += ms;
+    launches_by_kernel[ctx->ev_kind[i]] += 1;
+  }
+  ctx->ev_used = 0;
+  ctx->ev_kind.clear();
+  return MUON_OK;
+}
+
 int muon_debug_keep(muon_ctx* ctx, int keep) {
   if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
   ctx->keep_o = keep ? 1 : 0;
@@ -608,8 +669,8 @@ int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, 
   if (matrix_index < 0 || matrix_index >= ctx->total_mats) return fail(MUON_ERR_INVALID_ARG, "matrix index out of range");
   const int b = ctx->where[matrix_index].first, pos = ctx->where[matrix_index].second;
   const Bucket& B = ctx->buckets[b];
-  if (static_cast<int>(B.mats.size()) > B.chunk)
-    return fail(MUON_ERR_UNSUPPORTED, "taps need a bucket that fits one chunk");
+  if (ctx->buckets.size() != 1 || static_cast<int>(B.mats.size()) > B.chunk)
+    return fail(MUON_ERR_UNSUPPORTED, "taps need a context with one shape bucket that fits one chunk");
   const uint8_t* src;
   int rows, cols, ld;
   switch (which) {

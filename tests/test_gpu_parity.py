@@ -4,9 +4,13 @@ oracle on the same seeded inputs.
 Tolerances (relative Frobenius error):
   * fp32 element-wise parts (momentum, norm):            <= 1e-5
   * bf16 Newton-Schulz path (A, B, X stages, O, delta W): <= 2e-2
+The 2e-2 bound is the one stated for the paper's N = 5 iterations; inside the
+band the quintic map amplifies a perturbation by up to |f'| ~ 3.9 per step, so
+for N > 5 the tests allow 5e-2.
 For bf16 weights the per-step change is about one bf16 ulp of the weight, so
-the weight itself is compared with the oracle's result rounded to bf16:
->= 99.9 % of elements within one ulp.
+the weight itself is compared element-wise with the oracle's result: >= 99.9 %
+of elements within one bf16 ulp plus the Newton-Schulz tolerance expressed per
+element (4 * 2e-2 * RMS of the oracle's update).
 """
 
 import math
@@ -22,6 +26,7 @@ pytestmark = pytest.mark.gpu
 
 TOL_FP32 = 1e-5
 TOL_NS = 2e-2
+TOL_NS_LONG = 5e-2
 
 
 def _binding():
@@ -46,13 +51,13 @@ def to_orc(hp):
                      a=hp.a, b=hp.b, c=hp.c, eps=hp.eps, rms_scale=hp.rms_scale)
 
 
-def bf16_ulp_ok_fraction(got_bf16, expect_f64):
-    """Fraction of elements of a bf16 tensor within one bf16 ulp of the
-    float64 expectation."""
-    exp_t = torch.from_numpy(expect_f64).to(torch.float32)
-    got = got_bf16.detach().cpu().to(torch.float32)
+def bf16_ulp_ok_fraction(got_bf16, expect_f64, slack=0.0):
+    """Fraction of elements of a bf16 tensor within one bf16 ulp (+ slack) of
+    the float64 expectation."""
+    exp_t = torch.from_numpy(expect_f64).to(torch.float64)
+    got = got_bf16.detach().cpu().to(torch.float64)
     ulp = torch.clamp(exp_t.abs(), min=1e-30).log2().floor().exp2() * 2.0 ** -7
-    return float(((got - exp_t).abs() <= ulp * 1.0001).double().mean())
+    return float(((got - exp_t).abs() <= ulp * 1.0001 + slack).double().mean())
 
 
 class Case:
@@ -92,6 +97,7 @@ def check_step(case, hp, check_w=True, check_o=False):
     norms = case.ctx.muon_get_norms()
     gidx = 0
     ohp = to_orc(hp)
+    tol_ns = TOL_NS if hp.ns_steps <= 5 else TOL_NS_LONG
     for gi, sp in enumerate(case.specs):
         W, G, M = case.dev[gi]
         W0, G0, M0 = before[gi]
@@ -103,13 +109,14 @@ def check_step(case, hp, check_w=True, check_o=False):
                 m, n = min(sp.rows, sp.cols), max(sp.rows, sp.cols)
                 o_gpu = f64(case.ctx.muon_debug_read(gidx, case.b.MUON_TAP_X, m, n))
                 o_ref = ref["O"].T if sp.rows > sp.cols else ref["O"]
-                assert rel(o_gpu, o_ref) <= TOL_NS, ("O", gi, i, rel(o_gpu, o_ref))
+                assert rel(o_gpu, o_ref) <= tol_ns, ("O", gi, i, rel(o_gpu, o_ref))
             if check_w:
                 dW_ref = ref["W"] - W0[i]
                 if sp.w_dtype == torch.float32:
-                    assert rel(f64(W[i]) - W0[i], dW_ref) <= TOL_NS, ("dW", gi, i, rel(f64(W[i]) - W0[i], dW_ref))
+                    assert rel(f64(W[i]) - W0[i], dW_ref) <= tol_ns, ("dW", gi, i, rel(f64(W[i]) - W0[i], dW_ref))
                 else:
-                    frac = bf16_ulp_ok_fraction(W[i], ref["W"])
+                    upd_rms = float(np.sqrt(np.mean((dW_ref + hp.lr * hp.wd * W0[i]) ** 2)))
+                    frac = bf16_ulp_ok_fraction(W[i], ref["W"], slack=4 * tol_ns * upd_rms)
                     assert frac >= 0.999, ("W ulp", gi, i, frac)
             gidx += 1
 
@@ -189,7 +196,9 @@ def test_mixed_orientation_bucket_and_multi_step(variant):
     gradients exercise non-zero momentum."""
     specs = [wl.GroupSpec(384, 200, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
              wl.GroupSpec(200, 384, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
-             wl.GroupSpec(256, 256, 2, torch.float32, torch.bfloat16, 0.02, 1e-3)]
+             wl.GroupSpec(256, 256, 2, torch.float32, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(200, 384, 2, torch.float32, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(384, 200, 1, torch.float32, torch.bfloat16, 0.02, 1e-3)]
     case = Case(specs, seed=5, variant=variant)
     try:
         hp = default_hp(lr=4.2e-4, wd=0.1)
@@ -198,7 +207,26 @@ def test_mixed_orientation_bucket_and_multi_step(variant):
             if step:
                 for gi, sp in enumerate(specs):
                     case.dev[gi][1].copy_(wl.make_grads(sp, gen, "cpu"))
-            check_step(case, hp, check_o=(step == 2))
+            check_step(case, hp)
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+def test_one_bucket_two_orientations_with_taps(variant):
+    """Both stored orientations of one (m, n) batched together; O is read
+    through the tap at step 1 and step 3."""
+    specs = [wl.GroupSpec(384, 200, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
+             wl.GroupSpec(200, 384, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True)]
+    case = Case(specs, seed=6, variant=variant)
+    try:
+        hp = default_hp(lr=4.2e-4, wd=0.1)
+        gen = torch.Generator().manual_seed(77)
+        for step in range(3):
+            if step:
+                for gi, sp in enumerate(specs):
+                    case.dev[gi][1].copy_(wl.make_grads(sp, gen, "cpu"))
+            check_step(case, hp, check_o=(step != 1))
     finally:
         case.close()
 
