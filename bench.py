@@ -183,8 +183,10 @@ def run_reference(args, rank):
     hp = hp_dict_default()
     times, flops_per = [], 0.0
     desc, threads = "", 1
+    # each step is a bounded sample; the whole run is kept to about two minutes
+    budget = min(args.ref_budget, 120.0 / max(1, args.warmup + args.steps))
     for i in range(args.warmup + args.steps):
-        fl, secs, desc, threads = oracle_sample_time(specs, hp, budget_s=args.ref_budget, max_mats=args.ref_mats)
+        fl, secs, desc, threads = oracle_sample_time(specs, hp, budget_s=budget, max_mats=args.ref_mats)
         if i >= args.warmup:
             times.append(secs)
             flops_per = fl
