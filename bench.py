@@ -213,6 +213,7 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="shrink configs 2 and 5 (tests only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0, choices=[0, 1])
+    ap.add_argument("--ns-steps", type=int, default=5, help="Newton-Schulz iterations (the paper uses 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--max-count", type=int, default=None,
@@ -248,6 +249,7 @@ def main():
         import dataclasses
         specs = [dataclasses.replace(s, count=min(s.count, args.max_count)) for s in specs]
     hpd = hp_dict_default()
+    hpd["ns_steps"] = args.ns_steps
     hp = binding.Hyper(**hpd)
     binding.muon_debug_set_variant(args.variant)
 

@@ -207,16 +207,25 @@ int muon_debug_keep(muon_ctx* ctx, int keep);
 int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, size_t dst_bytes);
 
 /*
- * Test/bench knob: operand layout of the a*X + B*X product, process-wide, read
+ * Test/bench knob: which Newton-Schulz GEMM kernel runs, process-wide, read
  * by muon_workspace_bytes and muon_init (contexts keep the value they were
  * created with).
- *   0 = the X operand is read from X itself (MN-major shared-memory
- *       descriptor); default,
- *   1 = the X operand is read from a transposed copy X^T kept beside X
- *       (K-major descriptor); costs extra workspace and traffic.
+ *   0 = CTA-pair kernel (cta_group::2), column tiles up to 256 wide; default,
+ *   2 = CTA-pair kernel with 128-wide column tiles only,
+ *   3 = single-CTA kernel (cta_group::1, 128x128 tiles), X read as an MN-major
+ *       operand from X itself,
+ *   1 = single-CTA kernel, X operand read from a transposed copy X^T kept
+ *       beside X (K-major descriptors only); costs extra workspace and traffic.
  * Returns the previous value.
  */
 int muon_debug_set_variant(int variant);
+
+/*
+ * Test tap: the TMEM base address each CTA of the last CTA-pair GEMM launch
+ * obtained (indexed by CTA; 0xFFFFFFFF where no CTA ran).  Copies `n` (at most
+ * 1024) values to the HOST array.  Synchronises the device.
+ */
+int muon_debug_tmem_bases(muon_ctx* ctx, unsigned* out_host, int n);
 
 #ifdef __cplusplus
 }

@@ -32,7 +32,7 @@ EXPORTED = [
     "muon_workspace_bytes", "muon_init", "muon_step", "muon_step_host", "muon_status",
     "muon_get_norms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_variant",
-    "muon_profile_enable", "muon_profile_read",
+    "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
 ]
 KERNEL_KINDS = ["momentum", "norm", "gram", "poly", "comb", "update"]
 
@@ -87,6 +87,7 @@ def lib():
     L.muon_debug_keep.argtypes = [C.c_void_p, C.c_int]
     L.muon_debug_read.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
     L.muon_debug_set_variant.argtypes = [C.c_int]
+    L.muon_debug_tmem_bases.argtypes = [C.c_void_p, C.POINTER(C.c_uint), C.c_int]
     L.muon_profile_enable.argtypes = [C.c_void_p, C.c_int]
     L.muon_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int)]
     for name in EXPORTED:
@@ -259,6 +260,11 @@ class MuonContext:
         cnt = (C.c_int * n)()
         _check(lib().muon_profile_read(self._ctx, ms, cnt))
         return {k: (ms[i], cnt[i]) for i, k in enumerate(KERNEL_KINDS)}
+
+    def muon_debug_tmem_bases(self, n: int = 296):
+        out = (C.c_uint * n)()
+        _check(lib().muon_debug_tmem_bases(self._ctx, out, n))
+        return list(out)
 
     def muon_debug_keep(self, keep: bool):
         _check(lib().muon_debug_keep(self._ctx, int(keep)))

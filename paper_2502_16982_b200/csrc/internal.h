@@ -18,7 +18,7 @@ constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: UMMA, warps 2-5: epil
 // Tile of the streaming momentum kernel (source orientation rows x cols).
 constexpr int kSTR = 64;
 constexpr int kSTC = 128;
-constexpr int kStreamThreads = 256;
+constexpr int kStreamThreads = 512;
 
 // Per-matrix descriptor in device memory.
 struct MatDesc {
@@ -77,6 +77,40 @@ struct GemmParams {
   const MatDesc* descs;  // chunk-relative
   const MatScal* scal;   // chunk-relative
   DevStatus* status;
+};
+
+// One entry of a tile table of the CTA-pair kernel: the pair covers row blocks
+// 2*p and 2*p+1 (128 rows each, one per CTA) and `nbw` (1 or 2) column blocks
+// starting at block `jb`.
+struct PairTile {
+  short p, jb, nbw, pad_;
+};
+
+// Parameters of the CTA-pair Newton-Schulz GEMM kernel (cta_group::2).
+struct PairGemmParams {
+  CUtensorMap map_a;      // operand A rows, box {64 K, 128 rows}, 128B swizzle
+  CUtensorMap map_b;      // operand B, box {64, 64}, 128B swizzle (K-major: {K, rows};
+                          // MN-major: {N, K})
+  CUtensorMap map_in;     // epilogue input, box {64, 128}, 128B swizzle
+  CUtensorMap map_out;    // output, box {64, 128}, 128B swizzle
+  CUtensorMap map_out_t;  // mirrored output, box {128, 64}, no swizzle
+  const PairTile* tiles;  // tile table of one matrix
+  int tiles_per_matrix;
+  int count;       // matrices in this launch
+  int k;           // contraction length
+  int symmetric;   // upper-triangle blocks only, mirrored
+  int has_in;
+  int write_direct;
+  int scale_kind;  // 0: none, 1: s^2, 2: s
+  int last;        // fused weight update
+  int b_mn_major;
+  float c_acc, c_in;
+  float upd_scale, decay;
+  int w_fp32;
+  const MatDesc* descs;
+  const MatScal* scal;
+  DevStatus* status;
+  unsigned* debug;  // optional: TMEM base addresses seen by each CTA (test builds)
 };
 
 struct StreamParams {

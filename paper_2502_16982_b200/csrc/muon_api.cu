@@ -30,11 +30,18 @@ cudaError_t launch_update_noiter(const MatDesc* descs, const MatScal* scal, cons
                                  float upd_scale, float decay, bool w_fp32, cudaStream_t stream);
 cudaError_t gemm_configure();
 cudaError_t launch_ns_gemm(const GemmParams& P, int num_sms, cudaStream_t stream);
+cudaError_t pair_gemm_configure();
+cudaError_t pair_gemm_max_clusters(int acc_cols, int* out);
+cudaError_t launch_ns_gemm_pair(const PairGemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream);
 
 namespace {
 
 thread_local std::string g_last_error;
-int g_default_variant = 0;  // 0: MN-major B operand, 1: transposed copy (K-major)
+// 0: CTA-pair kernel, N up to 256 (default); 2: CTA-pair kernel, N = 128;
+// 1: single-CTA kernel with a transposed copy of X (K-major operands only);
+// 3: single-CTA kernel, X read as an MN-major operand.
+int g_default_variant = 0;
+inline bool variant_is_pair(int v) { return v == 0 || v == 2; }
 
 int fail(int code, const char* fmt, ...) {
   char buf[512];
@@ -68,6 +75,10 @@ struct Bucket {
   int stream_tiles;                      // CTAs per matrix of the streaming kernel
   // workspace offsets (bytes) of the chunk buffers
   size_t off_x[2], off_xt[2], off_a, off_b, off_partials, off_scal, off_descs;
+  size_t off_sym_tiles, off_comb_tiles;
+  std::vector<PairTile> sym_tiles, comb_tiles;  // CTA-pair tile tables of one matrix
+  CUtensorMap a_b64;                 // A as operand B of the pair kernel: box {64,64} swizzled
+  CUtensorMap a_out_t64, b_out_t64;  // A, B mirrored output of the pair kernel: box {128,64} plain
   // tensor maps over the chunk buffers
   CUtensorMap x_op[2];    // X as K-major operand / tile input / tile output: box {64,128} swizzled
   CUtensorMap x_mn[2];    // X as MN-major operand: box {64,64} swizzled
@@ -81,6 +92,7 @@ struct PlanSizes {
   size_t total;
   size_t off_status;
   size_t off_norms;  // float per matrix (global order)
+  size_t off_debug;  // TMEM base addresses seen by the CTAs of the pair kernel
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -224,7 +236,31 @@ int make_plan(const muon_group* groups, int n_groups, int variant, std::vector<B
   for (Bucket& B : *buckets) {
     B.off_descs = off;
     off = align_up(off + B.mats.size() * sizeof(MatDesc), 1024);
+    // tile tables of the CTA-pair kernel: row pair p covers row blocks 2p, 2p+1;
+    // column tiles are one or two 128-blocks wide
+    B.sym_tiles.clear();
+    B.comb_tiles.clear();
+    const int nb = ceil_div(B.m, 128), ncb = ceil_div(B.n, 128), np = ceil_div(nb, 2);
+    const int max_w = variant == 2 ? 1 : 2;
+    for (int p = 0; p < np; ++p) {
+      for (int jb = 2 * p; jb < nb;) {
+        const int w = std::min(max_w, nb - jb);
+        B.sym_tiles.push_back(PairTile{static_cast<short>(p), static_cast<short>(jb), static_cast<short>(w), 0});
+        jb += w;
+      }
+      for (int jb = 0; jb < ncb;) {
+        const int w = std::min(max_w, ncb - jb);
+        B.comb_tiles.push_back(PairTile{static_cast<short>(p), static_cast<short>(jb), static_cast<short>(w), 0});
+        jb += w;
+      }
+    }
+    B.off_sym_tiles = off;
+    off = align_up(off + B.sym_tiles.size() * sizeof(PairTile), 1024);
+    B.off_comb_tiles = off;
+    off = align_up(off + B.comb_tiles.size() * sizeof(PairTile), 1024);
   }
+  sizes->off_debug = off;
+  off = align_up(off + 1024 * sizeof(unsigned), 1024);
   sizes->off_status = off;
   off = align_up(off + sizeof(DevStatus), 1024);
   sizes->off_norms = off;
@@ -241,6 +277,7 @@ using namespace muon;
 struct muon_ctx {
   int device;
   int num_sms;
+  int max_clusters;  // co-resident CTA pairs of the pair kernel
   int variant;
   int keep_o;
   int last_launches;
@@ -298,7 +335,7 @@ const char* muon_last_error(void) { return g_last_error.c_str(); }
 
 int muon_debug_set_variant(int variant) {
   int prev = g_default_variant;
-  if (variant == 0 || variant == 1) g_default_variant = variant;
+  if (variant >= 0 && variant <= 3) g_default_variant = variant;
   return prev;
 }
 
@@ -355,6 +392,9 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   }
   ctx->num_sms = prop.multiProcessorCount;
   ce = gemm_configure();
+  if (ce == cudaSuccess) ce = pair_gemm_configure();
+  if (ce == cudaSuccess) ce = pair_gemm_max_clusters(ctx->variant == 2 ? 128 : 256, &ctx->max_clusters);
+  if (ce == cudaSuccess && ctx->max_clusters < 1) ctx->max_clusters = 1;
   if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ce)); }
 
   // own copies of the descriptor arrays
@@ -399,6 +439,12 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
       ctx->where[r.global] = std::make_pair(static_cast<int>(b), static_cast<int>(i));
     }
     ce = cudaMemcpy(ctx->ws + B.off_descs, descs.data(), descs.size() * sizeof(MatDesc), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess)
+      ce = cudaMemcpy(ctx->ws + B.off_sym_tiles, B.sym_tiles.data(), B.sym_tiles.size() * sizeof(PairTile),
+                      cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess)
+      ce = cudaMemcpy(ctx->ws + B.off_comb_tiles, B.comb_tiles.data(), B.comb_tiles.size() * sizeof(PairTile),
+                      cudaMemcpyHostToDevice);
     if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "descriptor upload: %s", cudaGetErrorString(ce)); }
 
     for (int p = 0; p < 2 && rc == MUON_OK; ++p) {
@@ -417,6 +463,9 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     if (rc == MUON_OK) rc = encode_map(&B.a_out_t, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 128, false);
     if (rc == MUON_OK) rc = encode_map(&B.b_op, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 128, true);
     if (rc == MUON_OK) rc = encode_map(&B.b_out_t, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 128, false);
+    if (rc == MUON_OK) rc = encode_map(&B.a_b64, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 64, true);
+    if (rc == MUON_OK) rc = encode_map(&B.a_out_t64, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 64, false);
+    if (rc == MUON_OK) rc = encode_map(&B.b_out_t64, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 64, false);
     if (rc != MUON_OK) { delete ctx; return rc; }
   }
   ce = cudaMemset(ctx->ws + ctx->sizes.off_status, 0, sizeof(DevStatus));
@@ -425,6 +474,7 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     ce = cudaMemcpy(ctx->ws + ctx->sizes.off_status, &init, sizeof(init), cudaMemcpyHostToDevice);
   }
   if (ce == cudaSuccess) ce = cudaMemset(ctx->ws + ctx->sizes.off_norms, 0, ctx->total_mats * sizeof(float));
+  if (ce == cudaSuccess) ce = cudaMemset(ctx->ws + ctx->sizes.off_debug, 0xFF, 1024 * sizeof(unsigned));
   if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "workspace init: %s", cudaGetErrorString(ce)); }
   *out_ctx = ctx;
   return MUON_OK;
@@ -491,7 +541,73 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
         ++launches;
       }
       const int nb = ceil_div(B.m, kBM);
-      for (int it = 0; it < hp->ns_steps; ++it) {
+      const bool pair = variant_is_pair(ctx->variant);
+      for (int it = 0; pair && it < hp->ns_steps; ++it) {
+        const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
+        const int nxt = cur ^ 1;
+        const int acc_cols = ctx->variant == 2 ? 128 : 256;
+        PairGemmParams P{};
+        P.descs = descs;
+        P.scal = scal;
+        P.status = status;
+        P.debug = reinterpret_cast<unsigned*>(ctx->ws + ctx->sizes.off_debug);
+        P.count = count;
+        P.upd_scale = upd_scale;
+        P.decay = decay;
+        P.w_fp32 = B.w_dtype == MUON_DTYPE_FP32;
+
+        // A = X X^T (first iteration: times s^2, the deferred normalisation)
+        P.map_a = B.x_op[cur];
+        P.map_b = B.x_mn[cur];  // same {64,64} box, read K-major here
+        P.map_in = B.a_op;
+        P.map_out = B.a_op;
+        P.map_out_t = B.a_out_t64;
+        P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
+        P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
+        P.k = B.n;
+        P.symmetric = 1; P.has_in = 0; P.write_direct = 1;
+        P.scale_kind = first_it ? 1 : 0;
+        P.last = 0; P.b_mn_major = 0;
+        P.c_acc = 1.f; P.c_in = 0.f;
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm_pair(P, acc_cols, ctx->max_clusters, stream); }
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
+
+        // B = b*A + c*A*A^T
+        P.map_a = B.a_op;
+        P.map_b = B.a_b64;
+        P.map_in = B.a_op;
+        P.map_out = B.b_op;
+        P.map_out_t = B.b_out_t64;
+        P.k = B.m;
+        P.has_in = 1;
+        P.scale_kind = 0;
+        P.c_acc = hp->c; P.c_in = hp->b;
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm_pair(P, acc_cols, ctx->max_clusters, stream); }
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
+
+        // X' = a*X + B*X (first iteration: times s); last iteration updates W
+        P.map_a = B.b_op;
+        P.map_b = B.x_mn[cur];
+        P.b_mn_major = 1;
+        P.map_in = B.x_op[cur];
+        P.map_out = B.x_op[nxt];
+        P.map_out_t = B.b_out_t64;  // unused
+        P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles);
+        P.tiles_per_matrix = static_cast<int>(B.comb_tiles.size());
+        P.k = B.m;
+        P.symmetric = 0; P.has_in = 1;
+        P.write_direct = last_it ? (ctx->keep_o ? 1 : 0) : 1;
+        P.scale_kind = first_it ? 2 : 0;
+        P.last = last_it ? 1 : 0;
+        P.c_acc = 1.f; P.c_in = hp->a;
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm_pair(P, acc_cols, ctx->max_clusters, stream); }
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
+        cur = nxt;
+      }
+      for (int it = 0; !pair && it < hp->ns_steps; ++it) {
         const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
         const int nxt = cur ^ 1;
         GemmParams P{};
@@ -655,6 +771,15 @@ int muon_profile_read(muon_ctx* ctx, double* ms_by_kernel, int* launches_by_kern
   }
   ctx->ev_used = 0;
   ctx->ev_kind.clear();
+  return MUON_OK;
+}
+
+int muon_debug_tmem_bases(muon_ctx* ctx, unsigned* out_host, int n) {
+  if (!ctx || !out_host || n < 0 || n > 1024) return fail(MUON_ERR_INVALID_ARG, "bad arguments");
+  cudaError_t ce = cudaDeviceSynchronize();
+  if (ce == cudaSuccess)
+    ce = cudaMemcpy(out_host, ctx->ws + ctx->sizes.off_debug, n * sizeof(unsigned), cudaMemcpyDeviceToHost);
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "debug read: %s", cudaGetErrorString(ce));
   return MUON_OK;
 }
 

@@ -16,6 +16,10 @@ namespace muon {
 
 namespace {
 
+constexpr int kRowStep = kStreamThreads / 16;        // rows covered by one pass of the CTA
+constexpr int kRowsPerThread = kSTR / kRowStep;      // passes
+static_assert(kRowsPerThread * kRowStep == kSTR, "tile rows must be a multiple of the pass");
+
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) {
   return __uint_as_float(bits16 << 16);
 }
@@ -51,9 +55,10 @@ __device__ __forceinline__ void load_g8(const void* g, long long off, bool vec, 
 
 // One CTA = one kSTR x kSTC (64 x 128) tile of one matrix in its stored
 // orientation.  Thread t owns 8 consecutive columns (t % 16) of rows
-// (t / 16) + 16*p, p = 0..3.
+// (t / 16) + 32*p, p = 0..1; two rows per thread keep the register count low
+// enough for two 512-thread CTAs per SM.
 template <bool kGradFp32>
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kStreamThreads, 2)
 momentum_cast_kernel(const StreamParams P) {
   // bf16 tile for the transposed store; +2 elements of row padding keeps the
   // column reads off a single bank.
@@ -77,10 +82,10 @@ momentum_cast_kernel(const StreamParams P) {
   const int valid = min(8, max(0, d.cols - col));
   const bool vec = d.vec_ok != 0;
 
-  float g[4][8], m[4][8];
+  float g[kRowsPerThread][8], m[kRowsPerThread][8];
 #pragma unroll
-  for (int p = 0; p < 4; ++p) {
-    const int row = row0 + rsub + 16 * p;
+  for (int p = 0; p < kRowsPerThread; ++p) {
+    const int row = row0 + rsub + kRowStep * p;
     const bool in = row < d.rows && valid > 0;
     if (in) {
       load_g8<kGradFp32>(d.g, static_cast<long long>(row) * d.ld_g + col, vec, valid, g[p]);
@@ -110,8 +115,8 @@ momentum_cast_kernel(const StreamParams P) {
 
   float sumsq = 0.f;
 #pragma unroll
-  for (int p = 0; p < 4; ++p) {
-    const int row = row0 + rsub + 16 * p;
+  for (int p = 0; p < kRowsPerThread; ++p) {
+    const int row = row0 + rsub + kRowStep * p;
     const bool in = row < d.rows && valid > 0;
     float u[8];
 #pragma unroll
@@ -143,7 +148,7 @@ momentum_cast_kernel(const StreamParams P) {
       }
     }
     if (transp != nullptr) {
-      const int lr = rsub + 16 * p;
+      const int lr = rsub + kRowStep * p;
       __nv_bfloat162* trow = reinterpret_cast<__nv_bfloat162*>(&tile[lr][cgrp * 8]);
 #pragma unroll
       for (int e = 0; e < 4; ++e) trow[e] = h[e];

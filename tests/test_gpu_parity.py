@@ -27,6 +27,9 @@ pytestmark = pytest.mark.gpu
 TOL_FP32 = 1e-5
 TOL_NS = 2e-2
 TOL_NS_LONG = 5e-2
+# GEMM kernel variants (muon_debug_set_variant): 0 CTA-pair kernel (default),
+# 2 CTA-pair kernel with 128-wide tiles, 3 / 1 single-CTA kernels.
+VARIANTS = [0, 2, 3, 1]
 
 
 def _binding():
@@ -130,7 +133,7 @@ def default_hp(**kw):
 
 
 # ---------------------------------------------------------------------------
-@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("variant", VARIANTS)
 def test_config1_full_step(variant):
     specs = wl.config_groups(1)
     case = Case(specs, seed=0, variant=variant)
@@ -140,7 +143,7 @@ def test_config1_full_step(variant):
         case.close()
 
 
-@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("variant", VARIANTS)
 @pytest.mark.parametrize("rows,cols", [(128, 256), (256, 128), (320, 704), (576, 200)])
 def test_stagewise_one_iteration(rows, cols, variant):
     """X0, A, B, X of a single Newton-Schulz iteration against the oracle's."""
@@ -177,7 +180,7 @@ def test_stagewise_one_iteration(rows, cols, variant):
 RAGGED = [(1, 300), (300, 1), (129, 257), (257, 129), (8, 8), (130, 130), (64, 1000), (1000, 72), (333, 515)]
 
 
-@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("variant", VARIANTS)
 @pytest.mark.parametrize("rows,cols", RAGGED)
 @pytest.mark.parametrize("wdt", [torch.float32, torch.bfloat16])
 def test_ragged_shapes(rows, cols, wdt, variant):
@@ -190,7 +193,7 @@ def test_ragged_shapes(rows, cols, wdt, variant):
         case.close()
 
 
-@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("variant", VARIANTS)
 def test_mixed_orientation_bucket_and_multi_step(variant):
     """Two orientations of one (m, n) share a bucket; three steps with fresh
     gradients exercise non-zero momentum."""
@@ -212,7 +215,7 @@ def test_mixed_orientation_bucket_and_multi_step(variant):
         case.close()
 
 
-@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("variant", VARIANTS)
 def test_one_bucket_two_orientations_with_taps(variant):
     """Both stored orientations of one (m, n) batched together; O is read
     through the tap at step 1 and step 3."""
