@@ -227,6 +227,51 @@ int muon_debug_set_variant(int variant);
  */
 int muon_debug_tmem_bases(muon_ctx* ctx, unsigned* out_host, int n);
 
+/*
+ * Momentum update and Frobenius norm of ONE matrix with no workspace and no
+ * allocation of any kind (the paper has no counterpart; this is a library
+ * convenience, not a step of its method):
+ *
+ *   M <- mu*M + G;   U = mu*M + G if nesterov else M;   *norm_out = ||U||_F
+ *
+ * Who needs it: code that wants this reduction but cannot obtain device
+ * memory for a workspace - for instance a monitoring hook in a process whose
+ * framework has already reserved the whole GPU for its own pool, so a raw
+ * cudaMalloc would fail, or a caller running where an allocation's implicit
+ * device-wide synchronisation is not acceptable.  The per-tile partial sums
+ * that muon_step keeps in the caller's workspace live here in a fixed array
+ * inside the library image: MUON_STATIC_MAX_TILES floats (256 KiB), held by
+ * every GPU that loads the library until the process exits.
+ *
+ *   g        : DEVICE, rows x cols, row stride ld_g elements, dtype g_dtype.
+ *   m        : DEVICE, fp32, rows x cols, row stride ld_m; updated in place.
+ *   norm_out : DEVICE, one float, written by the call (stream-ordered).
+ *   device   : ordinal the pointers live on; it becomes the calling thread's
+ *              current device.
+ *   stream   : cudaStream_t as void* (NULL = legacy default stream).
+ *
+ * Limit: ceil(rows/64) * ceil(cols/128) must not exceed MUON_STATIC_MAX_TILES
+ * (e.g. 16384 x 32768); larger matrices get MUON_ERR_UNSUPPORTED and nothing
+ * is launched - use muon_step with a workspace for those.
+ *
+ * The first call for a device looks up the device address of the built-in
+ * array (cudaGetSymbolAddress) and caches it; make that first call before
+ * starting any stream capture.  Later calls only enqueue two kernels.  The call
+ * never invokes cudaMalloc, cudaFree or any allocating routine and does not
+ * synchronise.
+ *
+ * All calls on one GPU share the one array, and it keeps whatever the last
+ * call left in it.  Nothing in it needs clearing (each call overwrites the
+ * entries it later reads), but two calls that can overlap on the GPU - different
+ * streams, or different host threads without stream ordering between them -
+ * race on it and may return wrong norms.  Keep the calls of one GPU on one
+ * stream, or order them with events.
+ */
+#define MUON_STATIC_MAX_TILES 65536
+int muon_momentum_norm_static(const void* g, float* m, int rows, int cols, int64_t ld_g, int64_t ld_m,
+                              int g_dtype, float mu, int nesterov, float* norm_out, int device,
+                              void* stream);
+
 #ifdef __cplusplus
 }
 #endif

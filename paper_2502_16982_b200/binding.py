@@ -33,7 +33,9 @@ EXPORTED = [
     "muon_get_norms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_variant",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
+    "muon_momentum_norm_static",
 ]
+MUON_STATIC_MAX_TILES = 65536
 KERNEL_KINDS = ["momentum", "norm", "gram", "poly", "comb", "update"]
 
 
@@ -90,6 +92,8 @@ def lib():
     L.muon_debug_tmem_bases.argtypes = [C.c_void_p, C.POINTER(C.c_uint), C.c_int]
     L.muon_profile_enable.argtypes = [C.c_void_p, C.c_int]
     L.muon_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int)]
+    L.muon_momentum_norm_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64,
+                                            C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
     for name in EXPORTED:
         if name != "muon_last_error":
             getattr(L, name).restype = C.c_int
@@ -176,6 +180,29 @@ def muon_workspace_bytes(groups_c, n_groups) -> int:
 
 def muon_debug_set_variant(variant: int) -> int:
     return lib().muon_debug_set_variant(int(variant))
+
+
+def muon_momentum_norm_static(g, m, mu: float, nesterov: bool, norm_out, stream=None):
+    """M <- mu*M + G in place and ``norm_out[0] = ||U||_F`` for one 2-D CUDA
+    matrix, through the entry point that needs no workspace: the library's
+    built-in scratch array is used, so nothing is allocated here either
+    (``norm_out`` is a one-element fp32 CUDA tensor the caller already owns).
+    Meant for callers that cannot get device memory of their own, e.g. because
+    the framework's pool has reserved the whole GPU.  Calls on one GPU share
+    the scratch: keep them on one stream."""
+    import torch
+    if g.dim() != 2 or m.shape != g.shape or g.stride(1) != 1 or m.stride(1) != 1:
+        raise MuonError(MUON_ERR_INVALID_ARG, "g and m must be equal-shaped 2-D tensors with contiguous rows")
+    if m.dtype != torch.float32 or norm_out.dtype != torch.float32:
+        raise MuonError(MUON_ERR_INVALID_ARG, "m and norm_out must be fp32")
+    dev = g.device.index
+    s = torch.cuda.current_stream(dev) if stream is None else stream
+    rows, cols = g.shape
+    ld_g = g.stride(0) if rows > 1 else max(g.stride(0), cols)
+    ld_m = m.stride(0) if rows > 1 else max(m.stride(0), cols)
+    _check(lib().muon_momentum_norm_static(
+        C.c_void_p(g.data_ptr()), C.c_void_p(m.data_ptr()), rows, cols, ld_g, ld_m, _dtype_code(g),
+        float(mu), int(bool(nesterov)), C.c_void_p(norm_out.data_ptr()), dev, C.c_void_p(s.cuda_stream)))
 
 
 class MuonContext:

@@ -270,6 +270,10 @@ int make_plan(const muon_group* groups, int n_groups, int variant, std::vector<B
 }
 
 }  // namespace
+
+// Lets the other translation units of the library report through muon_last_error().
+void set_last_error(const char* msg) { g_last_error = msg ? msg : ""; }
+
 }  // namespace muon
 
 using namespace muon;
