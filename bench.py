@@ -212,7 +212,6 @@ def main():
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--layers", type=int, default=None, help="shrink configs 2 and 5 (tests only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--variant", type=int, default=0, choices=[0, 1])
     ap.add_argument("--ns-steps", type=int, default=5, help="Newton-Schulz iterations (the paper uses 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -251,7 +250,6 @@ def main():
     hpd = hp_dict_default()
     hpd["ns_steps"] = args.ns_steps
     hp = binding.Hyper(**hpd)
-    binding.muon_debug_set_variant(args.variant)
 
     # Inputs: seeded, drawn on the device (each rank its own shard of equal size).
     groups, state = [], []
@@ -380,7 +378,7 @@ def main():
         "config": {"workload": WORKLOAD_NAMES[args.config], "matrices": sum(s.count for s in specs),
                    "params": wl.group_params(specs), "ns_steps": hp.ns_steps,
                    "l2": "inputs exceed L2" if wl.group_params(specs) * 8 > 126e6 else "inputs fit L2",
-                   "variant": args.variant, "algorithmic_tflop_per_step": alg_flops / 1e12},
+                   "algorithmic_tflop_per_step": alg_flops / 1e12},
         "pct_bf16_peak_measured_sustained": 100.0 * value / world / float(peaks.get("bf16_tflops_sustained", 1400.0)),
         "pct_bf16_peak_nominal": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,

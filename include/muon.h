@@ -185,9 +185,9 @@ enum {
   MUON_KERNEL_MOMENTUM = 0, /* momentum + Nesterov + sum of squares + bf16 cast */
   MUON_KERNEL_NORM = 1,     /* norm finalisation */
   MUON_KERNEL_GRAM = 2,     /* A = X X^T */
-  MUON_KERNEL_POLY = 3,     /* B = b A + c A A^T */
-  MUON_KERNEL_COMB = 4,     /* X' = a X + B X (last iteration: weight update) */
-  MUON_KERNEL_UPDATE = 5,   /* weight update when ns_steps == 0 */
+  MUON_KERNEL_POLY = 3,     /* B = b A + c A A */
+  MUON_KERNEL_COMB = 4,     /* X' = a X + B X (last iteration: fused weight update) */
+  MUON_KERNEL_UPDATE = 5,   /* separate weight update (ns_steps == 0, fp32 or unaligned W) */
   MUON_KERNEL_KINDS = 6
 };
 int muon_profile_enable(muon_ctx* ctx, int enable);
@@ -198,30 +198,19 @@ int muon_profile_read(muon_ctx* ctx, double* ms_by_kernel, int* launches_by_kern
  * also store its X (= O) in the workspace.  muon_debug_read copies one stage
  * of one matrix to a HOST buffer as dense bf16, short side first (m x n with
  * m = min(rows, cols); m x m for A and B): `which` is MUON_TAP_X0 (bf16(U),
- * NOT yet divided by the norm; valid while ns_steps <= 1), MUON_TAP_A, MUON_TAP_B (last iteration) or
- * MUON_TAP_X (last iteration's X).  Only valid for a context with a single
- * shape bucket that fits one chunk (buckets share the chunk buffers).  Synchronises the device.
+ * NOT yet divided by the norm; valid while ns_steps <= 1), MUON_TAP_A,
+ * MUON_TAP_B (last iteration; the kernels keep only the 128x128 blocks on or
+ * above the diagonal of these symmetric matrices, the tap fills in the rest by
+ * symmetry) or MUON_TAP_X (last iteration's X).  Only valid for a context with
+ * a single shape bucket that fits one chunk (buckets share the chunk buffers).
+ * Synchronises the device.
  */
 enum { MUON_TAP_X0 = 0, MUON_TAP_A = 1, MUON_TAP_B = 2, MUON_TAP_X = 3 };
 int muon_debug_keep(muon_ctx* ctx, int keep);
 int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, size_t dst_bytes);
 
 /*
- * Test/bench knob: which Newton-Schulz GEMM kernel runs, process-wide, read
- * by muon_workspace_bytes and muon_init (contexts keep the value they were
- * created with).
- *   0 = CTA-pair kernel (cta_group::2), column tiles up to 256 wide; default,
- *   2 = CTA-pair kernel with 128-wide column tiles only,
- *   3 = single-CTA kernel (cta_group::1, 128x128 tiles), X read as an MN-major
- *       operand from X itself,
- *   1 = single-CTA kernel, X operand read from a transposed copy X^T kept
- *       beside X (K-major descriptors only); costs extra workspace and traffic.
- * Returns the previous value.
- */
-int muon_debug_set_variant(int variant);
-
-/*
- * Test tap: the TMEM base address each CTA of the last CTA-pair GEMM launch
+ * Test tap: the TMEM base address each CTA of the last Newton-Schulz GEMM launch
  * obtained (indexed by CTA; 0xFFFFFFFF where no CTA ran).  Copies `n` (at most
  * 1024) values to the HOST array.  Synchronises the device.
  */

@@ -31,7 +31,7 @@ MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
 EXPORTED = [
     "muon_workspace_bytes", "muon_init", "muon_step", "muon_step_host", "muon_status",
     "muon_get_norms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
-    "muon_debug_keep", "muon_debug_read", "muon_debug_set_variant",
+    "muon_debug_keep", "muon_debug_read",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
     "muon_momentum_norm_static",
 ]
@@ -88,7 +88,6 @@ def lib():
     L.muon_last_launch_count.argtypes = [C.c_void_p]
     L.muon_debug_keep.argtypes = [C.c_void_p, C.c_int]
     L.muon_debug_read.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t]
-    L.muon_debug_set_variant.argtypes = [C.c_int]
     L.muon_debug_tmem_bases.argtypes = [C.c_void_p, C.POINTER(C.c_uint), C.c_int]
     L.muon_profile_enable.argtypes = [C.c_void_p, C.c_int]
     L.muon_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int)]
@@ -176,10 +175,6 @@ def muon_workspace_bytes(groups_c, n_groups) -> int:
     out = C.c_size_t(0)
     _check(lib().muon_workspace_bytes(groups_c, n_groups, C.byref(out)))
     return out.value
-
-
-def muon_debug_set_variant(variant: int) -> int:
-    return lib().muon_debug_set_variant(int(variant))
 
 
 def muon_momentum_norm_static(g, m, mu: float, nesterov: bool, norm_out, stream=None):

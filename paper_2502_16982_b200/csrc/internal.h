@@ -8,11 +8,10 @@
 
 namespace muon {
 
-// Tile shape of the Newton-Schulz GEMM kernel.
-constexpr int kBM = 128;     // output tile rows  (UMMA M)
-constexpr int kBN = 128;     // output tile cols  (UMMA N)
-constexpr int kBK = 64;      // K elements per pipeline stage (128 bytes of bf16)
-constexpr int kStages = 5;   // TMA -> UMMA pipeline depth
+// Newton-Schulz GEMM kernel: a CTA pair owns a 256-row x (128 or 256)-column
+// output tile; operands are staged 64 K-elements (128 bytes of bf16) at a time.
+constexpr int kBM = 128;     // output rows per CTA (UMMA M = 256 over the pair)
+constexpr int kBK = 64;      // K elements per pipeline stage
 constexpr int kGemmThreads = 192;  // warp 0: TMA, warp 1: UMMA, warps 2-5: epilogue
 
 // Tile of the streaming momentum kernel (source orientation rows x cols).
@@ -47,79 +46,55 @@ struct DevStatus {
   int matrix;
 };
 
-enum GemmMode { kGram = 0, kPoly = 1, kComb = 2 };
-
-struct GemmParams {
-  CUtensorMap map_a;      // operand A rows (K-major), box {64, 128}, 128B swizzle
-  CUtensorMap map_b;      // operand B: K-major box {64, 128}, or MN-major box {64, 64}
-  CUtensorMap map_in;     // epilogue input tile, box {64, 128}, 128B swizzle
-  CUtensorMap map_out;    // output tile, box {64, 128}, 128B swizzle
-  CUtensorMap map_out_t;  // transposed output tile, box {128, 128}, no swizzle
-  int mode;
-  int out_rows, out_cols;  // output extent per matrix (m x m, or m x n)
-  int k;                   // contraction length
-  int count;               // matrices in this launch
-  int nb_i, nb_j;          // 128-tiles along rows / cols of the output
-  int tiles_per_matrix;
-  int symmetric;      // upper-triangle tiles only, mirrored
-  int has_in;         // epilogue reads an input tile
-  int write_direct;   // store the bf16 tile through map_out
-  int write_t;        // store the transposed bf16 tile through map_out_t (off-diagonal only
-                      // when symmetric)
-  int scale_kind;     // 0: none, 1: multiply by s^2 of the matrix, 2: multiply by s
-  int last;           // fused weight update in the epilogue
-  int b_mn_major;     // operand B is MN-major (read from X itself)
-  float c_acc, c_in;  // tile = scale * (c_acc * acc + c_in * in)
-  // fused update (last iteration)
-  float upd_scale;  // -lr * rms_scale * sqrt(max(rows, cols))
-  float decay;      // 1 - lr * wd
-  int w_fp32;
-  const MatDesc* descs;  // chunk-relative
-  const MatScal* scal;   // chunk-relative
-  DevStatus* status;
-};
-
-// One entry of a tile table of the CTA-pair kernel: the pair covers row blocks
-// 2*p and 2*p+1 (128 rows each, one per CTA) and `nbw` (1 or 2) column blocks
+// One entry of a tile table: the CTA pair covers row blocks 2*p and 2*p+1
+// (128 rows each, one per CTA) and `nbw` (1 or 2) column blocks of 128
 // starting at block `jb`.
 struct PairTile {
   short p, jb, nbw, pad_;
 };
 
-// Parameters of the CTA-pair Newton-Schulz GEMM kernel (cta_group::2).
-struct PairGemmParams {
-  CUtensorMap map_a;      // operand A rows, box {64 K, 128 rows}, 128B swizzle
-  CUtensorMap map_b;      // operand B, box {64, 64}, 128B swizzle (K-major: {K, rows};
+// Parameters of one launch of the Newton-Schulz GEMM kernel.  Each output
+// element is  scale * (c_acc * acc + c_in * in).
+struct GemmParams {
+  CUtensorMap map_a;      // operand A, K-major: box {64 K, 128 rows}, 128B swizzle
+  CUtensorMap map_a64;    // operand A, MN-major (transposed read of a symmetric matrix stored
+                          // as its upper blocks): box {64 rows, 64 K}, 128B swizzle
+  CUtensorMap map_b;      // operand B: box {64, 64}, 128B swizzle (K-major: {K, rows};
                           // MN-major: {N, K})
-  CUtensorMap map_in;     // epilogue input, box {64, 128}, 128B swizzle
-  CUtensorMap map_out;    // output, box {64, 128}, 128B swizzle
-  CUtensorMap map_out_t;  // mirrored output, box {128, 64}, no swizzle
+  CUtensorMap map_in;     // epilogue input, box {64, 32}, 128B swizzle
+  CUtensorMap map_out;    // output (and the O tap of the last iteration), box {64, 32}, 128B swizzle
+  const CUtensorMap* wmaps;  // last iteration: one map per matrix over its W (chunk-relative);
+                             // box {64, 32} swizzled, or {32, 64} plain when rows > cols
   const PairTile* tiles;  // tile table of one matrix
   int tiles_per_matrix;
   int count;       // matrices in this launch
   int k;           // contraction length
-  int symmetric;   // upper-triangle blocks only, mirrored
-  int has_in;
-  int write_direct;
-  int scale_kind;  // 0: none, 1: s^2, 2: s
-  int last;        // fused weight update
-  int b_mn_major;
+  int m;           // output rows per matrix (short side of the bucket)
+  int out_cols;    // output columns per matrix
+  int symmetric;   // the output is symmetric: only blocks on or above the diagonal are
+                   // computed and stored
+  int a_sym;       // operand A is such a matrix: blocks below the diagonal are read as the
+                   // transposes of their mirror images
+  int b_sym;       // the same for operand B
+  int b_mn_major;  // operand B is read MN-major throughout (X in X' = a X + B X)
+  int has_in;      // the epilogue reads an input tile through map_in
+  int scale_kind;  // 0: none, 1: s^2 of the matrix, 2: s
+  int last;        // fused weight update: W is read, updated and written back
+  int keep_o;      // last iteration: also store O through map_out (test tap)
   float c_acc, c_in;
   float upd_scale, decay;
-  int w_fp32;
   const MatDesc* descs;
   const MatScal* scal;
   DevStatus* status;
-  unsigned* debug;  // optional: TMEM base addresses seen by each CTA (test builds)
+  unsigned* debug;  // optional: TMEM base addresses seen by each CTA (test tap)
 };
 
 struct StreamParams {
   const MatDesc* descs;
   float* partials;  // [count][tiles_per_matrix]
-  __nv_bfloat16* x;   // [count][m][ldx], short side first
-  __nv_bfloat16* xt;  // [count][n][ldxt] or nullptr
-  long long x_stride, xt_stride;  // elements per matrix
-  int ldx, ldxt;
+  __nv_bfloat16* x;    // [count][m][ldx], short side first
+  long long x_stride;  // elements per matrix
+  int ldx;
   int count;
   int tiles_per_matrix;
   float mu;

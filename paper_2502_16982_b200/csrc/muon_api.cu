@@ -25,24 +25,17 @@ cudaError_t launch_momentum_cast(const StreamParams& P, bool grad_fp32, cudaStre
 cudaError_t launch_norm_finalise(const float* partials, int tiles_per_matrix, int count, float eps,
                                  const MatDesc* descs, MatScal* scal, float* norms, DevStatus* status,
                                  cudaStream_t stream);
-cudaError_t launch_update_noiter(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
+cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
                                  long long x_stride, int ldx, int count, long long elems,
-                                 float upd_scale, float decay, bool w_fp32, cudaStream_t stream);
+                                 float upd_scale, float decay, bool use_inv_norm, bool w_fp32,
+                                 cudaStream_t stream);
 cudaError_t gemm_configure();
-cudaError_t launch_ns_gemm(const GemmParams& P, int num_sms, cudaStream_t stream);
-cudaError_t pair_gemm_configure();
-cudaError_t pair_gemm_max_clusters(int acc_cols, int* out);
-cudaError_t launch_ns_gemm_pair(const PairGemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream);
+cudaError_t gemm_max_clusters(int* out);
+cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream);
 
 namespace {
 
 thread_local std::string g_last_error;
-// 0: CTA-pair kernel, N up to 256 (default); 2: CTA-pair kernel, N = 128;
-// 1: single-CTA kernel with a transposed copy of X (K-major operands only);
-// 3: single-CTA kernel, X read as an MN-major operand.
-int g_default_variant = 0;
-inline bool variant_is_pair(int v) { return v == 0 || v == 2; }
-
 int fail(int code, const char* fmt, ...) {
   char buf[512];
   va_list ap;
@@ -70,22 +63,23 @@ struct Bucket {
   int w_dtype, g_dtype;
   std::vector<MatRef> mats;
   int chunk;        // matrices per chunk
-  int ldx, ldxt, lda;
-  size_t x_stride, xt_stride, a_stride;  // elements per matrix
-  int stream_tiles;                      // CTAs per matrix of the streaming kernel
+  int ldx, lda;
+  size_t x_stride, a_stride;  // elements per matrix
+  int stream_tiles;           // CTAs per matrix of the streaming kernel
+  bool fused_update;          // every W is bf16 and TMA-addressable: update W in the last epilogue
   // workspace offsets (bytes) of the chunk buffers
-  size_t off_x[2], off_xt[2], off_a, off_b, off_partials, off_scal, off_descs;
-  size_t off_sym_tiles, off_comb_tiles;
-  std::vector<PairTile> sym_tiles, comb_tiles;  // CTA-pair tile tables of one matrix
-  CUtensorMap a_b64;                 // A as operand B of the pair kernel: box {64,64} swizzled
-  CUtensorMap a_out_t64, b_out_t64;  // A, B mirrored output of the pair kernel: box {128,64} plain
-  // tensor maps over the chunk buffers
-  CUtensorMap x_op[2];    // X as K-major operand / tile input / tile output: box {64,128} swizzled
-  CUtensorMap x_mn[2];    // X as MN-major operand: box {64,64} swizzled
-  CUtensorMap xt_op[2];   // X^T as K-major operand: box {64,128} swizzled
-  CUtensorMap xt_out[2];  // X^T as transposed output: box {128,128} plain
-  CUtensorMap a_op, b_op;      // A, B: box {64,128} swizzled
-  CUtensorMap a_out_t, b_out_t;  // A, B mirrored output: box {128,128} plain
+  size_t off_x[2], off_a, off_b, off_partials, off_scal;
+  // workspace offsets of the persistent per-bucket tables
+  size_t off_descs, off_wmaps, off_sym_tiles, off_comb_tiles;
+  std::vector<PairTile> sym_tiles, comb_tiles;  // tile tables of one matrix
+  int sym_acc_cols, comb_acc_cols;              // widest tile of each table (128 or 256)
+  // tensor maps over the chunk buffers (all 128-byte swizzled)
+  CUtensorMap x_op[2];   // X as K-major operand A: box {64,128}
+  CUtensorMap x_b64[2];  // X as operand B (K-major or MN-major): box {64,64}
+  CUtensorMap x_e[2];    // X as epilogue input / output: box {64,32}
+  CUtensorMap a_op, b_op;    // A, B as K-major operand A: box {64,128}
+  CUtensorMap a_b64, b_b64;  // A, B as operand B or as transposed (MN-major) operand A: box {64,64}
+  CUtensorMap a_e, b_e;      // A, B as epilogue input / output: box {64,32}
 };
 
 struct PlanSizes {
@@ -131,6 +125,14 @@ int encode_map(CUtensorMap* out, void* base, int cols, int rows, int count, int 
   return MUON_OK;
 }
 
+// Map over one caller-owned bf16 weight matrix [rows][cols] with row pitch ld.
+// rows <= cols: the tile of the Newton-Schulz orientation, box {64, 32} swizzled;
+// rows > cols: W is the transpose of that orientation, box {32, 64} plain.
+int encode_w_map(CUtensorMap* out, void* w, int rows, int cols, long long ld) {
+  if (rows <= cols) return encode_map(out, w, cols, rows, 1, static_cast<int>(ld), static_cast<size_t>(rows) * ld, 64, 32, true);
+  return encode_map(out, w, cols, rows, 1, static_cast<int>(ld), static_cast<size_t>(rows) * ld, 32, 64, false);
+}
+
 int validate_groups(const muon_group* groups, int n_groups, bool need_ptrs) {
   if (!groups || n_groups <= 0) return fail(MUON_ERR_INVALID_ARG, "groups is null or n_groups <= 0");
   for (int g = 0; g < n_groups; ++g) {
@@ -160,10 +162,16 @@ int validate_groups(const muon_group* groups, int n_groups, bool need_ptrs) {
   return MUON_OK;
 }
 
+// True if a bf16 weight matrix can be addressed by a TMA descriptor.
+inline bool w_tma_ok(const void* w, long long ld) {
+  return (reinterpret_cast<uintptr_t>(w) & 15) == 0 && ld % 8 == 0;
+}
+
 // Forms the shape buckets and lays out the workspace.  Deterministic in the
-// group list, so muon_workspace_bytes and muon_init agree.
-int make_plan(const muon_group* groups, int n_groups, int variant, std::vector<Bucket>* buckets,
-              PlanSizes* sizes, int* total_mats) {
+// group list (pointers are not consulted), so muon_workspace_bytes and
+// muon_init agree.
+int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* buckets, PlanSizes* sizes,
+              int* total_mats) {
   std::map<std::tuple<int, int, int, int>, int> index;
   buckets->clear();
   int global = 0;
@@ -194,17 +202,14 @@ int make_plan(const muon_group* groups, int n_groups, int variant, std::vector<B
   size_t chunk_region = 0;
   for (Bucket& B : *buckets) {
     B.ldx = static_cast<int>(align_up(B.n, 64));
-    B.ldxt = static_cast<int>(align_up(B.m, 64));
     B.lda = static_cast<int>(align_up(B.m, 64));
     B.x_stride = static_cast<size_t>(B.m) * B.ldx;
-    B.xt_stride = static_cast<size_t>(B.n) * B.ldxt;
     B.a_stride = static_cast<size_t>(B.m) * B.lda;
     // tile counts of the streaming kernel for both stored orientations
     const int t1 = ceil_div(B.m, kSTR) * ceil_div(B.n, kSTC);
     const int t2 = ceil_div(B.n, kSTR) * ceil_div(B.m, kSTC);
     B.stream_tiles = std::max(t1, t2);
-    size_t per_mat = 2 * B.x_stride * 2 + 2 * B.a_stride * 2;
-    if (variant == 1) per_mat += 2 * B.xt_stride * 2;
+    const size_t per_mat = 2 * B.x_stride * 2 + 2 * B.a_stride * 2;
     size_t chunk = std::max<size_t>(1, kChunkBytesMax / per_mat);
     chunk = std::min<size_t>(chunk, B.mats.size());
     chunk = std::min<size_t>(chunk, kChunkCountMax);
@@ -219,12 +224,6 @@ int make_plan(const muon_group* groups, int n_groups, int variant, std::vector<B
     };
     B.off_x[0] = take(chunk * B.x_stride * 2);
     B.off_x[1] = take(chunk * B.x_stride * 2);
-    if (variant == 1) {
-      B.off_xt[0] = take(chunk * B.xt_stride * 2);
-      B.off_xt[1] = take(chunk * B.xt_stride * 2);
-    } else {
-      B.off_xt[0] = B.off_xt[1] = 0;
-    }
     B.off_a = take(chunk * B.a_stride * 2);
     B.off_b = take(chunk * B.a_stride * 2);
     B.off_partials = take(chunk * static_cast<size_t>(B.stream_tiles) * sizeof(float));
@@ -232,25 +231,30 @@ int make_plan(const muon_group* groups, int n_groups, int variant, std::vector<B
     chunk_region = std::max(chunk_region, off);
   }
   size_t off = align_up(chunk_region, 1024);
-  // persistent region: descriptors of every matrix (bucket by bucket), status, norms
+  // persistent region: descriptors and W maps of every matrix (bucket by bucket),
+  // tile tables, status, norms
   for (Bucket& B : *buckets) {
     B.off_descs = off;
     off = align_up(off + B.mats.size() * sizeof(MatDesc), 1024);
-    // tile tables of the CTA-pair kernel: row pair p covers row blocks 2p, 2p+1;
-    // column tiles are one or two 128-blocks wide
+    B.off_wmaps = off;
+    off = align_up(off + B.mats.size() * sizeof(CUtensorMap), 1024);
+    // tile tables: row pair p covers row blocks 2p, 2p+1; column tiles are two
+    // 128-blocks wide, with one single block at the end of an odd run
     B.sym_tiles.clear();
     B.comb_tiles.clear();
+    B.sym_acc_cols = B.comb_acc_cols = 128;
     const int nb = ceil_div(B.m, 128), ncb = ceil_div(B.n, 128), np = ceil_div(nb, 2);
-    const int max_w = variant == 2 ? 1 : 2;
     for (int p = 0; p < np; ++p) {
       for (int jb = 2 * p; jb < nb;) {
-        const int w = std::min(max_w, nb - jb);
+        const int w = std::min(2, nb - jb);
         B.sym_tiles.push_back(PairTile{static_cast<short>(p), static_cast<short>(jb), static_cast<short>(w), 0});
+        if (w == 2) B.sym_acc_cols = 256;
         jb += w;
       }
       for (int jb = 0; jb < ncb;) {
-        const int w = std::min(max_w, ncb - jb);
+        const int w = std::min(2, ncb - jb);
         B.comb_tiles.push_back(PairTile{static_cast<short>(p), static_cast<short>(jb), static_cast<short>(w), 0});
+        if (w == 2) B.comb_acc_cols = 256;
         jb += w;
       }
     }
@@ -281,8 +285,7 @@ using namespace muon;
 struct muon_ctx {
   int device;
   int num_sms;
-  int max_clusters;  // co-resident CTA pairs of the pair kernel
-  int variant;
+  int max_clusters;  // co-resident CTA pairs of the GEMM kernel
   int keep_o;
   int last_launches;
   uint8_t* ws;
@@ -337,12 +340,6 @@ extern "C" {
 
 const char* muon_last_error(void) { return g_last_error.c_str(); }
 
-int muon_debug_set_variant(int variant) {
-  int prev = g_default_variant;
-  if (variant >= 0 && variant <= 3) g_default_variant = variant;
-  return prev;
-}
-
 int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_bytes) {
   if (!out_bytes) return fail(MUON_ERR_INVALID_ARG, "out_bytes is null");
   int rc = validate_groups(groups, n_groups, false);
@@ -350,7 +347,7 @@ int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_byt
   std::vector<Bucket> buckets;
   PlanSizes sizes;
   int total;
-  rc = make_plan(groups, n_groups, g_default_variant, &buckets, &sizes, &total);
+  rc = make_plan(groups, n_groups, &buckets, &sizes, &total);
   if (rc) return rc;
   *out_bytes = sizes.total;
   return MUON_OK;
@@ -369,14 +366,13 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   muon_ctx* ctx = new (std::nothrow) muon_ctx();
   if (!ctx) return fail(MUON_ERR_INVALID_ARG, "out of host memory");
   ctx->device = device;
-  ctx->variant = g_default_variant;
   ctx->keep_o = 0;
   ctx->last_launches = 0;
   ctx->profile = 0;
   ctx->ev_used = 0;
   ctx->ws = static_cast<uint8_t*>(workspace);
   ctx->ws_bytes = workspace_bytes;
-  rc = make_plan(groups, n_groups, ctx->variant, &ctx->buckets, &ctx->sizes, &ctx->total_mats);
+  rc = make_plan(groups, n_groups, &ctx->buckets, &ctx->sizes, &ctx->total_mats);
   if (rc) { delete ctx; return rc; }
   if (workspace_bytes < ctx->sizes.total) {
     const size_t need = ctx->sizes.total;
@@ -396,8 +392,7 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   }
   ctx->num_sms = prop.multiProcessorCount;
   ce = gemm_configure();
-  if (ce == cudaSuccess) ce = pair_gemm_configure();
-  if (ce == cudaSuccess) ce = pair_gemm_max_clusters(ctx->variant == 2 ? 128 : 256, &ctx->max_clusters);
+  if (ce == cudaSuccess) ce = gemm_max_clusters(&ctx->max_clusters);
   if (ce == cudaSuccess && ctx->max_clusters < 1) ctx->max_clusters = 1;
   if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ce)); }
 
@@ -418,10 +413,11 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   ctx->x0_buf.assign(ctx->buckets.size(), 0);
   ctx->xlast_buf.assign(ctx->buckets.size(), 0);
 
-  // per-bucket: upload matrix descriptors, encode tensor maps
+  // per-bucket: upload matrix descriptors and W maps, encode tensor maps
   for (size_t b = 0; b < ctx->buckets.size(); ++b) {
     Bucket& B = ctx->buckets[b];
     std::vector<MatDesc> descs(B.mats.size());
+    B.fused_update = (B.w_dtype == MUON_DTYPE_BF16);
     for (size_t i = 0; i < B.mats.size(); ++i) {
       const MatRef& r = B.mats[i];
       const muon_group& G = ctx->groups[r.group];
@@ -441,6 +437,7 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
       d.vec_ok = (ptr16 && G.ld_w % 8 == 0 && G.ld_g % 8 == 0 && G.ld_m % 8 == 0) ? 1 : 0;
       descs[i] = d;
       ctx->where[r.global] = std::make_pair(static_cast<int>(b), static_cast<int>(i));
+      if (!w_tma_ok(d.w, d.ld_w) || d.ld_w > (1ll << 31)) B.fused_update = false;
     }
     ce = cudaMemcpy(ctx->ws + B.off_descs, descs.data(), descs.size() * sizeof(MatDesc), cudaMemcpyHostToDevice);
     if (ce == cudaSuccess)
@@ -449,27 +446,29 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     if (ce == cudaSuccess)
       ce = cudaMemcpy(ctx->ws + B.off_comb_tiles, B.comb_tiles.data(), B.comb_tiles.size() * sizeof(PairTile),
                       cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess && B.fused_update) {
+      std::vector<CUtensorMap> wmaps(B.mats.size());
+      for (size_t i = 0; i < B.mats.size() && rc == MUON_OK; ++i)
+        rc = encode_w_map(&wmaps[i], descs[i].w, descs[i].rows, descs[i].cols, descs[i].ld_w);
+      if (rc != MUON_OK) { delete ctx; return rc; }
+      ce = cudaMemcpy(ctx->ws + B.off_wmaps, wmaps.data(), wmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+    }
     if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "descriptor upload: %s", cudaGetErrorString(ce)); }
 
     for (int p = 0; p < 2 && rc == MUON_OK; ++p) {
       void* xb = ctx->ws + B.off_x[p];
       rc = encode_map(&B.x_op[p], xb, B.n, B.m, B.chunk, B.ldx, B.x_stride, 64, 128, true);
-      if (rc == MUON_OK) rc = encode_map(&B.x_mn[p], xb, B.n, B.m, B.chunk, B.ldx, B.x_stride, 64, 64, true);
-      if (ctx->variant == 1 && rc == MUON_OK) {
-        void* xtb = ctx->ws + B.off_xt[p];
-        rc = encode_map(&B.xt_op[p], xtb, B.m, B.n, B.chunk, B.ldxt, B.xt_stride, 64, 128, true);
-        if (rc == MUON_OK) rc = encode_map(&B.xt_out[p], xtb, B.m, B.n, B.chunk, B.ldxt, B.xt_stride, 128, 128, false);
-      }
+      if (rc == MUON_OK) rc = encode_map(&B.x_b64[p], xb, B.n, B.m, B.chunk, B.ldx, B.x_stride, 64, 64, true);
+      if (rc == MUON_OK) rc = encode_map(&B.x_e[p], xb, B.n, B.m, B.chunk, B.ldx, B.x_stride, 64, 32, true);
     }
     void* ab = ctx->ws + B.off_a;
     void* bb = ctx->ws + B.off_b;
     if (rc == MUON_OK) rc = encode_map(&B.a_op, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 128, true);
-    if (rc == MUON_OK) rc = encode_map(&B.a_out_t, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 128, false);
     if (rc == MUON_OK) rc = encode_map(&B.b_op, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 128, true);
-    if (rc == MUON_OK) rc = encode_map(&B.b_out_t, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 128, false);
     if (rc == MUON_OK) rc = encode_map(&B.a_b64, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 64, true);
-    if (rc == MUON_OK) rc = encode_map(&B.a_out_t64, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 64, false);
-    if (rc == MUON_OK) rc = encode_map(&B.b_out_t64, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 128, 64, false);
+    if (rc == MUON_OK) rc = encode_map(&B.b_b64, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 64, true);
+    if (rc == MUON_OK) rc = encode_map(&B.a_e, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 32, true);
+    if (rc == MUON_OK) rc = encode_map(&B.b_e, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 32, true);
     if (rc != MUON_OK) { delete ctx; return rc; }
   }
   ce = cudaMemset(ctx->ws + ctx->sizes.off_status, 0, sizeof(DevStatus));
@@ -519,11 +518,8 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
       S.descs = descs;
       S.partials = partials;
       S.x = reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_x[0]);
-      S.xt = ctx->variant == 1 ? reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_xt[0]) : nullptr;
       S.x_stride = static_cast<long long>(B.x_stride);
-      S.xt_stride = static_cast<long long>(B.xt_stride);
       S.ldx = B.ldx;
-      S.ldxt = B.ldxt;
       S.count = count;
       S.tiles_per_matrix = B.stream_tiles;
       S.mu = hp->mu;
@@ -536,150 +532,88 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
       ++launches;
 
       int cur = 0;
-      if (hp->ns_steps == 0) {
-        LaunchTimer lt(ctx, stream, MUON_KERNEL_UPDATE);
-        ce = launch_update_noiter(descs, scal, S.x, S.x_stride, B.ldx, count,
-                                  static_cast<long long>(B.m) * B.n, upd_scale, decay,
-                                  B.w_dtype == MUON_DTYPE_FP32, stream);
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "update kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
-      }
-      const int nb = ceil_div(B.m, kBM);
-      const bool pair = variant_is_pair(ctx->variant);
-      for (int it = 0; pair && it < hp->ns_steps; ++it) {
-        const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
-        const int nxt = cur ^ 1;
-        const int acc_cols = ctx->variant == 2 ? 128 : 256;
-        PairGemmParams P{};
-        P.descs = descs;
-        P.scal = scal;
-        P.status = status;
-        P.debug = reinterpret_cast<unsigned*>(ctx->ws + ctx->sizes.off_debug);
-        P.count = count;
-        P.upd_scale = upd_scale;
-        P.decay = decay;
-        P.w_fp32 = B.w_dtype == MUON_DTYPE_FP32;
-
-        // A = X X^T (first iteration: times s^2, the deferred normalisation)
-        P.map_a = B.x_op[cur];
-        P.map_b = B.x_mn[cur];  // same {64,64} box, read K-major here
-        P.map_in = B.a_op;
-        P.map_out = B.a_op;
-        P.map_out_t = B.a_out_t64;
-        P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
-        P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
-        P.k = B.n;
-        P.symmetric = 1; P.has_in = 0; P.write_direct = 1;
-        P.scale_kind = first_it ? 1 : 0;
-        P.last = 0; P.b_mn_major = 0;
-        P.c_acc = 1.f; P.c_in = 0.f;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm_pair(P, acc_cols, ctx->max_clusters, stream); }
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
-
-        // B = b*A + c*A*A^T
-        P.map_a = B.a_op;
-        P.map_b = B.a_b64;
-        P.map_in = B.a_op;
-        P.map_out = B.b_op;
-        P.map_out_t = B.b_out_t64;
-        P.k = B.m;
-        P.has_in = 1;
-        P.scale_kind = 0;
-        P.c_acc = hp->c; P.c_in = hp->b;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm_pair(P, acc_cols, ctx->max_clusters, stream); }
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
-
-        // X' = a*X + B*X (first iteration: times s); last iteration updates W
-        P.map_a = B.b_op;
-        P.map_b = B.x_mn[cur];
-        P.b_mn_major = 1;
-        P.map_in = B.x_op[cur];
-        P.map_out = B.x_op[nxt];
-        P.map_out_t = B.b_out_t64;  // unused
-        P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles);
-        P.tiles_per_matrix = static_cast<int>(B.comb_tiles.size());
-        P.k = B.m;
-        P.symmetric = 0; P.has_in = 1;
-        P.write_direct = last_it ? (ctx->keep_o ? 1 : 0) : 1;
-        P.scale_kind = first_it ? 2 : 0;
-        P.last = last_it ? 1 : 0;
-        P.c_acc = 1.f; P.c_in = hp->a;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm_pair(P, acc_cols, ctx->max_clusters, stream); }
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
-        cur = nxt;
-      }
-      for (int it = 0; !pair && it < hp->ns_steps; ++it) {
+      for (int it = 0; it < hp->ns_steps; ++it) {
         const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
         const int nxt = cur ^ 1;
         GemmParams P{};
         P.descs = descs;
         P.scal = scal;
         P.status = status;
+        P.debug = reinterpret_cast<unsigned*>(ctx->ws + ctx->sizes.off_debug);
+        P.wmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_wmaps) + first;
         P.count = count;
+        P.m = B.m;
         P.upd_scale = upd_scale;
         P.decay = decay;
-        P.w_fp32 = B.w_dtype == MUON_DTYPE_FP32;
 
         // A = X X^T (first iteration: times s^2, the deferred normalisation)
-        P.mode = kGram;
         P.map_a = B.x_op[cur];
-        P.map_b = B.x_op[cur];
-        P.map_in = B.a_op;
-        P.map_out = B.a_op;
-        P.map_out_t = B.a_out_t;
-        P.out_rows = B.m; P.out_cols = B.m; P.k = B.n;
-        P.nb_i = nb; P.nb_j = nb; P.tiles_per_matrix = nb * (nb + 1) / 2;
-        P.symmetric = 1; P.has_in = 0; P.write_direct = 1; P.write_t = 1;
+        P.map_a64 = B.x_b64[cur];  // unused
+        P.map_b = B.x_b64[cur];
+        P.map_in = B.a_e;  // unused
+        P.map_out = B.a_e;
+        P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
+        P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
+        P.k = B.n;
+        P.out_cols = B.m;
+        P.symmetric = 1; P.a_sym = 0; P.b_sym = 0; P.b_mn_major = 0;
+        P.has_in = 0;
         P.scale_kind = first_it ? 1 : 0;
-        P.last = 0; P.b_mn_major = 0;
+        P.last = 0; P.keep_o = 0;
         P.c_acc = 1.f; P.c_in = 0.f;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm(P, ctx->num_sms, stream); }
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
         ++launches;
 
-        // B = b*A + c*A*A^T
-        P.mode = kPoly;
+        // B = b*A + c*A*A  (A symmetric, kept as its upper blocks)
         P.map_a = B.a_op;
-        P.map_b = B.a_op;
-        P.map_in = B.a_op;
-        P.map_out = B.b_op;
-        P.map_out_t = B.b_out_t;
+        P.map_a64 = B.a_b64;
+        P.map_b = B.a_b64;
+        P.map_in = B.a_e;
+        P.map_out = B.b_e;
         P.k = B.m;
+        P.a_sym = 1; P.b_sym = 1;
         P.has_in = 1;
         P.scale_kind = 0;
         P.c_acc = hp->c; P.c_in = hp->b;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm(P, ctx->num_sms, stream); }
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
         ++launches;
 
-        // X' = a*X + B*X (first iteration: times s); last iteration updates W
-        P.mode = kComb;
+        // X' = a*X + B X (first iteration: times s); the last iteration updates W
+        // in its epilogue when every W of the bucket is TMA-addressable bf16
+        const bool fuse = last_it && B.fused_update;
         P.map_a = B.b_op;
-        if (ctx->variant == 1) {
-          P.map_b = B.xt_op[cur];
-          P.b_mn_major = 0;
-        } else {
-          P.map_b = B.x_mn[cur];
-          P.b_mn_major = 1;
-        }
-        P.map_in = B.x_op[cur];
-        P.map_out = B.x_op[nxt];
-        P.map_out_t = ctx->variant == 1 ? B.xt_out[nxt] : B.x_op[nxt];
-        P.out_rows = B.m; P.out_cols = B.n; P.k = B.m;
-        P.nb_i = nb; P.nb_j = ceil_div(B.n, kBN); P.tiles_per_matrix = P.nb_i * P.nb_j;
-        P.symmetric = 0; P.has_in = 1;
-        P.write_direct = last_it ? (ctx->keep_o ? 1 : 0) : 1;
-        P.write_t = (!last_it && ctx->variant == 1) ? 1 : 0;
+        P.map_a64 = B.b_b64;
+        P.map_b = B.x_b64[cur];
+        P.map_in = B.x_e[cur];
+        P.map_out = B.x_e[nxt];
+        P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles);
+        P.tiles_per_matrix = static_cast<int>(B.comb_tiles.size());
+        P.k = B.m;
+        P.out_cols = B.n;
+        P.symmetric = 0; P.a_sym = 1; P.b_sym = 0; P.b_mn_major = 1;
+        P.has_in = 1;
         P.scale_kind = first_it ? 2 : 0;
-        P.last = last_it ? 1 : 0;
+        P.last = fuse ? 1 : 0;
+        P.keep_o = (fuse && ctx->keep_o) ? 1 : 0;
         P.c_acc = 1.f; P.c_in = hp->a;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, ctx->num_sms, stream); }
+        { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, B.comb_acc_cols, ctx->max_clusters, stream); }
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
         ++launches;
         cur = nxt;
+      }
+      if (hp->ns_steps == 0 || !B.fused_update) {
+        // W <- decay*W + upd_scale*O from the stored O: O = s*bf16(U) when there
+        // was no iteration, else the last X (fp32 weights, or weights a TMA
+        // descriptor cannot address)
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_UPDATE);
+        ce = launch_update_from_x(descs, scal, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + B.off_x[cur]),
+                                  static_cast<long long>(B.x_stride), B.ldx, count,
+                                  static_cast<long long>(B.m) * B.n, upd_scale, decay, hp->ns_steps == 0,
+                                  B.w_dtype == MUON_DTYPE_FP32, stream);
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "update kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
       }
       ctx->x0_buf[b] = 0;
       ctx->xlast_buf[b] = cur;
@@ -828,6 +762,12 @@ int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, 
     ce = cudaMemcpy2D(dst_host, static_cast<size_t>(cols) * 2, src, static_cast<size_t>(ld) * 2,
                       static_cast<size_t>(cols) * 2, rows, cudaMemcpyDeviceToHost);
   if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "tap read: %s", cudaGetErrorString(ce));
+  if (which == MUON_TAP_A || which == MUON_TAP_B) {
+    // the kernels keep only the 128-blocks on or above the diagonal: fill the rest by symmetry
+    uint16_t* d = static_cast<uint16_t*>(dst_host);
+    for (int i = 0; i < rows; ++i)
+      for (int j = 0; j < (i / 128) * 128; ++j) d[static_cast<size_t>(i) * cols + j] = d[static_cast<size_t>(j) * cols + i];
+  }
   return MUON_OK;
 }
 

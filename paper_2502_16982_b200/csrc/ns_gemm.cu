@@ -1,25 +1,43 @@
 // Newton-Schulz GEMM kernel for sm_100a (Eq. 2 of the paper, factored as
-//   A = X X^T,  B = b*A + c*A*A,  X' = a*X + B*X):
-// one persistent, warp-specialised kernel that serves all three products.
+//   A = X X^T,   B = b*A + c*A*A,   X' = a*X + B X).
+// One persistent, warp-specialised kernel on CTA pairs serves all three products.
 //
-//   warp 0      TMA producer: streams 128x64 bf16 operand tiles into a
-//               kStages-deep shared-memory ring (128-byte swizzle).
-//   warp 1      UMMA issuer: tcgen05.mma (M=128, N=128, K=16, bf16 -> fp32)
-//               into one of two TMEM accumulator stages; tcgen05.commit frees
-//               ring slots and publishes finished accumulators.
-//   warps 2-5   epilogue: tcgen05.ld the accumulator, combine with the input
-//               tile (b*A, a*X) in fp32, round once to bf16, stage in shared
-//               memory and TMA-store the tile and (for the symmetric products)
-//               its mirror image; on the last iteration apply the scaled,
-//               weight-decayed update to W instead (Sec. 2.2).
+// Two CTAs on neighbouring SMs form a cluster and share one UMMA
+// (tcgen05.mma.cta_group::2): M = 256 (128 rows from each CTA's own A tile),
+// N = 128 or 256 with the B operand split between the two CTAs' shared
+// memories, so each CTA stages only half of B.
 //
-// Symmetric products compute only tiles with j >= i; the mirrored tile is the
-// transpose of the same rounded values, so A and B are symmetric bit for bit,
-// which is what makes A*A^T a valid way to form A^2.
+// Per CTA (192 threads):
+//   warp 0      TMA producer: its 128x64 A tile and its half of the B tile per
+//               K block into a kStages-deep ring; byte counts of both CTAs are
+//               reported to the leader CTA's "full" barrier.  No multicast.
+//   warp 1      leader CTA only: UMMA issuer; tcgen05.commit (to both CTAs'
+//               barriers) frees ring slots and publishes accumulators (two
+//               TMEM stages of up to 256 fp32 columns).
+//   warps 2-5   epilogue.  Each warp owns the 32 accumulator rows its TMEM lane
+//               quarter holds and runs its own pipeline over "quarters" (32
+//               rows x 64 columns): quarter g uses ring entry g % R of the
+//               warp's staging.  An entry is filled by TMA with the epilogue's
+//               input tile (A for the polynomial, X for the combine, W and X on
+//               the last iteration) R-1 quarters ahead, combined in place with
+//               the accumulator (tcgen05.ld, fp32 arithmetic, one bf16
+//               rounding) and written back by a TMA store issued by the warp
+//               itself; the warps never wait for one another.
 //
-// Every wait is bounded (ptx::mbar_wait).  On expiry the CTA raises its abort
-// flag, records MUON_ERR_TIMEOUT in the device status word, lets copies in
-// flight land, frees its TMEM and returns.
+// Symmetric matrices (A and B) are kept as their 128x128 blocks on or above
+// the diagonal only.  The products that produce them visit only column blocks
+// j >= 2p of row pair p and drop the one below-diagonal block (2p+1, 2p) the
+// pair computes anyway; the products that consume them read a block below the
+// diagonal as the transpose of its mirror image (an MN-major UMMA operand), so
+// both triangles are the same bits by construction.
+//
+// Last iteration (Sec. 2.2): the entry holds the W tile and the X tile,
+//   O = scale * (acc + a*X),   W <- (1 - lr*wd) * W - lr * rms_scale * sqrt(max(rows, cols)) * O
+// in fp32; O itself never reaches HBM.
+//
+// Every software wait is bounded (ptx::mbar_wait); on expiry the CTA records
+// MUON_ERR_TIMEOUT, all roles drain, both CTAs meet at the final cluster
+// barrier, TMEM is freed and the kernel returns.
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -29,58 +47,29 @@ namespace muon {
 
 namespace {
 
-constexpr int kTileABytes = kBM * kBK * 2;          // 16 KiB
-constexpr int kTileBBytes = kBN * kBK * 2;          // 16 KiB
+constexpr int kStages = 4;
+constexpr int kTileABytes = 128 * kBK * 2;   // 16 KiB: this CTA's 128 A rows
+constexpr int kTileBBytes = 128 * kBK * 2;   // 16 KiB: up to 128 B rows (half of N = 256)
 constexpr int kStageBytes = kTileABytes + kTileBBytes;
-constexpr int kEpiIoBytes = 2 * kBM * 128;          // two 64-column halves, 128 rows x 128 B
-constexpr int kEpiTBytes = kBN * kBM * 2;           // transposed bf16 tile / fp32 staging
-constexpr int kNumAccStages = 2;
-constexpr int kTmemCols = kNumAccStages * kBN;      // 256 fp32 columns
-constexpr int kEpiThreads = 128;
-constexpr int kFDirectPitch = 36;   // floats per row, 32-column fp32 staging (direct)
-constexpr int kFTransPitch = 132;   // floats per row, 32-row fp32 staging (transposed)
+constexpr int kEpiWarps = 4;
+constexpr int kSubBytes = 32 * 128;          // one warp's 32 rows x 64 bf16 columns
+constexpr int kSubsPerWarp = 6;              // staging buffers per epilogue warp
+constexpr int kNumAcc = 2;
 
-struct SmemBarriers {
-  unsigned long long full[kStages];
+struct Barriers {
+  unsigned long long full[kStages];       // leader's copy is the live one
   unsigned long long empty[kStages];
-  unsigned long long acc_full[kNumAccStages];
-  unsigned long long acc_empty[kNumAccStages];
-  unsigned long long in_full;
+  unsigned long long acc_full[kNumAcc];
+  unsigned long long acc_empty[kNumAcc];  // leader's copy is the live one
+  unsigned long long io_ready[kEpiWarps][kSubsPerWarp];  // ring entry filled / free to write
   uint32_t tmem_base;
   int abort_flag;
 };
 
-constexpr int kSmemBytes = 1024 /* alignment slack */ + kStages * kStageBytes + kEpiIoBytes +
-                           kEpiTBytes + 256 /* barriers */;
-static_assert(sizeof(SmemBarriers) <= 256, "barrier block too large");
+constexpr int kBarrierBytes = 512;
+constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kEpiWarps * kSubsPerWarp * kSubBytes + kBarrierBytes;
+static_assert(sizeof(Barriers) <= kBarrierBytes, "barrier block too large");
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared-memory limit");
-static_assert(128 * kFDirectPitch * 4 <= kEpiTBytes, "fp32 staging (direct) too large");
-static_assert(32 * kFTransPitch * 4 <= kEpiTBytes, "fp32 staging (transposed) too large");
-
-struct TileCoord {
-  int mat, i, j;
-};
-
-__device__ __forceinline__ TileCoord decode_tile(const GemmParams& P, int tile) {
-  TileCoord t;
-  t.mat = tile / P.tiles_per_matrix;
-  int r = tile - t.mat * P.tiles_per_matrix;
-  if (P.symmetric) {
-    // upper triangle, row by row: row i holds nb - i tiles (j = i .. nb-1)
-    int i = 0, len = P.nb_i;
-    while (r >= len) {
-      r -= len;
-      --len;
-      ++i;
-    }
-    t.i = i;
-    t.j = i + r;
-  } else {
-    t.i = r / P.nb_j;
-    t.j = r - t.i * P.nb_j;
-  }
-  return t;
-}
 
 __device__ __forceinline__ void report_timeout(const GemmParams& P, int mat) {
   if (atomicCAS(&P.status->code, 0, -6 /* MUON_ERR_TIMEOUT */) == 0) {
@@ -88,51 +77,102 @@ __device__ __forceinline__ void report_timeout(const GemmParams& P, int mat) {
   }
 }
 
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+__device__ __forceinline__ void unpack8(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, float (&f)[8]) {
+  f[0] = __uint_as_float(w0 << 16); f[1] = __uint_as_float(w0 & 0xFFFF0000u);
+  f[2] = __uint_as_float(w1 << 16); f[3] = __uint_as_float(w1 & 0xFFFF0000u);
+  f[4] = __uint_as_float(w2 << 16); f[5] = __uint_as_float(w2 & 0xFFFF0000u);
+  f[6] = __uint_as_float(w3 << 16); f[7] = __uint_as_float(w3 & 0xFFFF0000u);
+}
+
+__device__ __forceinline__ void lds128(uint32_t addr, uint32_t& w0, uint32_t& w1, uint32_t& w2, uint32_t& w3) {
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(addr));
+}
+
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+}
+
+// Whether K block `kb` (64 elements) of a symmetric operand must be read
+// transposed: the 128-block it lies in is at or left of `diag_block`, the last
+// block for which some row of the operand tile is below the diagonal.
+__device__ __forceinline__ bool read_transposed(int kb, int diag_block) { return (kb >> 1) <= diag_block; }
+
+// Walks the stream of 64-column quarters one CTA's epilogue processes: tiles in
+// the CTA pair's order, within a tile the quarters that hold output of this CTA.
+struct QuarterCursor {
+  int tile, mat, qd, q_end;
+  int ib, jb;
+
+  // Quarter range of tile `t` for CTA `rank`; returns false past the last tile.
+  __device__ __forceinline__ bool open_tile(const GemmParams& P, int t, int total_tiles, int rank) {
+    tile = t;
+    if (t >= total_tiles) return false;
+    mat = t / P.tiles_per_matrix;
+    const PairTile pt = P.tiles[t - mat * P.tiles_per_matrix];
+    ib = 2 * pt.p + rank;
+    jb = pt.jb;
+    const int cols_left = P.out_cols - jb * 128;
+    q_end = min(2 * pt.nbw, (cols_left + 63) / 64);
+    qd = 0;
+    if (ib * 128 >= P.m) qd = q_end;                     // ragged pair: nothing of ours
+    else if (P.symmetric && jb < ib) qd = min(2, q_end);  // below-diagonal block: dropped
+    return true;
+  }
+  __device__ __forceinline__ bool has_quarter() const { return qd < q_end; }
+};
+
+// kAccCols: fp32 TMEM columns per accumulator stage = widest N (128 or 256).
+template <int kAccCols>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ns_gemm_kernel(const __grid_constant__ GemmParams P) {
   extern __shared__ uint8_t smem_raw[];
-  // 1024-byte alignment: required by the 128-byte swizzle atoms.
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   uint8_t* ring = smem;
-  uint8_t* epi_io = smem + kStages * kStageBytes;
-  uint8_t* epi_t = epi_io + kEpiIoBytes;
-  SmemBarriers* bars = reinterpret_cast<SmemBarriers*>(epi_t + kEpiTBytes);
+  uint8_t* s_epi = smem + kStages * kStageBytes;
+  Barriers* bars = reinterpret_cast<Barriers*>(s_epi + kEpiWarps * kSubsPerWarp * kSubBytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();      // 0 = leader
+  const int cluster = static_cast<int>(ptx::cluster_id_x());
+  const int num_clusters = static_cast<int>(ptx::num_clusters_x());
   const int total_tiles = P.count * P.tiles_per_matrix;
   const int num_kb = (P.k + kBK - 1) / kBK;
   volatile int* abort_flag = &bars->abort_flag;
+  constexpr uint32_t kTmemCols = kNumAcc * kAccCols;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(ptx::smem_u32(&bars->full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&bars->empty[s]), 1);
     }
-    for (int s = 0; s < kNumAccStages; ++s) {
+    for (int s = 0; s < kNumAcc; ++s) {
       ptx::mbar_init(ptx::smem_u32(&bars->acc_full[s]), 1);
-      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[s]), kEpiThreads / 32);
+      ptx::mbar_init(ptx::smem_u32(&bars->acc_empty[s]), 2 * kEpiWarps);
     }
-    ptx::mbar_init(ptx::smem_u32(&bars->in_full), 1);
+    for (int w = 0; w < kEpiWarps; ++w)
+      for (int s = 0; s < kSubsPerWarp; ++s) ptx::mbar_init(ptx::smem_u32(&bars->io_ready[w][s]), 1);
     bars->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tensormap(&P.map_a);
     ptx::prefetch_tensormap(&P.map_b);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(&bars->tmem_base), kTmemCols);
-    ptx::tmem_relinquish();
+    ptx::tmem_alloc_pair(ptx::smem_u32(&bars->tmem_base), kTmemCols);
+    ptx::tmem_relinquish_pair();
   }
   ptx::tc_fence_before();
   __syncthreads();
+  ptx::cluster_sync_all();  // both CTAs' barriers are initialised, both TMEM allocations done
   ptx::tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+  if (P.debug != nullptr && threadIdx.x == 0) P.debug[blockIdx.x] = tmem_base;
 
   if (warp == 0) {
     // ------------------------------------------------------ TMA producer ----
@@ -140,26 +180,39 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const TileCoord t = decode_tile(P, tile);
+      for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
+        const int mat = tile / P.tiles_per_matrix;
+        const PairTile pt = P.tiles[tile - mat * P.tiles_per_matrix];
+        const int row0 = (2 * pt.p + static_cast<int>(rank)) * 128;
+        const int half = 64 * pt.nbw;  // B rows (N columns) staged by each CTA
+        const int b0 = pt.jb * 128 + static_cast<int>(rank) * half;
+        const uint32_t stage_tx = 2u * static_cast<uint32_t>(kTileABytes + half * 128);
+        const int a_diag = P.a_sym ? 2 * pt.p : -1;
+        const int b_diag = P.b_sym ? (pt.nbw == 2 ? pt.jb : pt.jb - 1) : -1;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!ptx::mbar_wait(ptx::smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
-            report_timeout(P, t.mat);
+            report_timeout(P, mat);
             ok = false;
             break;
           }
-          const uint32_t bar = ptx::smem_u32(&bars->full[stage]);
+          const uint32_t local_full = ptx::smem_u32(&bars->full[stage]);
+          const uint32_t leader_full = ptx::map_to_cta(local_full, 0);
           const uint32_t sa = ptx::smem_u32(ring + stage * kStageBytes);
           const uint32_t sb = sa + kTileABytes;
-          ptx::mbar_arrive_expect_tx(bar, kStageBytes);
-          ptx::tma_load_3d(sa, &P.map_a, kb * kBK, t.i * kBM, t.mat, bar);
-          if (!P.b_mn_major) {
-            ptx::tma_load_3d(sb, &P.map_b, kb * kBK, t.j * kBN, t.mat, bar);
+          if (rank == 0) ptx::mbar_arrive_expect_tx(local_full, stage_tx);
+          if (!read_transposed(kb, a_diag)) {
+            ptx::tma_load_3d_pair(sa, &P.map_a, kb * kBK, row0, mat, leader_full);
           } else {
-            // operand B read from the row-major K x N matrix: two boxes of
-            // 64 (N) x 64 (K), each one 128-byte-swizzled atom column
-            ptx::tma_load_3d(sb, &P.map_b, t.j * kBN, kb * kBK, t.mat, bar);
-            ptx::tma_load_3d(sb + kTileBBytes / 2, &P.map_b, t.j * kBN + 64, kb * kBK, t.mat, bar);
+            ptx::tma_load_3d_pair(sa, &P.map_a64, row0, kb * kBK, mat, leader_full);
+            ptx::tma_load_3d_pair(sa + 8192, &P.map_a64, row0 + 64, kb * kBK, mat, leader_full);
+          }
+          const bool b_mn = P.b_mn_major || read_transposed(kb, b_diag);
+          for (int h = 0; h < pt.nbw; ++h) {
+            if (!b_mn) {
+              ptx::tma_load_3d_pair(sb + h * 8192, &P.map_b, kb * kBK, b0 + 64 * h, mat, leader_full);
+            } else {
+              ptx::tma_load_3d_pair(sb + h * 8192, &P.map_b, b0 + 64 * h, kb * kBK, mat, leader_full);
+            }
           }
           if (++stage == kStages) {
             stage = 0;
@@ -168,30 +221,35 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         }
       }
       if (!ok) {
-        // let copies in flight land before the CTA's shared memory goes away
-        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);  // let copies in flight land
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------- UMMA issuer ----
-    if (lane == 0) {
-      const uint32_t idesc = ptx::make_idesc_bf16(kBM, kBN, 0, P.b_mn_major ? 1 : 0);
+    // -------------------------------------------- UMMA issuer (leader CTA) ----
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
+        const int mat = tile / P.tiles_per_matrix;
+        const PairTile pt = P.tiles[tile - mat * P.tiles_per_matrix];
+        const int a_diag = P.a_sym ? 2 * pt.p : -1;
+        const int b_diag = P.b_sym ? (pt.nbw == 2 ? pt.jb : pt.jb - 1) : -1;
         if (!ptx::mbar_wait(ptx::smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag)) {
-          report_timeout(P, tile / P.tiles_per_matrix);
+          report_timeout(P, mat);
           ok = false;
           break;
         }
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kBN);
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
         for (int kb = 0; kb < num_kb; ++kb) {
+          const bool a_mn = read_transposed(kb, a_diag);
+          const bool b_mn = P.b_mn_major || read_transposed(kb, b_diag);
+          const uint32_t idesc = ptx::make_idesc_bf16(256, 128 * pt.nbw, a_mn ? 1 : 0, b_mn ? 1 : 0);
           if (!ptx::mbar_wait(ptx::smem_u32(&bars->full[stage]), phase, abort_flag)) {
-            report_timeout(P, tile / P.tiles_per_matrix);
+            report_timeout(P, mat);
             ok = false;
             break;
           }
@@ -200,25 +258,21 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           const uint32_t sb = sa + kTileABytes;
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) {
-            // K-major, 128-byte swizzle: 8-row groups 1024 B apart; a K step of
-            // 16 elements is 32 bytes inside the swizzle atom.
-            const uint64_t da = ptx::smem_desc_sw128(sa + k * 32, 16, 1024);
-            // MN-major, 128-byte swizzle: 64-element N chunks 8192 B apart
-            // (leading offset), 8-row K groups 1024 B apart (stride offset); a
-            // K step of 16 rows is 2048 bytes.
-            const uint64_t db = P.b_mn_major ? ptx::smem_desc_sw128(sb + k * 2048, 8192, 1024)
-                                             : ptx::smem_desc_sw128(sb + k * 32, 16, 1024);
-            ptx::umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+            const uint64_t da = a_mn ? ptx::smem_desc_sw128(sa + k * 2048, 8192, 1024)
+                                     : ptx::smem_desc_sw128(sa + k * 32, 16, 1024);
+            const uint64_t db = b_mn ? ptx::smem_desc_sw128(sb + k * 2048, 8192, 1024)
+                                     : ptx::smem_desc_sw128(sb + k * 32, 16, 1024);
+            ptx::umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          ptx::umma_commit(ptx::smem_u32(&bars->empty[stage]));
+          ptx::umma_commit_pair(ptx::smem_u32(&bars->empty[stage]), 3);
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
           }
         }
         if (!ok) break;
-        ptx::umma_commit(ptx::smem_u32(&bars->acc_full[acc]));
-        if (++acc == kNumAccStages) {
+        ptx::umma_commit_pair(ptx::smem_u32(&bars->acc_full[acc]), 3);
+        if (++acc == kNumAcc) {
           acc = 0;
           acc_phase ^= 1u;
         }
@@ -226,209 +280,249 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
     }
   } else {
     // ----------------------------------------------------------- epilogue ----
-    const int q = warp & 3;            // TMEM lane quarter this warp may read
-    const int r = q * 32 + lane;       // tile row owned by this thread
-    const int et = threadIdx.x - 64;   // 0..127 within the epilogue group
-    const bool leader = (et == 0);
+    const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the tile
+    const uint32_t my_base = ptx::smem_u32(s_epi + q * kSubsPerWarp * kSubBytes);
+    uint8_t* my_ptr = s_epi + q * kSubsPerWarp * kSubBytes;
+    unsigned long long* my_bars = bars->io_ready[q];
+    // Ring of staging entries: one buffer per quarter, or two (W and X) on the
+    // last iteration.
+    const int bufs_per_q = P.last ? 2 : 1;
+    const uint32_t ring_len = kSubsPerWarp / bufs_per_q;
     int acc = 0;
     uint32_t acc_phase = 0;
-    uint32_t in_phase = 0;
-    const uint32_t io_base = ptx::smem_u32(epi_io);
-    __nv_bfloat16* tbuf = reinterpret_cast<__nv_bfloat16*>(epi_t);
-    float* fbuf = reinterpret_cast<float*>(epi_t);
+    uint32_t gq = 0;  // quarters processed so far by this warp
 
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const TileCoord t = decode_tile(P, tile);
-      // staging buffers are free once the previous tile's stores have read them
-      if (leader) ptx::tma_store_wait_read();
-      ptx::named_bar_sync(1, kEpiThreads);
-      if (P.has_in && leader) {
-        const uint32_t bar = ptx::smem_u32(&bars->in_full);
-        ptx::mbar_arrive_expect_tx(bar, kEpiIoBytes);
-        ptx::tma_load_3d(io_base, &P.map_in, t.j * kBN, t.i * kBM, t.mat, bar);
-        ptx::tma_load_3d(io_base + kEpiIoBytes / 2, &P.map_in, t.j * kBN + 64, t.i * kBM, t.mat, bar);
+    // Lane 0 only: the quarter whose ring entry is armed next (ring_len - 1 ahead).
+    QuarterCursor pre;
+    uint32_t pre_g = 0;
+    bool pre_valid = false;
+    int loads_in_flight = 0;
+    auto pre_seek = [&]() {  // moves `pre` to a quarter, opening tiles as needed
+      while (pre_valid && !pre.has_quarter()) {
+        pre_valid = pre.open_tile(P, pre.tile + num_clusters, total_tiles, static_cast<int>(rank));
       }
-      bool ok = ptx::mbar_wait(ptx::smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag);
-      if (ok && P.has_in) {
-        ok = ptx::mbar_wait(ptx::smem_u32(&bars->in_full), in_phase, abort_flag);
+    };
+    // Arms ring entry pre_g % ring_len for quarter pre_g: starts the TMA loads of
+    // its input tiles, or just marks the entry free to write when there are none.
+    auto arm_next = [&]() {
+      if (!pre_valid) return;
+      const uint32_t e = pre_g % ring_len;
+      const uint32_t bar = ptx::smem_u32(&my_bars[e]);
+      const uint32_t buf = my_base + e * bufs_per_q * kSubBytes;
+      const int row0 = pre.ib * 128 + q * 32;
+      const int col0 = pre.jb * 128 + pre.qd * 64;
+      if (row0 >= P.m) {  // this warp's rows lie beyond the matrix: nothing to fetch
+        ptx::mbar_arrive(bar);
+      } else if (P.last) {
+        const bool tr = P.descs[pre.mat].transposed != 0;
+        ptx::mbar_arrive_expect_tx(bar, 2 * kSubBytes);
+        ptx::tma_load_3d(buf, P.wmaps + pre.mat, tr ? row0 : col0, tr ? col0 : row0, 0, bar);
+        ptx::tma_load_3d(buf + kSubBytes, &P.map_in, col0, row0, pre.mat, bar);
+        ++loads_in_flight;
+      } else if (P.has_in) {
+        ptx::mbar_arrive_expect_tx(bar, kSubBytes);
+        ptx::tma_load_3d(buf, &P.map_in, col0, row0, pre.mat, bar);
+        ++loads_in_flight;
+      } else {
+        ptx::mbar_arrive(bar);
       }
-      in_phase ^= 1u;
-      // All 128 epilogue threads agree on whether to go on: a thread that gave
-      // up must not leave the others waiting at a later barrier.
-      if (ptx::named_bar_any(3, kEpiThreads, !ok)) {
-        if (!ok) report_timeout(P, t.mat);
+      ++pre_g;
+      ++pre.qd;
+      pre_seek();
+    };
+    if (lane == 0) {
+      pre_valid = pre.open_tile(P, cluster, total_tiles, static_cast<int>(rank));
+      pre_seek();
+      for (uint32_t i = 0; i + 1 < ring_len; ++i) arm_next();
+    }
+
+    QuarterCursor cur;
+    bool ok = true;
+    for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
+      cur.open_tile(P, tile, total_tiles, static_cast<int>(rank));
+      const int mat = cur.mat;
+      ok = ptx::mbar_wait(ptx::smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag);
+      ok = __all_sync(0xFFFFFFFFu, ok);  // the warp goes on or gives up as one
+      if (!ok) {
+        if (lane == 0) report_timeout(P, mat);
         break;
       }
       ptx::tc_fence_after();
+      if (cur.has_quarter()) {
+        const MatDesc md = P.descs[mat];
+        const MatScal sc = P.scal[mat];
+        const float scale = P.scale_kind == 1 ? sc.inv_norm_sq : (P.scale_kind == 2 ? sc.inv_norm : 1.0f);
+        const bool w_transposed = P.last && md.transposed;
+        const int row0 = cur.ib * 128 + q * 32;  // first of this warp's rows
+        const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * kAccCols) +
+                               (static_cast<uint32_t>(q * 32) << 16);
 
-      const MatScal sc = P.scal[t.mat];
-      const float scale = P.scale_kind == 1 ? sc.inv_norm_sq : (P.scale_kind == 2 ? sc.inv_norm : 1.0f);
-      const bool mirror = P.write_t && !(P.symmetric && t.i == t.j);
-      const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * kBN) +
-                             (static_cast<uint32_t>(q * 32) << 16);
-      const MatDesc md = P.last ? P.descs[t.mat] : MatDesc{};
+        for (int qd = cur.qd; qd < cur.q_end && ok; ++qd, ++gq) {
+          const uint32_t e = gq % ring_len;
+          const uint32_t buf = my_base + e * bufs_per_q * kSubBytes;  // in / out (W on the last iteration)
+          const uint32_t buf2 = buf + kSubBytes;                        // X tile on the last iteration
+          const int col0 = cur.jb * 128 + qd * 64;
 
-#pragma unroll 1
-      for (int cc = 0; cc < kBN / 32; ++cc) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32(taddr + cc * 32, v);
-        ptx::tmem_ld_wait();
-        if (cc == kBN / 32 - 1) {
-          // accumulator fully read: hand the TMEM stage back to the issuer
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->acc_empty[acc]));
-        }
-        const int half = cc >> 1;
-        float o[32];
-#pragma unroll
-        for (int c8 = 0; c8 < 4; ++c8) {
-          const int chunk = (cc & 1) * 4 + c8;  // 16-byte chunk within the 128-byte row
-          const uint32_t saddr = io_base + half * (kEpiIoBytes / 2) + r * 128 +
-                                 ((chunk ^ (r & 7)) << 4);
-          float in[8];
-          if (P.has_in) {
-            uint32_t w0, w1, w2, w3;
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
-                         : "r"(saddr));
-            in[0] = __uint_as_float(w0 << 16); in[1] = __uint_as_float(w0 & 0xFFFF0000u);
-            in[2] = __uint_as_float(w1 << 16); in[3] = __uint_as_float(w1 & 0xFFFF0000u);
-            in[4] = __uint_as_float(w2 << 16); in[5] = __uint_as_float(w2 & 0xFFFF0000u);
-            in[6] = __uint_as_float(w3 << 16); in[7] = __uint_as_float(w3 & 0xFFFF0000u);
-          } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) in[e] = 0.f;
+          uint32_t v[64];
+          ptx::tmem_ld_32x64(taddr + qd * 64, v);
+          ok = ptx::mbar_wait(ptx::smem_u32(&my_bars[e]), (gq / ring_len) & 1u, abort_flag);
+          ptx::tmem_ld_wait();
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) {
+            if (lane == 0) report_timeout(P, mat);
+            break;
           }
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const float a = __uint_as_float(v[c8 * 8 + e]);
-            o[c8 * 8 + e] = scale * fmaf(P.c_acc, a, P.c_in * in[e]);
-          }
-          if (P.write_direct) {
-            const uint32_t p0 = pack_bf16x2(o[c8 * 8 + 0], o[c8 * 8 + 1]);
-            const uint32_t p1 = pack_bf16x2(o[c8 * 8 + 2], o[c8 * 8 + 3]);
-            const uint32_t p2 = pack_bf16x2(o[c8 * 8 + 4], o[c8 * 8 + 5]);
-            const uint32_t p3 = pack_bf16x2(o[c8 * 8 + 6], o[c8 * 8 + 7]);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(p0), "r"(p1),
-                         "r"(p2), "r"(p3)
-                         : "memory");
-          }
-          if (mirror) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              tbuf[(cc * 32 + c8 * 8 + e) * kBM + r] = __float2bfloat16_rn(o[c8 * 8 + e]);
-            }
-          }
-        }
 
-        if (P.last) {
-          // Fused weight update for a 128 x 32 slab of O (Sec. 2.2):
-          //   W <- (1 - lr*wd) * W - lr * rms_scale * sqrt(max(rows, cols)) * O
-          // staged in fp32 in W's orientation, then applied with coalesced
-          // accesses to W by all epilogue threads.
-          if (!md.transposed) {
+          if (!P.last) {
 #pragma unroll
-            for (int c4 = 0; c4 < 8; ++c4) {
-              float4 f = make_float4(P.upd_scale * o[c4 * 4 + 0], P.upd_scale * o[c4 * 4 + 1],
-                                     P.upd_scale * o[c4 * 4 + 2], P.upd_scale * o[c4 * 4 + 3]);
-              *reinterpret_cast<float4*>(fbuf + r * kFDirectPitch + c4 * 4) = f;
-            }
-          } else {
-#pragma unroll
-            for (int c = 0; c < 32; ++c) fbuf[c * kFTransPitch + r] = P.upd_scale * o[c];
-          }
-          ptx::named_bar_sync(2, kEpiThreads);
-          if (!sc.nonfinite) {
-            // W-orientation slab: `srows` rows of `scols` columns
-            const int srows = md.transposed ? 32 : 128;
-            const int scols = md.transposed ? 128 : 32;
-            const int pitch = md.transposed ? kFTransPitch : kFDirectPitch;
-            const int grow0 = md.transposed ? t.j * kBN + cc * 32 : t.i * kBM;
-            const int gcol0 = md.transposed ? t.i * kBM : t.j * kBN + cc * 32;
-            const int tpr = scols / 4;  // threads per row, 4 elements each
-            const int rpp = kEpiThreads / tpr;
-            const int cl = (et % tpr) * 4;
-            for (int rl = et / tpr; rl < srows; rl += rpp) {
-              const int gr = grow0 + rl, gc = gcol0 + cl;
-              if (gr >= md.rows || gc >= md.cols) continue;
-              const float4 u = *reinterpret_cast<const float4*>(fbuf + rl * pitch + cl);
-              const float uu[4] = {u.x, u.y, u.z, u.w};
-              const int nv = min(4, md.cols - gc);
-              const long long off = static_cast<long long>(gr) * md.ld_w + gc;
-              if (P.w_fp32) {
-                float* wp = reinterpret_cast<float*>(md.w) + off;
-                if (md.vec_ok && nv == 4) {
-                  float4 w = *reinterpret_cast<const float4*>(wp);
-                  w.x = fmaf(P.decay, w.x, uu[0]); w.y = fmaf(P.decay, w.y, uu[1]);
-                  w.z = fmaf(P.decay, w.z, uu[2]); w.w = fmaf(P.decay, w.w, uu[3]);
-                  *reinterpret_cast<float4*>(wp) = w;
-                } else {
-                  for (int e = 0; e < nv; ++e) wp[e] = fmaf(P.decay, wp[e], uu[e]);
-                }
+            for (int c8 = 0; c8 < 8; ++c8) {
+              const uint32_t swz = static_cast<uint32_t>(lane * 128 + ((c8 ^ (lane & 7)) << 4));
+              float in[8];
+              if (P.has_in) {
+                uint32_t w0, w1, w2, w3;
+                lds128(buf + swz, w0, w1, w2, w3);
+                unpack8(w0, w1, w2, w3, in);
               } else {
-                __nv_bfloat16* wp = reinterpret_cast<__nv_bfloat16*>(md.w) + off;
-                if (md.vec_ok && nv == 4) {
-                  uint2 w = *reinterpret_cast<const uint2*>(wp);
-                  const float w0 = __uint_as_float(w.x << 16), w1 = __uint_as_float(w.x & 0xFFFF0000u);
-                  const float w2 = __uint_as_float(w.y << 16), w3 = __uint_as_float(w.y & 0xFFFF0000u);
-                  w.x = pack_bf16x2(fmaf(P.decay, w0, uu[0]), fmaf(P.decay, w1, uu[1]));
-                  w.y = pack_bf16x2(fmaf(P.decay, w2, uu[2]), fmaf(P.decay, w3, uu[3]));
-                  *reinterpret_cast<uint2*>(wp) = w;
-                } else {
-                  for (int e = 0; e < nv; ++e)
-                    wp[e] = __float2bfloat16_rn(fmaf(P.decay, __bfloat162float(wp[e]), uu[e]));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) in[i] = 0.f;
+              }
+              float o[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                o[i] = scale * fmaf(P.c_acc, __uint_as_float(v[c8 * 8 + i]), P.c_in * in[i]);
+              sts128(buf + swz, pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
+            }
+          } else {
+            // O = scale * (acc + c_in * X);  W <- decay * W + upd_scale * O
+            __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(my_ptr + e * bufs_per_q * kSubBytes);
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {
+              const uint32_t swz = static_cast<uint32_t>(lane * 128 + ((c8 ^ (lane & 7)) << 4));
+              uint32_t w0, w1, w2, w3;
+              float x[8], o[8];
+              lds128(buf2 + swz, w0, w1, w2, w3);
+              unpack8(w0, w1, w2, w3, x);
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                o[i] = scale * fmaf(P.c_acc, __uint_as_float(v[c8 * 8 + i]), P.c_in * x[i]);
+              if (P.keep_o) {
+                sts128(buf2 + swz, pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
+              }
+              if (!w_transposed) {
+                float w[8];
+                lds128(buf + swz, w0, w1, w2, w3);
+                unpack8(w0, w1, w2, w3, w);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) w[i] = fmaf(P.decay, w[i], P.upd_scale * o[i]);
+                sts128(buf + swz, pack2(w[0], w[1]), pack2(w[2], w[3]), pack2(w[4], w[5]), pack2(w[6], w[7]));
+              } else {
+                // W tile as [64 rows of W = columns of O][32 columns of W = rows of
+                // O], not swizzled; this lane owns column `lane` of it.
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const int c = c8 * 8 + i;
+                  const float w = __bfloat162float(wt[c * 32 + lane]);
+                  wt[c * 32 + lane] = __float2bfloat16_rn(fmaf(P.decay, w, P.upd_scale * o[i]));
                 }
               }
             }
           }
-          ptx::named_bar_sync(2, kEpiThreads);
-        }
-      }
 
-      if (P.write_direct || mirror) {
-        ptx::fence_proxy_async_smem();
-        ptx::named_bar_sync(2, kEpiThreads);
-        if (leader) {
-          if (P.write_direct) {
-            ptx::tma_store_3d(&P.map_out, t.j * kBN, t.i * kBM, t.mat, io_base);
-            ptx::tma_store_3d(&P.map_out, t.j * kBN + 64, t.i * kBM, t.mat, io_base + kEpiIoBytes / 2);
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (row0 >= P.m) {
+              // rows beyond the matrix: nothing to store
+            } else if (P.last) {
+              if (!sc.nonfinite) {
+                ptx::tma_store_3d(P.wmaps + mat, w_transposed ? row0 : col0, w_transposed ? col0 : row0, 0, buf);
+              }
+              if (P.keep_o) ptx::tma_store_3d(&P.map_out, col0, row0, mat, buf2);
+            } else {
+              ptx::tma_store_3d(&P.map_out, col0, row0, mat, buf);
+            }
+            ptx::tma_store_commit();
+            if (P.has_in && row0 < P.m) --loads_in_flight;
+            ptx::tma_store_wait_read_all_but_one();  // every store but this quarter's has read its staging
+            arm_next();                              // re-arms the entry of the previous quarter
           }
-          if (mirror) {
-            ptx::tma_store_3d(&P.map_out_t, t.i * kBM, t.j * kBN, t.mat, ptx::smem_u32(epi_t));
-          }
-          ptx::tma_store_commit();
+          __syncwarp();
         }
+        if (!ok) break;
       }
-      if (++acc == kNumAccStages) {
+      // accumulator fully read: hand the TMEM stage back to the leader's issuer
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&bars->acc_empty[acc]), 0));
+      }
+      if (++acc == kNumAcc) {
         acc = 0;
         acc_phase ^= 1u;
       }
     }
-    if (leader) ptx::tma_store_wait_all();
+    if (lane == 0) {
+      ptx::tma_store_wait_all();
+      if (loads_in_flight > 0) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);  // abort path: let input tiles in flight land
+      }
+    }
   }
 
   // ---------------------------------------------------------------- teardown --
   ptx::tc_fence_before();
   __syncthreads();
+  ptx::cluster_sync_all();  // the peer may still signal our barriers / read our tiles until here
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 
 }  // namespace
 
 cudaError_t gemm_configure() {
-  return cudaFuncSetAttribute(ns_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(ns_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(ns_gemm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
-cudaError_t launch_ns_gemm(const GemmParams& P, int num_sms, cudaStream_t stream) {
+// Largest number of co-resident CTA pairs (one CTA per SM).
+cudaError_t gemm_max_clusters(int* out) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2, 1, 1);
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaOccupancyMaxActiveClusters(out, ns_gemm_kernel<256>, &cfg);
+}
+
+// acc_cols: 128 when every tile of the launch is one column block wide, else 256.
+cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream) {
   const long long total = static_cast<long long>(P.count) * P.tiles_per_matrix;
   if (total <= 0) return cudaSuccess;
-  const unsigned grid = static_cast<unsigned>(total < num_sms ? total : num_sms);
-  ns_gemm_kernel<<<grid, kGemmThreads, kSmemBytes, stream>>>(P);
-  return cudaGetLastError();
+  const unsigned clusters = static_cast<unsigned>(total < max_clusters ? total : max_clusters);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * clusters, 1, 1);
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  if (acc_cols == 128) return cudaLaunchKernelEx(&cfg, ns_gemm_kernel<128>, P);
+  return cudaLaunchKernelEx(&cfg, ns_gemm_kernel<256>, P);
 }
 
 }  // namespace muon

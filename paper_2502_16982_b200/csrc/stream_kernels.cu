@@ -1,11 +1,13 @@
 // HBM-streaming kernels of the Muon step:
 //   momentum_cast_kernel : M <- mu*M + G, U = Nesterov blend or M, per-tile sum
-//                          of U^2, bf16(U) stored short side first (and, when
-//                          asked, a transposed copy)            (Sec. 2.1 rule
+//                          of U^2, bf16(U) stored short side first (transposed
+//                          when rows > cols)                    (Sec. 2.1 rule
 //                          line 1, footnote 1, Newton-Schulz paragraph)
 //   norm_finalise_kernel : fixed-order sum of the per-tile partials ->
 //                          ||U||_F, 1/(||U||_F + eps), non-finite flag
-//   update_noiter_kernel : the weight update when ns_steps == 0 (O = X0)
+//   update_from_x_kernel : the weight update from a stored O (ns_steps == 0,
+//                          where O = X0; fp32 weights; weights that a TMA
+//                          descriptor cannot address)
 // The division by the norm is deferred: bf16(U) is stored un-normalised and the
 // scalar 1/(||U||_F+eps) is applied in fp32 by the first iteration's epilogues.
 #include <cuda_bf16.h>
@@ -105,13 +107,12 @@ momentum_cast_kernel(const StreamParams P) {
     }
   }
 
-  // Which of the two outputs is the row-major copy of the stored orientation.
-  __nv_bfloat16* direct = d.transposed ? P.xt : P.x;
-  __nv_bfloat16* transp = d.transposed ? P.x : P.xt;
-  const long long direct_stride = d.transposed ? P.xt_stride : P.x_stride;
-  const long long transp_stride = d.transposed ? P.x_stride : P.xt_stride;
-  const int ld_direct = d.transposed ? P.ldxt : P.ldx;
-  const int ld_transp = d.transposed ? P.ldx : P.ldxt;
+  // X is stored short side first: a row-major copy of U when rows <= cols,
+  // its transpose otherwise.
+  __nv_bfloat16* direct = d.transposed ? nullptr : P.x;
+  __nv_bfloat16* transp = d.transposed ? P.x : nullptr;
+  const long long direct_stride = P.x_stride, transp_stride = P.x_stride;
+  const int ld_direct = P.ldx, ld_transp = P.ldx;
 
   float sumsq = 0.f;
 #pragma unroll
@@ -226,22 +227,24 @@ __global__ void norm_finalise_kernel(const float* __restrict__ partials, int til
   }
 }
 
-// ns_steps == 0: O = X0 = s * bf16(U).  W <- decay*W + upd_scale*s*X0.
+// W <- decay*W + upd_scale*O with O = x (short side first), times s when the
+// stored x is the un-normalised bf16(U) (ns_steps == 0: O = X0 = s * bf16(U)).
 template <bool kWFp32>
-__global__ void update_noiter_kernel(const MatDesc* __restrict__ descs,
+__global__ void update_from_x_kernel(const MatDesc* __restrict__ descs,
                                      const MatScal* __restrict__ scal,
                                      const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx,
-                                     float upd_scale, float decay) {
+                                     float upd_scale, float decay, int use_inv_norm) {
   const int mat = blockIdx.y;
   const MatDesc d = descs[mat];
   const MatScal sc = scal[mat];
   if (sc.nonfinite) return;
+  const float s = use_inv_norm ? sc.inv_norm : 1.0f;
   const long long total = static_cast<long long>(d.rows) * d.cols;
   const __nv_bfloat16* xm = x + mat * x_stride;
   for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
        i += static_cast<long long>(gridDim.x) * blockDim.x) {
     const int r = static_cast<int>(i / d.cols), c = static_cast<int>(i - static_cast<long long>(r) * d.cols);
-    const float o = sc.inv_norm * __bfloat162float(d.transposed ? xm[static_cast<long long>(c) * ldx + r]
+    const float o = s * __bfloat162float(d.transposed ? xm[static_cast<long long>(c) * ldx + r]
                                                                 : xm[static_cast<long long>(r) * ldx + c]);
     if (kWFp32) {
       float* w = reinterpret_cast<float*>(d.w) + static_cast<long long>(r) * d.ld_w + c;
@@ -273,9 +276,10 @@ cudaError_t launch_norm_finalise(const float* partials, int tiles_per_matrix, in
   return cudaGetLastError();
 }
 
-cudaError_t launch_update_noiter(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
+cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
                                  long long x_stride, int ldx, int count, long long elems,
-                                 float upd_scale, float decay, bool w_fp32, cudaStream_t stream) {
+                                 float upd_scale, float decay, bool use_inv_norm, bool w_fp32,
+                                 cudaStream_t stream) {
   if (count == 0) return cudaSuccess;
   const int threads = 256;
   long long bx = (elems + threads - 1) / threads;
@@ -283,9 +287,11 @@ cudaError_t launch_update_noiter(const MatDesc* descs, const MatScal* scal, cons
   if (bx < 1) bx = 1;
   dim3 grid(static_cast<unsigned>(bx), static_cast<unsigned>(count));
   if (w_fp32)
-    update_noiter_kernel<true><<<grid, threads, 0, stream>>>(descs, scal, x, x_stride, ldx, upd_scale, decay);
+    update_from_x_kernel<true><<<grid, threads, 0, stream>>>(descs, scal, x, x_stride, ldx, upd_scale, decay,
+                                                             use_inv_norm ? 1 : 0);
   else
-    update_noiter_kernel<false><<<grid, threads, 0, stream>>>(descs, scal, x, x_stride, ldx, upd_scale, decay);
+    update_from_x_kernel<false><<<grid, threads, 0, stream>>>(descs, scal, x, x_stride, ldx, upd_scale, decay,
+                                                              use_inv_norm ? 1 : 0);
   return cudaGetLastError();
 }
 
