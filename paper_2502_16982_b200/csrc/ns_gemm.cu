@@ -70,6 +70,7 @@ constexpr int kBarrierBytes = 512;
 constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kEpiWarps * kSubsPerWarp * kSubBytes + kBarrierBytes;
 static_assert(sizeof(Barriers) <= kBarrierBytes, "barrier block too large");
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared-memory limit");
+static_assert(kBK == 64, "the issuer loop issues four K = 16 steps per stage");
 
 __device__ __forceinline__ void report_timeout(const GemmParams& P, int mat) {
   if (atomicCAS(&P.status->code, 0, -6 /* MUON_ERR_TIMEOUT */) == 0) {
@@ -96,11 +97,6 @@ __device__ __forceinline__ void lds128(uint32_t addr, uint32_t& w0, uint32_t& w1
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
 }
-
-// Whether K block `kb` (64 elements) of a symmetric operand must be read
-// transposed: the 128-block it lies in is at or left of `diag_block`, the last
-// block for which some row of the operand tile is below the diagonal.
-__device__ __forceinline__ bool read_transposed(int kb, int diag_block) { return (kb >> 1) <= diag_block; }
 
 // Walks the stream of 64-column quarters one CTA's epilogue processes: tiles in
 // the CTA pair's order, within a tile the quarters that hold output of this CTA.
@@ -177,9 +173,12 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
   if (warp == 0) {
     // ------------------------------------------------------ TMA producer ----
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+      uint32_t stage = 0, phase = 0;
       bool ok = true;
+      const uint32_t ring_u32 = ptx::smem_u32(ring);
+      const uint32_t full0 = ptx::smem_u32(&bars->full[0]);
+      const uint32_t empty0 = ptx::smem_u32(&bars->empty[0]);
+      const uint32_t leader_full0 = ptx::map_to_cta(full0, 0);  // the rank lives in the upper address bits
       for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
         const int mat = tile / P.tiles_per_matrix;
         const PairTile pt = P.tiles[tile - mat * P.tiles_per_matrix];
@@ -187,32 +186,33 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         const int half = 64 * pt.nbw;  // B rows (N columns) staged by each CTA
         const int b0 = pt.jb * 128 + static_cast<int>(rank) * half;
         const uint32_t stage_tx = 2u * static_cast<uint32_t>(kTileABytes + half * 128);
-        const int a_diag = P.a_sym ? 2 * pt.p : -1;
-        const int b_diag = P.b_sym ? (pt.nbw == 2 ? pt.jb : pt.jb - 1) : -1;
+        // K blocks [0, kb_a) of A and [0, kb_b) of B are read transposed
+        const int kb_a = P.a_sym ? min(num_kb, 2 * (2 * pt.p + 1)) : 0;
+        const int kb_b = P.b_mn_major ? num_kb
+                                      : (P.b_sym ? min(num_kb, 2 * (pt.nbw == 2 ? pt.jb + 1 : pt.jb)) : 0);
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!ptx::mbar_wait(ptx::smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
+          if (!ptx::mbar_wait(empty0 + stage * 8, phase ^ 1u, abort_flag)) {
             report_timeout(P, mat);
             ok = false;
             break;
           }
-          const uint32_t local_full = ptx::smem_u32(&bars->full[stage]);
-          const uint32_t leader_full = ptx::map_to_cta(local_full, 0);
-          const uint32_t sa = ptx::smem_u32(ring + stage * kStageBytes);
+          const uint32_t leader_full = leader_full0 + stage * 8;
+          const uint32_t sa = ring_u32 + stage * kStageBytes;
           const uint32_t sb = sa + kTileABytes;
-          if (rank == 0) ptx::mbar_arrive_expect_tx(local_full, stage_tx);
-          if (!read_transposed(kb, a_diag)) {
-            ptx::tma_load_3d_pair(sa, &P.map_a, kb * kBK, row0, mat, leader_full);
+          const int k0 = kb * kBK;
+          if (rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, stage_tx);
+          if (kb >= kb_a) {
+            ptx::tma_load_3d_pair(sa, &P.map_a, k0, row0, mat, leader_full);
           } else {
-            ptx::tma_load_3d_pair(sa, &P.map_a64, row0, kb * kBK, mat, leader_full);
-            ptx::tma_load_3d_pair(sa + 8192, &P.map_a64, row0 + 64, kb * kBK, mat, leader_full);
+            ptx::tma_load_3d_pair(sa, &P.map_a64, row0, k0, mat, leader_full);
+            ptx::tma_load_3d_pair(sa + 8192, &P.map_a64, row0 + 64, k0, mat, leader_full);
           }
-          const bool b_mn = P.b_mn_major || read_transposed(kb, b_diag);
-          for (int h = 0; h < pt.nbw; ++h) {
-            if (!b_mn) {
-              ptx::tma_load_3d_pair(sb + h * 8192, &P.map_b, kb * kBK, b0 + 64 * h, mat, leader_full);
-            } else {
-              ptx::tma_load_3d_pair(sb + h * 8192, &P.map_b, b0 + 64 * h, kb * kBK, mat, leader_full);
-            }
+          if (kb >= kb_b) {
+            ptx::tma_load_3d_pair(sb, &P.map_b, k0, b0, mat, leader_full);
+            if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, &P.map_b, k0, b0 + 64, mat, leader_full);
+          } else {
+            ptx::tma_load_3d_pair(sb, &P.map_b, b0, k0, mat, leader_full);
+            if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, &P.map_b, b0 + 64, k0, mat, leader_full);
           }
           if (++stage == kStages) {
             stage = 0;
@@ -226,17 +226,26 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
     }
   } else if (warp == 1) {
     // -------------------------------------------- UMMA issuer (leader CTA) ----
+    // The issuing thread is the pacemaker of the tensor pipe, so its loop is
+    // kept short: the shared-memory descriptors differ only in the low word
+    // (encoded start address), which advances by a constant per K = 16 step.
     if (lane == 0 && rank == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+      uint32_t stage = 0, phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      const uint32_t ring_enc = ptx::smem_u32(ring) >> 4;
+      const uint32_t full0 = ptx::smem_u32(&bars->full[0]);
+      const uint32_t empty0 = ptx::smem_u32(&bars->empty[0]);
+      constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO 1024, version 1, 128B swizzle
+      constexpr uint32_t kLboK = (16u >> 4) << 16;      // K-major: LBO 16
+      constexpr uint32_t kLboMN = (8192u >> 4) << 16;   // MN-major: LBO 8192 (next 64-element chunk)
       for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
         const int mat = tile / P.tiles_per_matrix;
         const PairTile pt = P.tiles[tile - mat * P.tiles_per_matrix];
-        const int a_diag = P.a_sym ? 2 * pt.p : -1;
-        const int b_diag = P.b_sym ? (pt.nbw == 2 ? pt.jb : pt.jb - 1) : -1;
+        const int kb_a = P.a_sym ? min(num_kb, 2 * (2 * pt.p + 1)) : 0;
+        const int kb_b = P.b_mn_major ? num_kb
+                                      : (P.b_sym ? min(num_kb, 2 * (pt.nbw == 2 ? pt.jb + 1 : pt.jb)) : 0);
         if (!ptx::mbar_wait(ptx::smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag)) {
           report_timeout(P, mat);
           ok = false;
@@ -244,30 +253,38 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
-        for (int kb = 0; kb < num_kb; ++kb) {
-          const bool a_mn = read_transposed(kb, a_diag);
-          const bool b_mn = P.b_mn_major || read_transposed(kb, b_diag);
+        uint32_t accumulate = 0;
+        // up to three runs of K blocks, each with one operand layout
+        const int cut1 = min(kb_a, kb_b), cut2 = max(kb_a, kb_b);
+        int kb = 0;
+#pragma unroll 1
+        for (int seg = 0; seg < 3 && ok; ++seg) {
+          const int seg_end = seg == 0 ? cut1 : (seg == 1 ? cut2 : num_kb);
+          if (kb >= seg_end) continue;
+          const bool a_mn = kb < kb_a, b_mn = kb < kb_b;
           const uint32_t idesc = ptx::make_idesc_bf16(256, 128 * pt.nbw, a_mn ? 1 : 0, b_mn ? 1 : 0);
-          if (!ptx::mbar_wait(ptx::smem_u32(&bars->full[stage]), phase, abort_flag)) {
-            report_timeout(P, mat);
-            ok = false;
-            break;
-          }
-          ptx::tc_fence_after();
-          const uint32_t sa = ptx::smem_u32(ring + stage * kStageBytes);
-          const uint32_t sb = sa + kTileABytes;
-#pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) {
-            const uint64_t da = a_mn ? ptx::smem_desc_sw128(sa + k * 2048, 8192, 1024)
-                                     : ptx::smem_desc_sw128(sa + k * 32, 16, 1024);
-            const uint64_t db = b_mn ? ptx::smem_desc_sw128(sb + k * 2048, 8192, 1024)
-                                     : ptx::smem_desc_sw128(sb + k * 32, 16, 1024);
-            ptx::umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
-          }
-          ptx::umma_commit_pair(ptx::smem_u32(&bars->empty[stage]), 3);
-          if (++stage == kStages) {
-            stage = 0;
-            phase ^= 1u;
+          const uint32_t a_fix = a_mn ? kLboMN : kLboK, b_fix = (b_mn ? kLboMN : kLboK) + (kTileABytes >> 4);
+          const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
+#pragma unroll 1
+          for (; kb < seg_end; ++kb) {
+            if (!ptx::mbar_wait(full0 + stage * 8, phase, abort_flag)) {
+              report_timeout(P, mat);
+              ok = false;
+              break;
+            }
+            ptx::tc_fence_after();
+            const uint32_t enc = ring_enc + stage * (kStageBytes >> 4);
+            const uint32_t a_lo = enc + a_fix, b_lo = enc + b_fix;
+            ptx::umma_bf16_pair_lohi(d_tmem, a_lo, b_lo, kDescHi, idesc, accumulate);
+            ptx::umma_bf16_pair_lohi(d_tmem, a_lo + a_step, b_lo + b_step, kDescHi, idesc, 1u);
+            ptx::umma_bf16_pair_lohi(d_tmem, a_lo + 2 * a_step, b_lo + 2 * b_step, kDescHi, idesc, 1u);
+            ptx::umma_bf16_pair_lohi(d_tmem, a_lo + 3 * a_step, b_lo + 3 * b_step, kDescHi, idesc, 1u);
+            accumulate = 1u;
+            ptx::umma_commit_pair(empty0 + stage * 8, 3);
+            if (++stage == kStages) {
+              stage = 0;
+              phase ^= 1u;
+            }
           }
         }
         if (!ok) break;
@@ -341,7 +358,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
     for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
       cur.open_tile(P, tile, total_tiles, static_cast<int>(rank));
       const int mat = cur.mat;
-      ok = ptx::mbar_wait(ptx::smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag);
+      ok = ptx::mbar_wait_relaxed(ptx::smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);  // the warp goes on or gives up as one
       if (!ok) {
         if (lane == 0) report_timeout(P, mat);
