@@ -172,7 +172,10 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
 
   if (warp == 0) {
     // ------------------------------------------------------ TMA producer ----
-    if (lane == 0) {
+    // The whole warp walks the loop (so that its counters stay warp-uniform);
+    // one elected lane issues the copies.
+    {
+      const bool elected = ptx::elect_one();
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       const uint32_t ring_u32 = ptx::smem_u32(ring);
@@ -191,29 +194,33 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         const int kb_b = P.b_mn_major ? num_kb
                                       : (P.b_sym ? min(num_kb, 2 * (pt.nbw == 2 ? pt.jb + 1 : pt.jb)) : 0);
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!ptx::mbar_wait(empty0 + stage * 8, phase ^ 1u, abort_flag)) {
-            report_timeout(P, mat);
-            ok = false;
+          ok = ptx::mbar_wait(empty0 + stage * 8, phase ^ 1u, abort_flag);
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) {
+            if (elected) report_timeout(P, mat);
             break;
           }
-          const uint32_t leader_full = leader_full0 + stage * 8;
-          const uint32_t sa = ring_u32 + stage * kStageBytes;
-          const uint32_t sb = sa + kTileABytes;
-          const int k0 = kb * kBK;
-          if (rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, stage_tx);
-          if (kb >= kb_a) {
-            ptx::tma_load_3d_pair(sa, &P.map_a, k0, row0, mat, leader_full);
-          } else {
-            ptx::tma_load_3d_pair(sa, &P.map_a64, row0, k0, mat, leader_full);
-            ptx::tma_load_3d_pair(sa + 8192, &P.map_a64, row0 + 64, k0, mat, leader_full);
+          if (elected) {
+            const uint32_t leader_full = leader_full0 + stage * 8;
+            const uint32_t sa = ring_u32 + stage * kStageBytes;
+            const uint32_t sb = sa + kTileABytes;
+            const int k0 = kb * kBK;
+            if (rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, stage_tx);
+            if (kb >= kb_a) {
+              ptx::tma_load_3d_pair(sa, &P.map_a, k0, row0, mat, leader_full);
+            } else {
+              ptx::tma_load_3d_pair(sa, &P.map_a64, row0, k0, mat, leader_full);
+              ptx::tma_load_3d_pair(sa + 8192, &P.map_a64, row0 + 64, k0, mat, leader_full);
+            }
+            if (kb >= kb_b) {
+              ptx::tma_load_3d_pair(sb, &P.map_b, k0, b0, mat, leader_full);
+              if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, &P.map_b, k0, b0 + 64, mat, leader_full);
+            } else {
+              ptx::tma_load_3d_pair(sb, &P.map_b, b0, k0, mat, leader_full);
+              if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, &P.map_b, b0 + 64, k0, mat, leader_full);
+            }
           }
-          if (kb >= kb_b) {
-            ptx::tma_load_3d_pair(sb, &P.map_b, k0, b0, mat, leader_full);
-            if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, &P.map_b, k0, b0 + 64, mat, leader_full);
-          } else {
-            ptx::tma_load_3d_pair(sb, &P.map_b, b0, k0, mat, leader_full);
-            if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, &P.map_b, b0 + 64, k0, mat, leader_full);
-          }
+          __syncwarp();
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
@@ -229,7 +236,10 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
     // The issuing thread is the pacemaker of the tensor pipe, so its loop is
     // kept short: the shared-memory descriptors differ only in the low word
     // (encoded start address), which advances by a constant per K = 16 step.
-    if (lane == 0 && rank == 0) {
+    // The whole warp walks the loop, so the operands of the UMMA instructions are
+    // warp-uniform values; one elected lane issues them and their commits.
+    if (rank == 0) {
+      const bool elected = ptx::elect_one();
       uint32_t stage = 0, phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
@@ -246,9 +256,10 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         const int kb_a = P.a_sym ? min(num_kb, 2 * (2 * pt.p + 1)) : 0;
         const int kb_b = P.b_mn_major ? num_kb
                                       : (P.b_sym ? min(num_kb, 2 * (pt.nbw == 2 ? pt.jb + 1 : pt.jb)) : 0);
-        if (!ptx::mbar_wait(ptx::smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag)) {
-          report_timeout(P, mat);
-          ok = false;
+        ok = ptx::mbar_wait(ptx::smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) {
+          if (elected) report_timeout(P, mat);
           break;
         }
         ptx::tc_fence_after();
@@ -267,20 +278,24 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
 #pragma unroll 1
           for (; kb < seg_end; ++kb) {
-            if (!ptx::mbar_wait(full0 + stage * 8, phase, abort_flag)) {
-              report_timeout(P, mat);
-              ok = false;
+            ok = ptx::mbar_wait(full0 + stage * 8, phase, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) {
+              if (elected) report_timeout(P, mat);
               break;
             }
             ptx::tc_fence_after();
             const uint32_t enc = ring_enc + stage * (kStageBytes >> 4);
             const uint32_t a_lo = enc + a_fix, b_lo = enc + b_fix;
-            ptx::umma_bf16_pair_lohi(d_tmem, a_lo, b_lo, kDescHi, idesc, accumulate);
-            ptx::umma_bf16_pair_lohi(d_tmem, a_lo + a_step, b_lo + b_step, kDescHi, idesc, 1u);
-            ptx::umma_bf16_pair_lohi(d_tmem, a_lo + 2 * a_step, b_lo + 2 * b_step, kDescHi, idesc, 1u);
-            ptx::umma_bf16_pair_lohi(d_tmem, a_lo + 3 * a_step, b_lo + 3 * b_step, kDescHi, idesc, 1u);
+            if (elected) {
+              ptx::umma_bf16_pair_lohi(d_tmem, a_lo, b_lo, kDescHi, idesc, accumulate);
+              ptx::umma_bf16_pair_lohi(d_tmem, a_lo + a_step, b_lo + b_step, kDescHi, idesc, 1u);
+              ptx::umma_bf16_pair_lohi(d_tmem, a_lo + 2 * a_step, b_lo + 2 * b_step, kDescHi, idesc, 1u);
+              ptx::umma_bf16_pair_lohi(d_tmem, a_lo + 3 * a_step, b_lo + 3 * b_step, kDescHi, idesc, 1u);
+              ptx::umma_commit_pair(empty0 + stage * 8, 3);
+            }
+            __syncwarp();
             accumulate = 1u;
-            ptx::umma_commit_pair(empty0 + stage * 8, 3);
             if (++stage == kStages) {
               stage = 0;
               phase ^= 1u;
@@ -288,7 +303,8 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           }
         }
         if (!ok) break;
-        ptx::umma_commit_pair(ptx::smem_u32(&bars->acc_full[acc]), 3);
+        if (elected) ptx::umma_commit_pair(ptx::smem_u32(&bars->acc_full[acc]), 3);
+        __syncwarp();
         if (++acc == kNumAcc) {
           acc = 0;
           acc_phase ^= 1u;
