@@ -171,6 +171,26 @@ def oracle_sample_time(specs, hp_dict, budget_s=20.0, max_mats=4):
     return flops, secs, "%d oracle steps on single matrices of %s" % (len(done), ", ".join(uniq)), threads
 
 
+def rank_seed(cfg, group_index, rank):
+    """Seed of one group's tensors on one rank: every rank owns its own shard
+    of equally many matrices (weak scaling), drawn from a different stream."""
+    return 1000 * cfg + group_index + 100000 * rank
+
+
+def max_over_ranks(value, dist, device):
+    """MAX-reduce of a scalar over the process group (identity without one)."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([float(value)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(flops_per_rank, world, ms_per_step):
+    """Aggregate metric: the work of all ranks over the slowest rank's time."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 def hp_dict_default():
     return dict(lr=4.2e-4, wd=0.1, mu=0.95, nesterov=True, ns_steps=5, a=3.4445, b=-4.7750, c=2.0315,
                 eps=1e-7, rms_scale=0.2)
@@ -254,7 +274,7 @@ def main():
     # Inputs: seeded, drawn on the device (each rank its own shard of equal size).
     groups, state = [], []
     for gi, sp in enumerate(specs):
-        W, G, M = wl.make_group(sp, 1000 * args.config + gi + 100000 * rank, dev)
+        W, G, M = wl.make_group(sp, rank_seed(args.config, gi, rank), dev)
         state.append((W, G, M))
         groups.append((wl.views(W), wl.views(G), wl.views(M)))
     ctx = binding.MuonContext(groups)
@@ -294,12 +314,9 @@ def main():
     status, which = ctx.muon_status()
     if status != 0:
         raise SystemExit("device status %d at matrix %d in the timed region" % (status, which))
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, dev)
     ms_step = ms_total / args.steps
-    value = world * alg_flops / (ms_step * 1e-3) / 1e12
+    value = whole_job_value(alg_flops, world, ms_step)
 
     # ---- end to end through muon_step_host --------------------------------------
     e2e = None
@@ -322,12 +339,8 @@ def main():
         e1.record(stream)
         barrier()
         ms_e2e = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        ms_e2e /= e2e_steps
-        e2e = {"value": world * alg_flops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e,
+        ms_e2e = max_over_ranks(ms_e2e, dist, dev) / e2e_steps
+        e2e = {"value": whole_job_value(alg_flops, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
 
     if rank != 0:
