@@ -101,4 +101,19 @@ struct StreamParams {
   int nesterov;
 };
 
+// Parameters of the TMA-pipelined momentum kernel (64 x 64 tiles).
+struct StreamTmaParams {
+  CUtensorMap map_x;         // bf16 X buffer [count][m][ldx], box {64, 64}, 128B swizzle
+  const CUtensorMap* gmaps;  // per matrix (chunk-relative): G, box {64, 64}, no swizzle
+  const CUtensorMap* mmaps;  // per matrix: M (fp32), box {64, 64}, no swizzle
+  const MatDesc* descs;
+  float* partials;           // [count][tiles_per_matrix]
+  DevStatus* status;
+  int count;
+  int tiles_per_matrix;      // ceil(m / 64) * ceil(n / 64)
+  int m, n;                  // short and long side of the bucket
+  float mu;
+  int nesterov;
+};
+
 }  // namespace muon

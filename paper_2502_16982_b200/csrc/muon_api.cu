@@ -29,6 +29,8 @@ cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, cons
                                  long long x_stride, int ldx, int count, long long elems,
                                  float upd_scale, float decay, bool use_inv_norm, bool w_fp32,
                                  cudaStream_t stream);
+cudaError_t stream_tma_configure();
+cudaError_t launch_momentum_tma(const StreamTmaParams& P, bool grad_fp32, int num_sms, cudaStream_t stream);
 cudaError_t gemm_configure();
 cudaError_t gemm_max_clusters(int* out);
 cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream);
@@ -65,12 +67,15 @@ struct Bucket {
   int chunk;        // matrices per chunk
   int ldx, lda;
   size_t x_stride, a_stride;  // elements per matrix
-  int stream_tiles;           // CTAs per matrix of the streaming kernel
+  int stream_tiles;           // per-matrix partial sums reserved for the streaming kernels
+  int stream_tiles_generic;   // tiles per matrix of the generic streaming kernel (64 x 128)
+  int stream_tiles_tma;       // tiles per matrix of the TMA streaming kernel (64 x 64)
   bool fused_update;          // every W is bf16 and TMA-addressable: update W in the last epilogue
+  bool stream_tma;            // every G and M is TMA-addressable: TMA-pipelined momentum kernel
   // workspace offsets (bytes) of the chunk buffers
   size_t off_x[2], off_a, off_b, off_partials, off_scal;
   // workspace offsets of the persistent per-bucket tables
-  size_t off_descs, off_wmaps, off_sym_tiles, off_comb_tiles;
+  size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_comb_tiles;
   std::vector<PairTile> sym_tiles, comb_tiles;  // tile tables of one matrix
   int sym_acc_cols, comb_acc_cols;              // widest tile of each table (128 or 256)
   // tensor maps over the chunk buffers (all 128-byte swizzled)
@@ -121,6 +126,24 @@ int encode_map(CUtensorMap* out, void* base, int cols, int rows, int count, int 
                   CU_TENSOR_MAP_INTERLEAVE_NONE,
                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(MUON_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return MUON_OK;
+}
+
+// Map over one caller-owned matrix [rows][cols] of bf16 or fp32 with row pitch
+// ld elements: box {64, 64}, not swizzled (tiles of the streaming kernel).
+int encode_stream_map(CUtensorMap* out, const void* base, int rows, int cols, long long ld, bool fp32) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return fail(MUON_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
+  const cuuint64_t es = fp32 ? 4 : 2;
+  cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows), 1};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld) * es, static_cast<cuuint64_t>(ld) * es * rows};
+  cuuint32_t box[3] = {64, 64, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(out, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                  const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(MUON_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
   return MUON_OK;
 }
@@ -208,7 +231,9 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     // tile counts of the streaming kernel for both stored orientations
     const int t1 = ceil_div(B.m, kSTR) * ceil_div(B.n, kSTC);
     const int t2 = ceil_div(B.n, kSTR) * ceil_div(B.m, kSTC);
-    B.stream_tiles = std::max(t1, t2);
+    B.stream_tiles_generic = std::max(t1, t2);
+    B.stream_tiles_tma = ceil_div(B.m, 64) * ceil_div(B.n, 64);
+    B.stream_tiles = std::max(B.stream_tiles_generic, B.stream_tiles_tma);
     const size_t per_mat = 2 * B.x_stride * 2 + 2 * B.a_stride * 2;
     size_t chunk = std::max<size_t>(1, kChunkBytesMax / per_mat);
     chunk = std::min<size_t>(chunk, B.mats.size());
@@ -237,6 +262,10 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     B.off_descs = off;
     off = align_up(off + B.mats.size() * sizeof(MatDesc), 1024);
     B.off_wmaps = off;
+    off = align_up(off + B.mats.size() * sizeof(CUtensorMap), 1024);
+    B.off_gmaps = off;
+    off = align_up(off + B.mats.size() * sizeof(CUtensorMap), 1024);
+    B.off_mmaps = off;
     off = align_up(off + B.mats.size() * sizeof(CUtensorMap), 1024);
     // tile tables: row pair p covers row blocks 2p, 2p+1; column tiles are two
     // 128-blocks wide, with one single block at the end of an odd run
@@ -392,6 +421,7 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   }
   ctx->num_sms = prop.multiProcessorCount;
   ce = gemm_configure();
+  if (ce == cudaSuccess) ce = stream_tma_configure();
   if (ce == cudaSuccess) ce = gemm_max_clusters(&ctx->max_clusters);
   if (ce == cudaSuccess && ctx->max_clusters < 1) ctx->max_clusters = 1;
   if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(ce)); }
@@ -418,6 +448,8 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     Bucket& B = ctx->buckets[b];
     std::vector<MatDesc> descs(B.mats.size());
     B.fused_update = (B.w_dtype == MUON_DTYPE_BF16);
+    B.stream_tma = true;
+    const long long g_es = B.g_dtype == MUON_DTYPE_FP32 ? 4 : 2;
     for (size_t i = 0; i < B.mats.size(); ++i) {
       const MatRef& r = B.mats[i];
       const muon_group& G = ctx->groups[r.group];
@@ -438,6 +470,9 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
       descs[i] = d;
       ctx->where[r.global] = std::make_pair(static_cast<int>(b), static_cast<int>(i));
       if (!w_tma_ok(d.w, d.ld_w) || d.ld_w > (1ll << 31)) B.fused_update = false;
+      if ((reinterpret_cast<uintptr_t>(d.g) & 15) || (d.ld_g * g_es) % 16 || (reinterpret_cast<uintptr_t>(d.m) & 15) ||
+          (d.ld_m * 4) % 16)
+        B.stream_tma = false;
     }
     ce = cudaMemcpy(ctx->ws + B.off_descs, descs.data(), descs.size() * sizeof(MatDesc), cudaMemcpyHostToDevice);
     if (ce == cudaSuccess)
@@ -452,6 +487,18 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
         rc = encode_w_map(&wmaps[i], descs[i].w, descs[i].rows, descs[i].cols, descs[i].ld_w);
       if (rc != MUON_OK) { delete ctx; return rc; }
       ce = cudaMemcpy(ctx->ws + B.off_wmaps, wmaps.data(), wmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+    }
+    if (ce == cudaSuccess && B.stream_tma) {
+      std::vector<CUtensorMap> gmaps(B.mats.size()), mmaps(B.mats.size());
+      for (size_t i = 0; i < B.mats.size() && rc == MUON_OK; ++i) {
+        rc = encode_stream_map(&gmaps[i], descs[i].g, descs[i].rows, descs[i].cols, descs[i].ld_g,
+                               B.g_dtype == MUON_DTYPE_FP32);
+        if (rc == MUON_OK) rc = encode_stream_map(&mmaps[i], descs[i].m, descs[i].rows, descs[i].cols, descs[i].ld_m, true);
+      }
+      if (rc != MUON_OK) { delete ctx; return rc; }
+      ce = cudaMemcpy(ctx->ws + B.off_gmaps, gmaps.data(), gmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
+      if (ce == cudaSuccess)
+        ce = cudaMemcpy(ctx->ws + B.off_mmaps, mmaps.data(), mmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
     }
     if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "descriptor upload: %s", cudaGetErrorString(ce)); }
 
@@ -514,20 +561,40 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
       MatScal* scal = reinterpret_cast<MatScal*>(ctx->ws + B.off_scal);
       float* partials = reinterpret_cast<float*>(ctx->ws + B.off_partials);
 
-      StreamParams S{};
-      S.descs = descs;
-      S.partials = partials;
-      S.x = reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_x[0]);
-      S.x_stride = static_cast<long long>(B.x_stride);
-      S.ldx = B.ldx;
-      S.count = count;
-      S.tiles_per_matrix = B.stream_tiles;
-      S.mu = hp->mu;
-      S.nesterov = hp->nesterov ? 1 : 0;
-      { LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM); ce = launch_momentum_cast(S, B.g_dtype == MUON_DTYPE_FP32, stream); }
+      const int stream_tiles = B.stream_tma ? B.stream_tiles_tma : B.stream_tiles_generic;
+      if (B.stream_tma) {
+        StreamTmaParams S{};
+        S.map_x = B.x_b64[0];
+        S.gmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_gmaps) + first;
+        S.mmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_mmaps) + first;
+        S.descs = descs;
+        S.partials = partials;
+        S.status = status;
+        S.count = count;
+        S.tiles_per_matrix = stream_tiles;
+        S.m = B.m;
+        S.n = B.n;
+        S.mu = hp->mu;
+        S.nesterov = hp->nesterov ? 1 : 0;
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM);
+        ce = launch_momentum_tma(S, B.g_dtype == MUON_DTYPE_FP32, ctx->num_sms, stream);
+      } else {
+        StreamParams S{};
+        S.descs = descs;
+        S.partials = partials;
+        S.x = reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_x[0]);
+        S.x_stride = static_cast<long long>(B.x_stride);
+        S.ldx = B.ldx;
+        S.count = count;
+        S.tiles_per_matrix = stream_tiles;
+        S.mu = hp->mu;
+        S.nesterov = hp->nesterov ? 1 : 0;
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM);
+        ce = launch_momentum_cast(S, B.g_dtype == MUON_DTYPE_FP32, stream);
+      }
       if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "momentum kernel launch: %s", cudaGetErrorString(ce));
       ++launches;
-      { LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM); ce = launch_norm_finalise(partials, B.stream_tiles, count, hp->eps, descs, scal, norms, status, stream); }
+      { LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM); ce = launch_norm_finalise(partials, stream_tiles, count, hp->eps, descs, scal, norms, status, stream); }
       if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "norm kernel launch: %s", cudaGetErrorString(ce));
       ++launches;
 

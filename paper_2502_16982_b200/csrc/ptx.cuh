@@ -173,6 +173,11 @@ __device__ __forceinline__ void tma_store_wait_read_all_but_one() {
   asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
 }
 
+// The same, leaving the two most recent groups pending.
+__device__ __forceinline__ void tma_store_wait_read_all_but_two() {
+  asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory");
+}
+
 // Wait until every committed store is complete (globally visible).
 __device__ __forceinline__ void tma_store_wait_all() {
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
