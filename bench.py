@@ -51,6 +51,10 @@ WORKLOAD_NAMES = {
     5: "cfg5: Moonlight-shaped full parameter set (5286 matrices, 15.3 G params)",
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/, taken on 64 matrices of the expert-bucket shapes; it scales with the matrix count.
+NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": 12.62e9, "gemm_launches_per_step": 15,
+               "momentum_bytes_per_launch": 2.158e9}
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 
@@ -370,13 +374,20 @@ def main():
             "flops_per_launch": alg_flops * args.steps / gemm_launches,
             "traffic": None,
         }
+        if args.config == 3 and hp.ns_steps == 5:
+            scale = sum(s.count for s in specs) / NCU_CAPTURE["matrices"]
+            roofline["traffic"] = NCU_CAPTURE["gemm_bytes_per_step"] * scale / NCU_CAPTURE["gemm_launches_per_step"]
+            roofline["traffic_note"] = "DRAM bytes per launch (average of the 15 launches of a step), scaled from a 64-matrix ncu capture"
     stream_roof = None
     if mom_launches:
         gbs = sbytes * args.steps / (mom_ms * 1e-3) / 1e9
-        stream_roof = {"kernel": "momentum_cast_kernel", "bound": "hbm", "achieved": gbs,
+        stream_roof = {"kernel": "momentum_tma_kernel", "bound": "hbm", "achieved": gbs,
                        "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]),
                        "peak_source": "%s hbm_gbs" % peaks["_source"], "frac_of_nominal": gbs / NOMINAL_HBM_GBS,
-                       "bytes_per_element": sbytes / wl.group_params(specs), "traffic": None}
+                       "bytes_per_element": sbytes / wl.group_params(specs), "traffic": None,
+                       "algorithmic_bytes_per_launch": sbytes / max(1, mom_launches // args.steps)}
+        if args.config == 3:
+            stream_roof["traffic"] = NCU_CAPTURE["momentum_bytes_per_launch"] * sum(s.count for s in specs) / NCU_CAPTURE["matrices"]
 
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:
