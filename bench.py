@@ -389,6 +389,37 @@ def main():
         if args.config == 3:
             stream_roof["traffic"] = NCU_CAPTURE["momentum_bytes_per_launch"] * sum(s.count for s in specs) / NCU_CAPTURE["matrices"]
 
+    # ---- shape sweep: every shape of the configuration on its own ---------------------
+    shapes = None
+    if args.config == 4 and world == 1:
+        shapes = []
+        ctx.muon_destroy()
+        for gi, sp in enumerate(specs):
+            one = binding.MuonContext([groups[gi]])
+            for _ in range(args.warmup):
+                one.muon_step(hp)
+            one.muon_profile_enable(True)
+            torch.cuda.synchronize(dev)
+            e0.record(stream)
+            for _ in range(args.steps):
+                one.muon_step(hp)
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            pr = one.muon_profile_read()
+            one.muon_profile_enable(False)
+            ms = e0.elapsed_time(e1) / args.steps
+            g_ms = sum(pr[k][0] for k in ("gram", "poly", "comb")) / args.steps
+            fl, _ = wl.ns_flops([sp], hp.ns_steps)
+            m_, n_ = min(sp.rows, sp.cols), max(sp.rows, sp.cols)
+            blocks, pairs = -(-m_ // 128), -(-(-(-m_ // 128)) // 2)
+            shapes.append({"shape": "%dx%d" % (sp.rows, sp.cols), "ms_per_step": ms,
+                           "step_tflops": fl / (ms * 1e-3) / 1e12,
+                           "gemm_tflops": fl / (g_ms * 1e-3) / 1e12,
+                           "gemm_frac_of_measured_sustained": fl / (g_ms * 1e-3) / 1e12 / float(peaks.get("bf16_tflops_sustained", 1400.0)),
+                           "row_blocks": blocks, "cta_pairs_per_column_tile": pairs})
+            one.muon_destroy()
+        ctx = binding.MuonContext(groups)
+
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:
         fl, secs, desc, threads = oracle_sample_time(specs, hpd, budget_s=args.ref_budget, max_mats=args.ref_mats)
@@ -409,6 +440,8 @@ def main():
         "roofline": roofline, "roofline_stream": stream_roof, "kernels": per_kernel,
         "cpu_baseline": cpu_baseline,
     }
+    if shapes is not None:
+        line["shapes"] = shapes
     print(json.dumps(line))
     ctx.muon_destroy()
     if dist is not None:

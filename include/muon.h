@@ -210,6 +210,16 @@ int muon_debug_keep(muon_ctx* ctx, int keep);
 int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, size_t dst_bytes);
 
 /*
+ * Test knob: upper bound, in bytes, on the Newton-Schulz operands (X, A, B) of
+ * one bucket chunk; a bucket that needs more is processed in several chunks
+ * that reuse the workspace.  Process-wide, read by muon_workspace_bytes and
+ * muon_init (a context keeps the plan it was created with).  0 restores the
+ * default of 8 GiB.  Returns the previous value.  Tests lower it to run the
+ * chunked path on small buckets.
+ */
+size_t muon_debug_set_chunk_bytes(size_t bytes);
+
+/*
  * Test tap: the TMEM base address each CTA of the last Newton-Schulz GEMM launch
  * obtained (indexed by CTA; 0xFFFFFFFF where no CTA ran).  Copies `n` (at most
  * 1024) values to the HOST array.  Synchronises the device.

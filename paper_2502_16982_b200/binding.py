@@ -31,7 +31,7 @@ MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
 EXPORTED = [
     "muon_workspace_bytes", "muon_init", "muon_step", "muon_step_host", "muon_status",
     "muon_get_norms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
-    "muon_debug_keep", "muon_debug_read",
+    "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
     "muon_momentum_norm_static",
 ]
@@ -93,8 +93,11 @@ def lib():
     L.muon_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int)]
     L.muon_momentum_norm_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64,
                                             C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
+    L.muon_debug_set_chunk_bytes.argtypes = [C.c_size_t]
     for name in EXPORTED:
-        if name != "muon_last_error":
+        if name == "muon_debug_set_chunk_bytes":
+            getattr(L, name).restype = C.c_size_t
+        elif name != "muon_last_error":
             getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -198,6 +201,12 @@ def muon_momentum_norm_static(g, m, mu: float, nesterov: bool, norm_out, stream=
     _check(lib().muon_momentum_norm_static(
         C.c_void_p(g.data_ptr()), C.c_void_p(m.data_ptr()), rows, cols, ld_g, ld_m, _dtype_code(g),
         float(mu), int(bool(nesterov)), C.c_void_p(norm_out.data_ptr()), dev, C.c_void_p(s.cuda_stream)))
+
+
+def muon_debug_set_chunk_bytes(nbytes: int) -> int:
+    """Test knob: bound on the Newton-Schulz operand bytes of one bucket chunk
+    (0 = default).  Returns the previous value."""
+    return lib().muon_debug_set_chunk_bytes(int(nbytes))
 
 
 class MuonContext:

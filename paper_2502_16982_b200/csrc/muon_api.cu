@@ -53,7 +53,8 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // Upper bound on the Newton-Schulz operand bytes of one chunk; larger buckets
 // are processed in several chunks that reuse the same workspace.
-constexpr size_t kChunkBytesMax = size_t(8) << 30;
+constexpr size_t kChunkBytesDefault = size_t(8) << 30;
+size_t g_chunk_bytes_max = kChunkBytesDefault;  // process-wide; see muon_debug_set_chunk_bytes
 constexpr int kChunkCountMax = 4096;
 
 struct MatRef {
@@ -235,7 +236,7 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     B.stream_tiles_tma = ceil_div(B.m, 64) * ceil_div(B.n, 64);
     B.stream_tiles = std::max(B.stream_tiles_generic, B.stream_tiles_tma);
     const size_t per_mat = 2 * B.x_stride * 2 + 2 * B.a_stride * 2;
-    size_t chunk = std::max<size_t>(1, kChunkBytesMax / per_mat);
+    size_t chunk = std::max<size_t>(1, g_chunk_bytes_max / per_mat);
     chunk = std::min<size_t>(chunk, B.mats.size());
     chunk = std::min<size_t>(chunk, kChunkCountMax);
     // keep the streaming grid within 2^31 CTAs
@@ -368,6 +369,12 @@ struct LaunchTimer {
 extern "C" {
 
 const char* muon_last_error(void) { return g_last_error.c_str(); }
+
+size_t muon_debug_set_chunk_bytes(size_t bytes) {
+  const size_t prev = g_chunk_bytes_max;
+  g_chunk_bytes_max = bytes ? bytes : kChunkBytesDefault;
+  return prev;
+}
 
 int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_bytes) {
   if (!out_bytes) return fail(MUON_ERR_INVALID_ARG, "out_bytes is null");

@@ -275,6 +275,31 @@ def test_column_slices_of_wider_buffers(rows, cols, off):
         ctx.muon_destroy()
 
 
+def test_chunked_bucket_matches_the_oracle():
+    """A bucket larger than the chunk limit is processed in several chunks that
+    reuse the workspace (as the 3432-matrix expert buckets of the full
+    Moonlight-shaped set are): 7 matrices, 3 per chunk, both orientations."""
+    b = _binding()
+    specs = [wl.GroupSpec(264, 200, 4, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
+             wl.GroupSpec(200, 264, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True)]
+    per_matrix = (2 * 200 * 320 + 2 * 200 * 256) * 2  # two X buffers, A and B, bf16, padded pitches
+    prev = b.muon_debug_set_chunk_bytes(3 * per_matrix + 64)
+    try:
+        case = Case(specs, seed=31)
+    finally:
+        b.muon_debug_set_chunk_bytes(prev)
+    try:
+        assert case.ctx.workspace_bytes < 5 * per_matrix  # really chunked: room for 3 matrices, not 7
+        hp = default_hp(lr=4.2e-4, wd=0.1)
+        check_step(case, hp)
+        gen = torch.Generator().manual_seed(32)
+        for gi, sp in enumerate(specs):
+            case.dev[gi][1].copy_(wl.make_grads(sp, gen, "cpu"))
+        check_step(case, hp)
+    finally:
+        case.close()
+
+
 def test_bitwise_reproducible():
     specs = [wl.GroupSpec(448, 640, 4, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
     outs = []
