@@ -164,6 +164,16 @@ int muon_status(muon_ctx* ctx, void* stream, int* device_status, int* matrix_ind
  */
 int muon_get_norms(muon_ctx* ctx, void* stream, float* out, int n);
 
+/*
+ * Per-matrix update RMS of the last step, the value Algorithm 1 returns for
+ * logging: sqrt(mean(u^2)) with u = rms_scale * sqrt(max(rows, cols)) * O (the
+ * scaled update before the learning rate; it sits near 0.2 by Sec. 2.2's
+ * design).  Copies `n` floats (global matrix order) to the HOST array `out`
+ * after synchronising `stream`.  A matrix whose input was non-finite reports
+ * an unspecified value.
+ */
+int muon_get_update_rms(muon_ctx* ctx, void* stream, float* out, int n);
+
 /* Free the host-side context.  Never touches caller memory. */
 int muon_destroy(muon_ctx* ctx);
 

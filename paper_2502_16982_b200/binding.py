@@ -30,7 +30,7 @@ MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
 
 EXPORTED = [
     "muon_workspace_bytes", "muon_init", "muon_step", "muon_step_host", "muon_status",
-    "muon_get_norms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
+    "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
     "muon_momentum_norm_static",
@@ -83,6 +83,7 @@ def lib():
                                  C.POINTER(C.POINTER(C.c_void_p)), C.c_void_p]
     L.muon_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     L.muon_get_norms.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_float), C.c_int]
+    L.muon_get_update_rms.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_float), C.c_int]
     L.muon_destroy.argtypes = [C.c_void_p]
     L.muon_last_error.restype = C.c_char_p
     L.muon_last_launch_count.argtypes = [C.c_void_p]
@@ -276,6 +277,13 @@ class MuonContext:
         s = torch.cuda.current_stream(self.device) if stream is None else stream
         out = (C.c_float * self.n_matrices)()
         _check(lib().muon_get_norms(self._ctx, C.c_void_p(s.cuda_stream), out, self.n_matrices))
+        return list(out)
+
+    def muon_get_update_rms(self, stream=None):
+        import torch
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        out = (C.c_float * self.n_matrices)()
+        _check(lib().muon_get_update_rms(self._ctx, C.c_void_p(s.cuda_stream), out, self.n_matrices))
         return list(out)
 
     def muon_last_launch_count(self) -> int:

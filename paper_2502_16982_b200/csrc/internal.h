@@ -86,6 +86,7 @@ struct GemmParams {
   const MatDesc* descs;
   const MatScal* scal;
   DevStatus* status;
+  float* rms_partials;  // last iteration: sums of O^2, [matrix][tile][CTA of the pair][epilogue warp]
   unsigned* debug;  // optional: TMEM base addresses seen by each CTA (test tap)
 };
 

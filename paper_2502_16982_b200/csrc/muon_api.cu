@@ -29,6 +29,11 @@ cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, cons
                                  long long x_stride, int ldx, int count, long long elems,
                                  float upd_scale, float decay, bool use_inv_norm, bool w_fp32,
                                  cudaStream_t stream);
+cudaError_t launch_rms_finalise(const float* partials, int per_matrix, int count, float factor,
+                                const MatDesc* descs, float* rms, cudaStream_t stream);
+cudaError_t launch_rms_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
+                              long long x_stride, int ldx, int m, int n, int count, float factor,
+                              bool use_inv_norm, float* rms, cudaStream_t stream);
 cudaError_t stream_tma_configure();
 cudaError_t launch_momentum_tma(const StreamTmaParams& P, bool grad_fp32, int num_sms, cudaStream_t stream);
 cudaError_t gemm_configure();
@@ -74,7 +79,7 @@ struct Bucket {
   bool fused_update;          // every W is bf16 and TMA-addressable: update W in the last epilogue
   bool stream_tma;            // every G and M is TMA-addressable: TMA-pipelined momentum kernel
   // workspace offsets (bytes) of the chunk buffers
-  size_t off_x[2], off_a, off_b, off_partials, off_scal;
+  size_t off_x[2], off_a, off_b, off_partials, off_scal, off_rms_partials;
   // workspace offsets of the persistent per-bucket tables
   size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_comb_tiles;
   std::vector<PairTile> sym_tiles, comb_tiles;  // tile tables of one matrix
@@ -92,6 +97,7 @@ struct PlanSizes {
   size_t total;
   size_t off_status;
   size_t off_norms;  // float per matrix (global order)
+  size_t off_rms;    // float per matrix: update RMS of the last step
   size_t off_debug;  // TMEM base addresses seen by the CTAs of the pair kernel
 };
 
@@ -254,6 +260,12 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     B.off_b = take(chunk * B.a_stride * 2);
     B.off_partials = take(chunk * static_cast<size_t>(B.stream_tiles) * sizeof(float));
     B.off_scal = take(chunk * sizeof(MatScal));
+    // sums of O^2 of the last epilogue: per matrix, comb tile, CTA of the pair and epilogue warp
+    {
+      const int ncb = ceil_div(B.n, 128), np = ceil_div(ceil_div(B.m, 128), 2);
+      const size_t comb_tiles = static_cast<size_t>(np) * ceil_div(ncb, 2);
+      B.off_rms_partials = take(chunk * comb_tiles * 8 * sizeof(float));
+    }
     chunk_region = std::max(chunk_region, off);
   }
   size_t off = align_up(chunk_region, 1024);
@@ -298,6 +310,8 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
   sizes->off_status = off;
   off = align_up(off + sizeof(DevStatus), 1024);
   sizes->off_norms = off;
+  off = align_up(off + static_cast<size_t>(global) * sizeof(float), 1024);
+  sizes->off_rms = off;
   off = align_up(off + static_cast<size_t>(global) * sizeof(float), 1024);
   sizes->total = off;
   return MUON_OK;
@@ -531,6 +545,7 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     ce = cudaMemcpy(ctx->ws + ctx->sizes.off_status, &init, sizeof(init), cudaMemcpyHostToDevice);
   }
   if (ce == cudaSuccess) ce = cudaMemset(ctx->ws + ctx->sizes.off_norms, 0, ctx->total_mats * sizeof(float));
+  if (ce == cudaSuccess) ce = cudaMemset(ctx->ws + ctx->sizes.off_rms, 0, ctx->total_mats * sizeof(float));
   if (ce == cudaSuccess) ce = cudaMemset(ctx->ws + ctx->sizes.off_debug, 0xFF, 1024 * sizeof(unsigned));
   if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "workspace init: %s", cudaGetErrorString(ce)); }
   *out_ctx = ctx;
@@ -614,6 +629,7 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
         P.scal = scal;
         P.status = status;
         P.debug = reinterpret_cast<unsigned*>(ctx->ws + ctx->sizes.off_debug);
+        P.rms_partials = reinterpret_cast<float*>(ctx->ws + B.off_rms_partials);
         P.wmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_wmaps) + first;
         P.count = count;
         P.m = B.m;
@@ -689,6 +705,22 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "update kernel launch: %s", cudaGetErrorString(ce));
         ++launches;
       }
+      // update RMS for logging (Algorithm 1, returned value): RMS of rms_scale*sqrt(max(rows,cols))*O
+      {
+        float* rms = reinterpret_cast<float*>(ctx->ws + ctx->sizes.off_rms);
+        const float factor = hp->rms_scale * std::sqrt(static_cast<float>(B.n));
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
+        if (hp->ns_steps > 0 && B.fused_update) {
+          ce = launch_rms_finalise(reinterpret_cast<const float*>(ctx->ws + B.off_rms_partials),
+                                   static_cast<int>(B.comb_tiles.size()) * 8, count, factor, descs, rms, stream);
+        } else {
+          ce = launch_rms_from_x(descs, scal, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + B.off_x[cur]),
+                                 static_cast<long long>(B.x_stride), B.ldx, B.m, B.n, count, factor,
+                                 hp->ns_steps == 0, rms, stream);
+        }
+        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
+        ++launches;
+      }
       ctx->x0_buf[b] = 0;
       ctx->xlast_buf[b] = cur;
     }
@@ -751,6 +783,15 @@ int muon_get_norms(muon_ctx* ctx, void* stream_v, float* out, int n) {
   cudaError_t ce = cudaMemcpyAsync(out, ctx->ws + ctx->sizes.off_norms, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
   if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "norm read: %s", cudaGetErrorString(ce));
+  return MUON_OK;
+}
+
+int muon_get_update_rms(muon_ctx* ctx, void* stream_v, float* out, int n) {
+  if (!ctx || !out || n < 0 || n > ctx->total_mats) return fail(MUON_ERR_INVALID_ARG, "bad arguments");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  cudaError_t ce = cudaMemcpyAsync(out, ctx->ws + ctx->sizes.off_rms, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms read: %s", cudaGetErrorString(ce));
   return MUON_OK;
 }
 

@@ -381,6 +381,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         break;
       }
       ptx::tc_fence_after();
+      float o_sq = 0.f;  // last iteration: this lane's sum of O^2 over the tile
       if (cur.has_quarter()) {
         const MatDesc md = P.descs[mat];
         const MatScal sc = P.scal[mat];
@@ -436,8 +437,10 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
               lds128(buf2 + swz, w0, w1, w2, w3);
               unpack8(w0, w1, w2, w3, x);
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
+              for (int i = 0; i < 8; ++i) {
                 o[i] = scale * fmaf(P.c_acc, __uint_as_float(v[c8 * 8 + i]), P.c_in * x[i]);
+                o_sq = fmaf(o[i], o[i], o_sq);
+              }
               if (P.keep_o) {
                 sts128(buf2 + swz, pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
               }
@@ -482,6 +485,15 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           __syncwarp();
         }
         if (!ok) break;
+        if (row0 >= P.m) o_sq = 0.f;  // rows beyond the matrix were never loaded
+      }
+      if (P.last) {
+        // Sum of O^2 of this warp's 32 rows of the tile (Algorithm 1 returns the
+        // update RMS): fixed order within the lane, fixed butterfly across lanes;
+        // one slot per (tile, CTA, warp), written even when it is zero.
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) o_sq += __shfl_xor_sync(0xFFFFFFFFu, o_sq, off);
+        if (lane == 0) P.rms_partials[(static_cast<long long>(tile) * 2 + rank) * kEpiWarps + q] = o_sq;
       }
       // accumulator fully read: hand the TMEM stage back to the leader's issuer
       ptx::tc_fence_before();

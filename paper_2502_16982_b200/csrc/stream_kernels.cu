@@ -256,7 +256,72 @@ __global__ void update_from_x_kernel(const MatDesc* __restrict__ descs,
   }
 }
 
+// Update RMS from the partial sums the last Newton-Schulz epilogue left:
+// rms = |factor| * sqrt(sum O^2 / (rows * cols)), one warp per matrix, fixed order.
+__global__ void rms_finalise_kernel(const float* __restrict__ partials, int per_matrix, int count,
+                                    float factor, const MatDesc* __restrict__ descs,
+                                    float* __restrict__ rms) {
+  const int mat = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (mat >= count) return;
+  const int lane = threadIdx.x & 31;
+  const float* p = partials + static_cast<long long>(mat) * per_matrix;
+  float s = 0.f;
+  for (int i = lane; i < per_matrix; i += 32) s += p[i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  if (lane == 0) {
+    const MatDesc d = descs[mat];
+    rms[d.global_index] = fabsf(factor) * sqrtf(s / (static_cast<float>(d.rows) * static_cast<float>(d.cols)));
+  }
+}
+
+// Update RMS from a stored O (x, short side first, m x n): one CTA per matrix,
+// thread-strided sequential sums and a fixed reduction tree.
+__global__ void __launch_bounds__(256)
+rms_from_x_kernel(const MatDesc* __restrict__ descs, const MatScal* __restrict__ scal,
+                  const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx, int m, int n,
+                  float factor, int use_inv_norm, float* __restrict__ rms) {
+  __shared__ float warp_sums[8];
+  const int mat = blockIdx.x;
+  const __nv_bfloat16* xm = x + mat * x_stride;
+  float s = 0.f;
+  const long long total = static_cast<long long>(m) * n;
+  for (long long i = threadIdx.x; i < total; i += blockDim.x) {
+    const int r = static_cast<int>(i / n), c = static_cast<int>(i - static_cast<long long>(r) * n);
+    const float v = __bfloat162float(xm[static_cast<long long>(r) * ldx + c]);
+    s = fmaf(v, v, s);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < 8; ++w) t += warp_sums[w];
+    const MatScal sc = scal[mat];
+    const float sn = use_inv_norm ? sc.inv_norm : 1.0f;
+    rms[descs[mat].global_index] = fabsf(factor * sn) * sqrtf(t / (static_cast<float>(m) * static_cast<float>(n)));
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_rms_finalise(const float* partials, int per_matrix, int count, float factor,
+                                const MatDesc* descs, float* rms, cudaStream_t stream) {
+  if (count == 0) return cudaSuccess;
+  const int warps = 4;
+  rms_finalise_kernel<<<(count + warps - 1) / warps, warps * 32, 0, stream>>>(partials, per_matrix, count, factor,
+                                                                               descs, rms);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rms_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
+                              long long x_stride, int ldx, int m, int n, int count, float factor,
+                              bool use_inv_norm, float* rms, cudaStream_t stream) {
+  if (count == 0) return cudaSuccess;
+  rms_from_x_kernel<<<count, 256, 0, stream>>>(descs, scal, x, x_stride, ldx, m, n, factor, use_inv_norm ? 1 : 0, rms);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_momentum_cast(const StreamParams& P, bool grad_fp32, cudaStream_t stream) {
   const unsigned grid = static_cast<unsigned>(P.count) * static_cast<unsigned>(P.tiles_per_matrix);

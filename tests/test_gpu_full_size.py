@@ -76,6 +76,9 @@ class DeviceCase:
         assert status == 0, (status, which)
         norms = np.array(self.ctx.muon_get_norms())
         assert np.all(np.isfinite(norms)) and np.all(norms > 0)
+        rms = np.array(self.ctx.muon_get_update_rms())
+        # Lemma 1 / Sec. 2.2: a full-rank update scaled by 0.2*sqrt(max(rows, cols)) has RMS near 0.2
+        assert np.all(rms > 0.1) and np.all(rms < 0.3), (rms.min(), rms.max())
         for gi, (W, G, M) in enumerate(self.state):
             changed = (W != w_before[gi]).flatten(1).any(dim=1)
             assert bool(changed.all()), ("unchanged weight in group", gi)
@@ -87,6 +90,7 @@ class DeviceCase:
             assert rel(f64(M[i]), ref["M"]) <= TOL_FP32, ("M", gi, i)
             nu = norms[self.first[gi] + i]
             assert abs(nu - ref["nu"]) <= TOL_FP32 * ref["nu"], ("nu", gi, i)
+            assert abs(rms[self.first[gi] + i] - ref["rms"]) <= TOL_NS * ref["rms"], ("rms", gi, i)
             upd_rms = float(np.sqrt(np.mean((ref["W"] - W0 + hp.lr * hp.wd * W0) ** 2)))
             frac = bf16_ulp_ok_fraction(W[i], ref["W"], slack=4 * TOL_NS * upd_rms)
             assert frac >= 0.999, ("W ulp", gi, i, frac)

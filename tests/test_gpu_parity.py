@@ -93,6 +93,7 @@ def check_step(case, hp, check_w=True, check_o=False):
     status, which = case.step(hp)
     assert status == 0, (status, which)
     norms = case.ctx.muon_get_norms()
+    rms = case.ctx.muon_get_update_rms()
     gidx = 0
     ohp = to_orc(hp)
     tol_ns = TOL_NS if hp.ns_steps <= 5 else TOL_NS_LONG
@@ -103,6 +104,8 @@ def check_step(case, hp, check_w=True, check_o=False):
             ref = orc.muon_step(W0[i], G0[i], M0[i], ohp)
             assert rel(f64(M[i]), ref["M"]) <= TOL_FP32, ("M", gi, i)
             assert abs(norms[gidx] - ref["nu"]) <= TOL_FP32 * ref["nu"] + 1e-30, ("nu", gi, i)
+            # update RMS returned for logging (Algorithm 1): follows O, so the Newton-Schulz tolerance
+            assert abs(rms[gidx] - ref["rms"]) <= tol_ns * ref["rms"] + 1e-30, ("rms", gi, i, rms[gidx], ref["rms"])
             if check_o and hp.ns_steps > 0:
                 m, n = min(sp.rows, sp.cols), max(sp.rows, sp.cols)
                 o_gpu = f64(case.ctx.muon_debug_read(gidx, case.b.MUON_TAP_X, m, n))
