@@ -61,6 +61,11 @@ enum { MUON_DTYPE_BF16 = 0, MUON_DTYPE_FP32 = 1 };
  *             allocated until muon_destroy.  W, G and M must not alias.
  *   w_dtype : dtype of W (bf16 or fp32).  g_dtype: dtype of G.  M is always
  *             fp32 and must be zero before the first step (M_0 = 0, Sec. 2.1).
+ *   w_shadow: optional (NULL = none) HOST array of `count` DEVICE pointers to
+ *             bf16 copies of fp32 weights (row stride ld_shadow): training
+ *             set-ups that keep fp32 master weights (Sec. 2.3 counts an fp32
+ *             parameter gather) and compute with a bf16 copy get both written
+ *             by the step.  Only with w_dtype = fp32.
  *   Alignment: every pointer aligned to its element size; ld_w, ld_g, ld_m >=
  *             cols.  The fast vector paths need 16-byte aligned pointers and
  *             ld_* that are multiples of 8; anything else takes a slower
@@ -79,6 +84,8 @@ typedef struct muon_group {
   int64_t ld_w;
   int64_t ld_g;
   int64_t ld_m;
+  void* const* w_shadow;
+  int64_t ld_shadow;
 } muon_group;
 
 /*
@@ -91,7 +98,15 @@ typedef struct muon_group {
  *   eps       : added to the Frobenius norm (the paper has none; 1e-7 keeps a
  *               zero input finite).
  *   rms_scale : the 0.2 of Sec. 2.2.
+ *   scale_mode: how the update is scaled (Sec. 3.1 "Consistent Update RMS"):
+ *               MUON_SCALE_ADJUSTED_LR  rms_scale * sqrt(max(rows, cols)) * O  (the method
+ *                                       the paper adopts, Sec. 2.2; the default, 0),
+ *               MUON_SCALE_FIXED_DIM    rms_scale * sqrt(scale_dim) * O  ("Baseline":
+ *                                       scale_dim = the model's hidden size H),
+ *               MUON_SCALE_UPDATE_NORM  rms_scale * O / RMS(O)  ("Update Norm").
+ *   scale_dim : H for MUON_SCALE_FIXED_DIM, ignored otherwise.
  */
+enum { MUON_SCALE_ADJUSTED_LR = 0, MUON_SCALE_FIXED_DIM = 1, MUON_SCALE_UPDATE_NORM = 2 };
 typedef struct muon_hparams {
   float lr;
   float wd;
@@ -103,6 +118,8 @@ typedef struct muon_hparams {
   float c;
   float eps;
   float rms_scale;
+  int32_t scale_mode;
+  float scale_dim;
 } muon_hparams;
 
 typedef struct muon_ctx muon_ctx;
@@ -166,9 +183,10 @@ int muon_get_norms(muon_ctx* ctx, void* stream, float* out, int n);
 
 /*
  * Per-matrix update RMS of the last step, the value Algorithm 1 returns for
- * logging: sqrt(mean(u^2)) with u = rms_scale * sqrt(max(rows, cols)) * O (the
- * scaled update before the learning rate; it sits near 0.2 by Sec. 2.2's
- * design).  Copies `n` floats (global matrix order) to the HOST array `out`
+ * logging: sqrt(mean(u^2)) with u the scaled update before the learning rate
+ * (rms_scale * sqrt(max(rows, cols)) * O in the default scale mode; it sits
+ * near 0.2 by Sec. 2.2's design, and is rms_scale exactly with
+ * MUON_SCALE_UPDATE_NORM).  Copies `n` floats (global matrix order) to the HOST array `out`
  * after synchronising `stream`.  A matrix whose input was non-finite reports
  * an unspecified value.
  */

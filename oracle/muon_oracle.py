@@ -25,6 +25,9 @@ Passages followed (paper = "Muon is Scalable for LLM Training"):
   * Sec. 2.2 "Weight Decay" (Eq. 3) and "Matching update RMS of AdamW"
     (the unnumbered equation with 0.2 * sqrt(max(A, B))).
   * Algorithm 1, last line: the update RMS returned for logging.
+  * Sec. 3.1 "Consistent Update RMS": the three ways of scaling the update
+    (Baseline 0.2*sqrt(H), Update Norm 0.2/RMS(O), Adjusted LR
+    0.2*sqrt(max(A, B)) -- the last is the method the paper adopts).
 """
 
 from __future__ import annotations
@@ -56,6 +59,10 @@ class Hyper:
     c: float = NS_C
     eps: float = 1e-7
     rms_scale: float = 0.2
+    # Sec. 3.1: "adjusted_lr" (default, the adopted method), "fixed_dim"
+    # (Baseline; scale_dim is the hidden size H) or "update_norm".
+    scale_mode: str = "adjusted_lr"
+    scale_dim: float = 0.0
 
 
 def _f64(x):
@@ -114,25 +121,40 @@ def newton_schulz(X0, steps, a=NS_A, b=NS_B, c=NS_C, trace=None):
     return np.ascontiguousarray(X)
 
 
-def apply_update(W, O, lr, wd, rms_scale=0.2):
-    """W_t = W_{t-1} - lr * (rms_scale * sqrt(max(A, B)) * O + wd * W_{t-1})
-    for a parameter of shape [A, B]  (Sec. 2.2, "Matching update RMS of
-    AdamW"; rms_scale is the paper's 0.2).  The decay term uses W_{t-1} and is
+def update_factor(O, rms_scale=0.2, scale_mode="adjusted_lr", scale_dim=0.0):
+    """The scalar that multiplies O in the weight step (Sec. 3.1, the three
+    numbered variants): rms_scale*sqrt(max(A, B)) ("Adjusted LR", also Sec. 2.2),
+    rms_scale*sqrt(H) ("Baseline") or rms_scale/RMS(O) ("Update Norm"), with
+    RMS(O) = sqrt(mean(O^2)).  A zero O under "Update Norm" gives factor 0."""
+    O = _f64(O)
+    rows, cols = O.shape
+    if scale_mode == "adjusted_lr":
+        return rms_scale * math.sqrt(max(rows, cols))
+    if scale_mode == "fixed_dim":
+        return rms_scale * math.sqrt(scale_dim)
+    if scale_mode == "update_norm":
+        o_rms = math.sqrt(float(np.mean(O * O)))
+        return rms_scale / o_rms if o_rms > 0.0 else 0.0
+    raise ValueError("unknown scale_mode %r" % (scale_mode,))
+
+
+def apply_update(W, O, lr, wd, rms_scale=0.2, scale_mode="adjusted_lr", scale_dim=0.0):
+    """W_t = W_{t-1} - lr * (factor * O + wd * W_{t-1}) with factor =
+    rms_scale * sqrt(max(A, B)) for a parameter of shape [A, B]  (Sec. 2.2,
+    "Matching update RMS of AdamW"; rms_scale is the paper's 0.2) or one of the
+    other two variants of Sec. 3.1.  The decay term uses W_{t-1} and is
     multiplied by the learning rate, as in Eq. 3."""
     W = _f64(W)
     O = _f64(O)
-    rows, cols = W.shape
-    scale = rms_scale * math.sqrt(max(rows, cols))
-    return W - lr * (scale * O + wd * W)
+    return W - lr * (update_factor(O, rms_scale, scale_mode, scale_dim) * O + wd * W)
 
 
-def update_rms(O, rms_scale=0.2):
-    """sqrt(mean(u^2)) of the scaled update u = rms_scale*sqrt(max(A,B))*O
-    (Algorithm 1, returned value; the reading taken is that u carries the
-    scale factor, so the value sits near 0.2 as Sec. 2.2 intends)."""
+def update_rms(O, rms_scale=0.2, scale_mode="adjusted_lr", scale_dim=0.0):
+    """sqrt(mean(u^2)) of the scaled update u = factor * O  (Algorithm 1,
+    returned value; the reading taken is that u carries the scale factor, so
+    the value sits near 0.2 as Sec. 2.2 intends)."""
     O = _f64(O)
-    rows, cols = O.shape
-    u = rms_scale * math.sqrt(max(rows, cols)) * O
+    u = update_factor(O, rms_scale, scale_mode, scale_dim) * O
     return math.sqrt(float(np.mean(u * u)))
 
 
@@ -161,10 +183,10 @@ def muon_step(W, G, M, hp: Hyper, trace=False):
     stages = [] if trace else None
     O = newton_schulz(X0, hp.ns_steps, hp.a, hp.b, hp.c, trace=stages)
     out.update(
-        W=apply_update(W, O, hp.lr, hp.wd, hp.rms_scale),
+        W=apply_update(W, O, hp.lr, hp.wd, hp.rms_scale, hp.scale_mode, hp.scale_dim),
         X0=X0,
         O=O,
-        rms=update_rms(O, hp.rms_scale),
+        rms=update_rms(O, hp.rms_scale, hp.scale_mode, hp.scale_dim),
     )
     if trace:
         out["stages"] = stages

@@ -27,6 +27,7 @@ MUON_ERR_NONFINITE = -7
 MUON_DTYPE_BF16 = 0
 MUON_DTYPE_FP32 = 1
 MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
+MUON_SCALE_ADJUSTED_LR, MUON_SCALE_FIXED_DIM, MUON_SCALE_UPDATE_NORM = 0, 1, 2
 
 EXPORTED = [
     "muon_workspace_bytes", "muon_init", "muon_step", "muon_step_host", "muon_status",
@@ -45,6 +46,7 @@ class muon_group(C.Structure):
         ("w_dtype", C.c_int32), ("g_dtype", C.c_int32), ("reserved", C.c_int32),
         ("w", C.POINTER(C.c_void_p)), ("g", C.POINTER(C.c_void_p)), ("m", C.POINTER(C.c_void_p)),
         ("ld_w", C.c_int64), ("ld_g", C.c_int64), ("ld_m", C.c_int64),
+        ("w_shadow", C.POINTER(C.c_void_p)), ("ld_shadow", C.c_int64),
     ]
 
 
@@ -54,6 +56,7 @@ class muon_hparams(C.Structure):
         ("nesterov", C.c_int32), ("ns_steps", C.c_int32),
         ("a", C.c_float), ("b", C.c_float), ("c", C.c_float),
         ("eps", C.c_float), ("rms_scale", C.c_float),
+        ("scale_mode", C.c_int32), ("scale_dim", C.c_float),
     ]
 
 
@@ -126,10 +129,13 @@ class Hyper:
     c: float = 2.0315
     eps: float = 1e-7
     rms_scale: float = 0.2
+    scale_mode: int = MUON_SCALE_ADJUSTED_LR
+    scale_dim: float = 0.0
 
     def to_c(self) -> muon_hparams:
         return muon_hparams(self.lr, self.wd, self.mu, int(bool(self.nesterov)), int(self.ns_steps),
-                            self.a, self.b, self.c, self.eps, self.rms_scale)
+                            self.a, self.b, self.c, self.eps, self.rms_scale, int(self.scale_mode),
+                            float(self.scale_dim))
 
 
 def _dtype_code(t):
@@ -144,9 +150,14 @@ def _dtype_code(t):
 class _GroupArrays:
     """Keeps the ctypes arrays of one param group alive."""
 
-    def __init__(self, ws, gs, ms):
+    def __init__(self, ws, gs, ms, shadows=None):
         w0, g0, m0 = ws[0], gs[0], ms[0]
         n = len(ws)
+        if shadows is not None:
+            import torch
+            for t in shadows:
+                if t.shape != w0.shape or t.dtype != torch.bfloat16 or t.stride(1) != 1 or t.stride(0) != shadows[0].stride(0):
+                    raise MuonError(MUON_ERR_INVALID_ARG, "shadow copies must be bf16, shaped like W, with one row stride")
         for t in list(ws) + list(gs) + list(ms):
             if t.dim() != 2 or t.shape != w0.shape or t.stride(1) != 1:
                 raise MuonError(MUON_ERR_INVALID_ARG, "matrices of a group must be 2-D, equal-shaped, rows contiguous")
@@ -163,7 +174,13 @@ class _GroupArrays:
             C.cast(self.m, C.POINTER(C.c_void_p)),
             w0.stride(0) if w0.shape[0] > 1 else max(w0.stride(0), w0.shape[1]),
             g0.stride(0) if g0.shape[0] > 1 else max(g0.stride(0), g0.shape[1]),
-            m0.stride(0) if m0.shape[0] > 1 else max(m0.stride(0), m0.shape[1]))
+            m0.stride(0) if m0.shape[0] > 1 else max(m0.stride(0), m0.shape[1]),
+            None, 0)
+        if shadows is not None:
+            s0 = shadows[0]
+            self.s = (C.c_void_p * n)(*[t.data_ptr() for t in shadows])
+            self.desc.w_shadow = C.cast(self.s, C.POINTER(C.c_void_p))
+            self.desc.ld_shadow = s0.stride(0) if s0.shape[0] > 1 else max(s0.stride(0), s0.shape[1])
 
 
 def shape_only_groups(shapes) -> "C.Array":
@@ -213,8 +230,9 @@ def muon_debug_set_chunk_bytes(nbytes: int) -> int:
 class MuonContext:
     """One initialised set of param groups.
 
-    ``groups`` is a list of (weights, grads, momenta) triples; each entry of a
-    triple is a list of equal-shaped 2-D CUDA tensors (bf16 or fp32 weights and
+    ``groups`` is a list of (weights, grads, momenta) triples, or
+    (weights, grads, momenta, shadows) with bf16 copies of fp32 weights; each
+    entry is a list of equal-shaped 2-D CUDA tensors (bf16 or fp32 weights and
     gradients, fp32 momenta).  Tensors must outlive the context.
     """
 
@@ -223,7 +241,7 @@ class MuonContext:
         if not torch.cuda.is_available():
             raise MuonError(MUON_ERR_CUDA, "no CUDA device: this library has no CPU path")
         L = lib()
-        self._arrays: List[_GroupArrays] = [_GroupArrays(ws, gs, ms) for ws, gs, ms in groups]
+        self._arrays: List[_GroupArrays] = [_GroupArrays(*g) for g in groups]
         self._tensors = groups
         n = len(self._arrays)
         self._groups_c = (muon_group * n)(*[a.desc for a in self._arrays])

@@ -30,6 +30,8 @@ struct MatDesc {
   int vec_ok;      // all three of W, G, M allow 16-byte vector access
   int global_index;  // position in the caller's group list (groups in order)
   int pad_;
+  void* w_shadow;    // optional bf16 copy of fp32 weights, written with every update
+  long long ld_ws;
 };
 
 // Per-matrix scalars written by the norm finalisation kernel.

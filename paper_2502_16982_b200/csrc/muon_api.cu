@@ -25,15 +25,15 @@ cudaError_t launch_momentum_cast(const StreamParams& P, bool grad_fp32, cudaStre
 cudaError_t launch_norm_finalise(const float* partials, int tiles_per_matrix, int count, float eps,
                                  const MatDesc* descs, MatScal* scal, float* norms, DevStatus* status,
                                  cudaStream_t stream);
-cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
-                                 long long x_stride, int ldx, int count, long long elems,
-                                 float upd_scale, float decay, bool use_inv_norm, bool w_fp32,
-                                 cudaStream_t stream);
+cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, const float* factors,
+                                 const __nv_bfloat16* x, long long x_stride, int ldx, int count, int m,
+                                 int n, float neg_lr, float decay, bool w_fp32, cudaStream_t stream);
 cudaError_t launch_rms_finalise(const float* partials, int per_matrix, int count, float factor,
                                 const MatDesc* descs, float* rms, cudaStream_t stream);
 cudaError_t launch_rms_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
                               long long x_stride, int ldx, int m, int n, int count, float factor,
-                              bool use_inv_norm, float* rms, cudaStream_t stream);
+                              bool use_inv_norm, float rms_target, bool normalise, float* rms,
+                              float* factors, cudaStream_t stream);
 cudaError_t stream_tma_configure();
 cudaError_t launch_momentum_tma(const StreamTmaParams& P, bool grad_fp32, int num_sms, cudaStream_t stream);
 cudaError_t gemm_configure();
@@ -79,7 +79,7 @@ struct Bucket {
   bool fused_update;          // every W is bf16 and TMA-addressable: update W in the last epilogue
   bool stream_tma;            // every G and M is TMA-addressable: TMA-pipelined momentum kernel
   // workspace offsets (bytes) of the chunk buffers
-  size_t off_x[2], off_a, off_b, off_partials, off_scal, off_rms_partials;
+  size_t off_x[2], off_a, off_b, off_partials, off_scal, off_rms_partials, off_factors;
   // workspace offsets of the persistent per-bucket tables
   size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_comb_tiles;
   std::vector<PairTile> sym_tiles, comb_tiles;  // tile tables of one matrix
@@ -187,6 +187,14 @@ int validate_groups(const muon_group* groups, int n_groups, bool need_ptrs) {
         return fail(MUON_ERR_ALIGNMENT, "group %d matrix %d: pointer not aligned to its element size", g, i);
       if (G.w[i] == G.g[i] || G.w[i] == (void*)G.m[i] || G.g[i] == (const void*)G.m[i])
         return fail(MUON_ERR_INVALID_ARG, "group %d matrix %d: W, G and M must not alias", g, i);
+      if (G.w_shadow) {
+        if (G.w_dtype != MUON_DTYPE_FP32)
+          return fail(MUON_ERR_INVALID_ARG, "group %d: a bf16 shadow copy needs fp32 weights", g);
+        if (!G.w_shadow[i] || (reinterpret_cast<uintptr_t>(G.w_shadow[i]) & 1) || G.ld_shadow < G.cols)
+          return fail(MUON_ERR_INVALID_ARG, "group %d matrix %d: bad shadow pointer or leading dimension", g, i);
+        if (G.w_shadow[i] == G.w[i] || G.w_shadow[i] == G.g[i] || G.w_shadow[i] == (void*)G.m[i])
+          return fail(MUON_ERR_INVALID_ARG, "group %d matrix %d: the shadow copy must not alias W, G or M", g, i);
+      }
     }
   }
   return MUON_OK;
@@ -266,6 +274,7 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
       const size_t comb_tiles = static_cast<size_t>(np) * ceil_div(ncb, 2);
       B.off_rms_partials = take(chunk * comb_tiles * 8 * sizeof(float));
     }
+    B.off_factors = take(chunk * sizeof(float));
     chunk_region = std::max(chunk_region, off);
   }
   size_t off = align_up(chunk_region, 1024);
@@ -338,6 +347,7 @@ struct muon_ctx {
   std::vector<std::vector<void*>> w_ptrs;    // per group
   std::vector<std::vector<const void*>> g_ptrs;
   std::vector<std::vector<float*>> m_ptrs;
+  std::vector<std::vector<void*>> s_ptrs;    // optional bf16 shadow copies
   std::vector<Bucket> buckets;
   PlanSizes sizes;
   int total_mats;
@@ -452,7 +462,12 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   ctx->w_ptrs.resize(n_groups);
   ctx->g_ptrs.resize(n_groups);
   ctx->m_ptrs.resize(n_groups);
+  ctx->s_ptrs.resize(n_groups);
   for (int g = 0; g < n_groups; ++g) {
+    if (groups[g].w_shadow) {
+      ctx->s_ptrs[g].assign(groups[g].w_shadow, groups[g].w_shadow + groups[g].count);
+      ctx->groups[g].w_shadow = ctx->s_ptrs[g].data();
+    }
     ctx->w_ptrs[g].assign(groups[g].w, groups[g].w + groups[g].count);
     ctx->g_ptrs[g].assign(groups[g].g, groups[g].g + groups[g].count);
     ctx->m_ptrs[g].assign(groups[g].m, groups[g].m + groups[g].count);
@@ -485,6 +500,8 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
       d.cols = G.cols;
       d.transposed = G.rows > G.cols ? 1 : 0;
       d.global_index = r.global;
+      d.w_shadow = G.w_shadow ? G.w_shadow[r.index] : nullptr;
+      d.ld_ws = G.ld_shadow;
       const bool ptr16 = ((reinterpret_cast<uintptr_t>(d.w) | reinterpret_cast<uintptr_t>(d.g) |
                            reinterpret_cast<uintptr_t>(d.m)) & 15) == 0;
       d.vec_ok = (ptr16 && G.ld_w % 8 == 0 && G.ld_g % 8 == 0 && G.ld_m % 8 == 0) ? 1 : 0;
@@ -556,6 +573,10 @@ static int check_hparams(const muon_hparams* hp) {
   if (!hp) return fail(MUON_ERR_INVALID_ARG, "hparams is null");
   if (hp->ns_steps < 0 || hp->ns_steps > 64) return fail(MUON_ERR_INVALID_ARG, "ns_steps must be in [0, 64]");
   if (!(hp->eps >= 0.f)) return fail(MUON_ERR_INVALID_ARG, "eps must be >= 0");
+  if (hp->scale_mode < MUON_SCALE_ADJUSTED_LR || hp->scale_mode > MUON_SCALE_UPDATE_NORM)
+    return fail(MUON_ERR_INVALID_ARG, "unknown scale_mode");
+  if (hp->scale_mode == MUON_SCALE_FIXED_DIM && !(hp->scale_dim > 0.f))
+    return fail(MUON_ERR_INVALID_ARG, "scale_dim must be positive with MUON_SCALE_FIXED_DIM");
   if (!std::isfinite(hp->lr) || !std::isfinite(hp->wd) || !std::isfinite(hp->mu) || !std::isfinite(hp->a) ||
       !std::isfinite(hp->b) || !std::isfinite(hp->c) || !std::isfinite(hp->rms_scale))
     return fail(MUON_ERR_INVALID_ARG, "hyper-parameters must be finite");
@@ -575,7 +596,12 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
   for (size_t b = 0; b < ctx->buckets.size(); ++b) {
     Bucket& B = ctx->buckets[b];
     const int total = static_cast<int>(B.mats.size());
-    const float upd_scale = -hp->lr * hp->rms_scale * std::sqrt(static_cast<float>(B.n));
+    // factor of O in the update (Sec. 2.2 / Sec. 3.1): 0.2*sqrt(max(rows, cols)), or 0.2*sqrt(H)
+    const float factor = hp->rms_scale * std::sqrt(hp->scale_mode == MUON_SCALE_FIXED_DIM
+                                                       ? hp->scale_dim : static_cast<float>(B.n));
+    const bool normalise = hp->scale_mode == MUON_SCALE_UPDATE_NORM;
+    const bool fused_update = B.fused_update && !normalise;
+    const float upd_scale = -hp->lr * factor;
     const float decay = 1.0f - hp->lr * hp->wd;
     for (int first = 0; first < total; first += B.chunk) {
       const int count = std::min(B.chunk, total - first);
@@ -672,7 +698,7 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
 
         // X' = a*X + B X (first iteration: times s); the last iteration updates W
         // in its epilogue when every W of the bucket is TMA-addressable bf16
-        const bool fuse = last_it && B.fused_update;
+        const bool fuse = last_it && fused_update;
         P.map_a = B.b_op;
         P.map_a64 = B.b_b64;
         P.map_b = B.x_b64[cur];
@@ -693,33 +719,36 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
         ++launches;
         cur = nxt;
       }
-      if (hp->ns_steps == 0 || !B.fused_update) {
-        // W <- decay*W + upd_scale*O from the stored O: O = s*bf16(U) when there
-        // was no iteration, else the last X (fp32 weights, or weights a TMA
-        // descriptor cannot address)
-        LaunchTimer lt(ctx, stream, MUON_KERNEL_UPDATE);
-        ce = launch_update_from_x(descs, scal, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + B.off_x[cur]),
-                                  static_cast<long long>(B.x_stride), B.ldx, count,
-                                  static_cast<long long>(B.m) * B.n, upd_scale, decay, hp->ns_steps == 0,
-                                  B.w_dtype == MUON_DTYPE_FP32, stream);
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "update kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
-      }
-      // update RMS for logging (Algorithm 1, returned value): RMS of rms_scale*sqrt(max(rows,cols))*O
       {
+        // Update RMS for logging (Algorithm 1, returned value) and, when the
+        // weights were not updated in the last epilogue (no iteration, fp32 or
+        // TMA-unaddressable weights, normalised update), the separate update
+        // W <- decay*W - lr*f*O from the stored O.
         float* rms = reinterpret_cast<float*>(ctx->ws + ctx->sizes.off_rms);
-        const float factor = hp->rms_scale * std::sqrt(static_cast<float>(B.n));
-        LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
-        if (hp->ns_steps > 0 && B.fused_update) {
+        if (hp->ns_steps > 0 && fused_update) {
+          LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
           ce = launch_rms_finalise(reinterpret_cast<const float*>(ctx->ws + B.off_rms_partials),
                                    static_cast<int>(B.comb_tiles.size()) * 8, count, factor, descs, rms, stream);
+          if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
+          ++launches;
         } else {
-          ce = launch_rms_from_x(descs, scal, reinterpret_cast<const __nv_bfloat16*>(ctx->ws + B.off_x[cur]),
-                                 static_cast<long long>(B.x_stride), B.ldx, B.m, B.n, count, factor,
-                                 hp->ns_steps == 0, rms, stream);
+          float* factors = reinterpret_cast<float*>(ctx->ws + B.off_factors);
+          const __nv_bfloat16* xo = reinterpret_cast<const __nv_bfloat16*>(ctx->ws + B.off_x[cur]);
+          {
+            LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
+            ce = launch_rms_from_x(descs, scal, xo, static_cast<long long>(B.x_stride), B.ldx, B.m, B.n, count,
+                                   factor, hp->ns_steps == 0, hp->rms_scale, normalise, rms, factors, stream);
+          }
+          if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
+          ++launches;
+          {
+            LaunchTimer lt(ctx, stream, MUON_KERNEL_UPDATE);
+            ce = launch_update_from_x(descs, scal, factors, xo, static_cast<long long>(B.x_stride), B.ldx, count,
+                                      B.m, B.n, -hp->lr, decay, B.w_dtype == MUON_DTYPE_FP32, stream);
+          }
+          if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "update kernel launch: %s", cudaGetErrorString(ce));
+          ++launches;
         }
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
       }
       ctx->x0_buf[b] = 0;
       ctx->xlast_buf[b] = cur;

@@ -227,31 +227,51 @@ __global__ void norm_finalise_kernel(const float* __restrict__ partials, int til
   }
 }
 
-// W <- decay*W + upd_scale*O with O = x (short side first), times s when the
-// stored x is the un-normalised bf16(U) (ns_steps == 0: O = X0 = s * bf16(U)).
+// W <- decay*W + f*O with O = x (short side first, transposed back when rows >
+// cols), f = -lr * (per-matrix update factor).  One CTA per 64 x 64 tile of W;
+// the O tile passes through shared memory so that both the read of x and the
+// accesses to W are coalesced in either orientation.  Optionally also writes a
+// bf16 copy of the new fp32 weights (w_shadow).
 template <bool kWFp32>
-__global__ void update_from_x_kernel(const MatDesc* __restrict__ descs,
-                                     const MatScal* __restrict__ scal,
-                                     const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx,
-                                     float upd_scale, float decay, int use_inv_norm) {
+__global__ void __launch_bounds__(256)
+update_from_x_kernel(const MatDesc* __restrict__ descs, const MatScal* __restrict__ scal,
+                     const float* __restrict__ factors, const __nv_bfloat16* __restrict__ x,
+                     long long x_stride, int ldx, float neg_lr, float decay) {
+  __shared__ float tile[64][65];
   const int mat = blockIdx.y;
   const MatDesc d = descs[mat];
-  const MatScal sc = scal[mat];
-  if (sc.nonfinite) return;
-  const float s = use_inv_norm ? sc.inv_norm : 1.0f;
-  const long long total = static_cast<long long>(d.rows) * d.cols;
+  if (scal[mat].nonfinite) return;
+  const int tiles_c = (d.cols + 63) / 64;
+  const int tr = blockIdx.x / tiles_c, tc = blockIdx.x - tr * tiles_c;
+  if (tr * 64 >= d.rows) return;
+  const int r0 = tr * 64, c0 = tc * 64;
+  const float f = neg_lr * factors[mat];
   const __nv_bfloat16* xm = x + mat * x_stride;
-  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
-       i += static_cast<long long>(gridDim.x) * blockDim.x) {
-    const int r = static_cast<int>(i / d.cols), c = static_cast<int>(i - static_cast<long long>(r) * d.cols);
-    const float o = s * __bfloat162float(d.transposed ? xm[static_cast<long long>(c) * ldx + r]
-                                                                : xm[static_cast<long long>(r) * ldx + c]);
+  // x tile: rows (short side) xr0.., columns (long side) xc0..
+  const int xr0 = d.transposed ? c0 : r0, xc0 = d.transposed ? r0 : c0;
+  const int x_rows = d.transposed ? d.cols : d.rows, x_cols = d.transposed ? d.rows : d.cols;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+#pragma unroll 4
+  for (int i = ty; i < 64; i += 4) {
+    const int xr = xr0 + i, xc = xc0 + tx;
+    tile[i][tx] = (xr < x_rows && xc < x_cols) ? __bfloat162float(xm[static_cast<long long>(xr) * ldx + xc]) : 0.f;
+  }
+  __syncthreads();
+#pragma unroll 4
+  for (int i = ty; i < 64; i += 4) {
+    const int r = r0 + i, c = c0 + tx;
+    if (r >= d.rows || c >= d.cols) continue;
+    const float o = d.transposed ? tile[tx][i] : tile[i][tx];
+    const long long off = static_cast<long long>(r) * d.ld_w + c;
     if (kWFp32) {
-      float* w = reinterpret_cast<float*>(d.w) + static_cast<long long>(r) * d.ld_w + c;
-      *w = fmaf(decay, *w, upd_scale * o);
+      float* w = reinterpret_cast<float*>(d.w) + off;
+      const float nw = fmaf(decay, *w, f * o);
+      *w = nw;
+      if (d.w_shadow != nullptr)
+        reinterpret_cast<__nv_bfloat16*>(d.w_shadow)[static_cast<long long>(r) * d.ld_ws + c] = __float2bfloat16_rn(nw);
     } else {
-      __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(d.w) + static_cast<long long>(r) * d.ld_w + c;
-      *w = __float2bfloat16_rn(fmaf(decay, __bfloat162float(*w), upd_scale * o));
+      __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(d.w) + off;
+      *w = __float2bfloat16_rn(fmaf(decay, __bfloat162float(*w), f * o));
     }
   }
 }
@@ -261,6 +281,7 @@ __global__ void update_from_x_kernel(const MatDesc* __restrict__ descs,
 __global__ void rms_finalise_kernel(const float* __restrict__ partials, int per_matrix, int count,
                                     float factor, const MatDesc* __restrict__ descs,
                                     float* __restrict__ rms) {
+  // (fused path: the update factor is fixed by the shape, nothing else to derive)
   const int mat = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (mat >= count) return;
   const int lane = threadIdx.x & 31;
@@ -276,11 +297,15 @@ __global__ void rms_finalise_kernel(const float* __restrict__ partials, int per_
 }
 
 // Update RMS from a stored O (x, short side first, m x n): one CTA per matrix,
-// thread-strided sequential sums and a fixed reduction tree.
+// thread-strided sequential sums and a fixed reduction tree.  Also leaves the
+// per-matrix factor the separate update kernel multiplies O by:
+// `factor` * s, or rms_target / RMS(O) * s when the update is normalised
+// (Sec. 3.1 "Update Norm"); s = 1/(||U||_F + eps) when x is the un-normalised bf16(U).
 __global__ void __launch_bounds__(256)
 rms_from_x_kernel(const MatDesc* __restrict__ descs, const MatScal* __restrict__ scal,
                   const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx, int m, int n,
-                  float factor, int use_inv_norm, float* __restrict__ rms) {
+                  float factor, int use_inv_norm, float rms_target, int normalise,
+                  float* __restrict__ rms, float* __restrict__ factors) {
   __shared__ float warp_sums[8];
   const int mat = blockIdx.x;
   const __nv_bfloat16* xm = x + mat * x_stride;
@@ -300,7 +325,14 @@ rms_from_x_kernel(const MatDesc* __restrict__ descs, const MatScal* __restrict__
     for (int w = 0; w < 8; ++w) t += warp_sums[w];
     const MatScal sc = scal[mat];
     const float sn = use_inv_norm ? sc.inv_norm : 1.0f;
-    rms[descs[mat].global_index] = fabsf(factor * sn) * sqrtf(t / (static_cast<float>(m) * static_cast<float>(n)));
+    const float o_rms = fabsf(sn) * sqrtf(t / (static_cast<float>(m) * static_cast<float>(n)));
+    if (normalise) {
+      rms[descs[mat].global_index] = o_rms > 0.f ? rms_target : 0.f;
+      factors[mat] = o_rms > 0.f ? sn * rms_target / o_rms : 0.f;
+    } else {
+      rms[descs[mat].global_index] = fabsf(factor) * o_rms;
+      factors[mat] = factor * sn;
+    }
   }
 }
 
@@ -317,9 +349,11 @@ cudaError_t launch_rms_finalise(const float* partials, int per_matrix, int count
 
 cudaError_t launch_rms_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
                               long long x_stride, int ldx, int m, int n, int count, float factor,
-                              bool use_inv_norm, float* rms, cudaStream_t stream) {
+                              bool use_inv_norm, float rms_target, bool normalise, float* rms,
+                              float* factors, cudaStream_t stream) {
   if (count == 0) return cudaSuccess;
-  rms_from_x_kernel<<<count, 256, 0, stream>>>(descs, scal, x, x_stride, ldx, m, n, factor, use_inv_norm ? 1 : 0, rms);
+  rms_from_x_kernel<<<count, 256, 0, stream>>>(descs, scal, x, x_stride, ldx, m, n, factor, use_inv_norm ? 1 : 0,
+                                               rms_target, normalise ? 1 : 0, rms, factors);
   return cudaGetLastError();
 }
 
@@ -341,22 +375,16 @@ cudaError_t launch_norm_finalise(const float* partials, int tiles_per_matrix, in
   return cudaGetLastError();
 }
 
-cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
-                                 long long x_stride, int ldx, int count, long long elems,
-                                 float upd_scale, float decay, bool use_inv_norm, bool w_fp32,
-                                 cudaStream_t stream) {
+cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, const float* factors,
+                                 const __nv_bfloat16* x, long long x_stride, int ldx, int count, int m,
+                                 int n, float neg_lr, float decay, bool w_fp32, cudaStream_t stream) {
   if (count == 0) return cudaSuccess;
-  const int threads = 256;
-  long long bx = (elems + threads - 1) / threads;
-  if (bx > 1024) bx = 1024;
-  if (bx < 1) bx = 1;
-  dim3 grid(static_cast<unsigned>(bx), static_cast<unsigned>(count));
+  // both orientations of a bucket have the same number of 64 x 64 tiles
+  dim3 grid(static_cast<unsigned>(((m + 63) / 64) * ((n + 63) / 64)), static_cast<unsigned>(count));
   if (w_fp32)
-    update_from_x_kernel<true><<<grid, threads, 0, stream>>>(descs, scal, x, x_stride, ldx, upd_scale, decay,
-                                                             use_inv_norm ? 1 : 0);
+    update_from_x_kernel<true><<<grid, 256, 0, stream>>>(descs, scal, factors, x, x_stride, ldx, neg_lr, decay);
   else
-    update_from_x_kernel<false><<<grid, threads, 0, stream>>>(descs, scal, x, x_stride, ldx, upd_scale, decay,
-                                                              use_inv_norm ? 1 : 0);
+    update_from_x_kernel<false><<<grid, 256, 0, stream>>>(descs, scal, factors, x, x_stride, ldx, neg_lr, decay);
   return cudaGetLastError();
 }
 

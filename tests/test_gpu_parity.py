@@ -46,9 +46,13 @@ def f64(t):
     return t.detach().cpu().to(torch.float64).numpy()
 
 
+SCALE_MODES = {0: "adjusted_lr", 1: "fixed_dim", 2: "update_norm"}
+
+
 def to_orc(hp):
     return orc.Hyper(lr=hp.lr, wd=hp.wd, mu=hp.mu, nesterov=hp.nesterov, ns_steps=hp.ns_steps,
-                     a=hp.a, b=hp.b, c=hp.c, eps=hp.eps, rms_scale=hp.rms_scale)
+                     a=hp.a, b=hp.b, c=hp.c, eps=hp.eps, rms_scale=hp.rms_scale,
+                     scale_mode=SCALE_MODES[hp.scale_mode], scale_dim=hp.scale_dim)
 
 
 def bf16_ulp_ok_fraction(got_bf16, expect_f64, slack=0.0):
@@ -301,6 +305,49 @@ def test_chunked_bucket_matches_the_oracle():
         check_step(case, hp)
     finally:
         case.close()
+
+
+@pytest.mark.parametrize("wdt", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("mode,dim", [(1, 1024.0), (2, 0.0)])
+def test_update_scale_variants(mode, dim, wdt):
+    """Sec. 3.1: "Baseline" 0.2*sqrt(H) and "Update Norm" 0.2/RMS(O), both
+    orientations, two steps."""
+    specs = [wl.GroupSpec(328, 200, 2, wdt, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(200, 328, 2, wdt, torch.bfloat16, 0.02, 1e-3)]
+    case = Case(specs, seed=41)
+    try:
+        hp = default_hp(lr=1e-2, wd=0.1, scale_mode=mode, scale_dim=dim)
+        check_step(case, hp)
+        check_step(case, hp)
+        if mode == 2:
+            assert all(abs(r - 0.2) < 1e-6 for r in case.ctx.muon_get_update_rms())
+    finally:
+        case.close()
+
+
+def test_fp32_master_weights_with_bf16_shadow():
+    """fp32 master weights plus a bf16 copy written by the step (Sec. 2.3's
+    distributed variant keeps fp32 parameters)."""
+    b = _binding()
+    sp = wl.GroupSpec(264, 392, 2, torch.float32, torch.bfloat16, 0.02, 1e-3)
+    W, G, M = wl.make_group(sp, 51, "cpu")
+    Wd, Gd, Md = W.cuda(), G.cuda(), M.cuda()
+    shadow = torch.zeros((2, 264, 392), dtype=torch.bfloat16, device="cuda")
+    ctx = b.MuonContext([(wl.views(Wd), wl.views(Gd), wl.views(Md), wl.views(shadow))])
+    try:
+        hp = default_hp(lr=1e-2, wd=0.1)
+        ctx.muon_step(hp)
+        assert ctx.muon_status()[0] == 0
+        for i in range(2):
+            ref = orc.muon_step(f64(W[i]), f64(G[i]), f64(M[i]), to_orc(hp))
+            assert rel(f64(Wd[i]) - f64(W[i]), ref["W"] - f64(W[i])) <= TOL_NS
+            # the shadow is the new fp32 weight rounded once to bf16
+            assert torch.equal(shadow[i], Wd[i].to(torch.bfloat16))
+    finally:
+        ctx.muon_destroy()
+    with pytest.raises(b.MuonError):  # a shadow needs fp32 weights
+        Wb = Wd.to(torch.bfloat16)
+        b.MuonContext([(wl.views(Wb), wl.views(Gd), wl.views(Md), wl.views(shadow))])
 
 
 def test_bitwise_reproducible():

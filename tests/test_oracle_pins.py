@@ -325,3 +325,45 @@ def test_pins_are_sensitive_to_planted_mistakes(monkeypatch):
     assert np.max(np.abs(o1["O"] - o2["O"])) > 1e-3
     o3 = orc.muon_step(W, G, M, orc.Hyper(wd=0.0))
     assert np.max(np.abs(o1["W"] - o3["W"])) > 1e-4
+
+
+# ---------------------------------------------------------------------------
+# Sec. 3.1: the three ways of scaling the update
+# ---------------------------------------------------------------------------
+def test_scale_variants_against_hand_formulas():
+    """With ns_steps = 0 and eps = 0 the orthogonalised update is O = U/||U||_F,
+    so every variant of Sec. 3.1 is closed-form element-wise arithmetic:
+      Adjusted LR:  W - lr*(0.2*sqrt(max(A,B)) * U/||U|| + wd*W)
+      Baseline:     W - lr*(0.2*sqrt(H)        * U/||U|| + wd*W)
+      Update Norm:  RMS(O) = ||O||_F/sqrt(A*B) = 1/sqrt(A*B), hence
+                    W - lr*(0.2*sqrt(A*B)      * U/||U|| + wd*W)."""
+    rng = np.random.default_rng(5)
+    rows, cols = 6, 10
+    W = rng.standard_normal((rows, cols))
+    G = rng.standard_normal((rows, cols))
+    M = rng.standard_normal((rows, cols))
+    mu, lr, wd = 0.9, 0.03, 0.2
+    Mn = mu * M + G
+    U = mu * Mn + G
+    unit = U / np.sqrt((U ** 2).sum())
+    for mode, dim, fac in (("adjusted_lr", 0.0, 0.2 * np.sqrt(10.0)),
+                           ("fixed_dim", 49.0, 0.2 * 7.0),
+                           ("update_norm", 0.0, 0.2 * np.sqrt(60.0))):
+        hp = orc.Hyper(lr=lr, wd=wd, mu=mu, nesterov=True, ns_steps=0, eps=0.0, scale_mode=mode, scale_dim=dim)
+        out = orc.muon_step(W, G, M, hp)
+        expect = W - lr * (fac * unit + wd * W)
+        assert np.allclose(out["W"], expect, rtol=1e-13, atol=1e-15), mode
+        assert abs(out["rms"] - fac / np.sqrt(60.0)) <= 1e-13, mode
+
+
+def test_update_norm_has_rms_exactly_point_two_after_the_iteration():
+    rng = np.random.default_rng(6)
+    W = rng.standard_normal((12, 7))
+    G = rng.standard_normal((12, 7))
+    hp = orc.Hyper(lr=0.01, wd=0.0, scale_mode="update_norm")
+    out = orc.muon_step(W, G, np.zeros_like(G), hp)
+    u = (W - out["W"]) / hp.lr
+    assert abs(np.sqrt(np.mean(u ** 2)) - 0.2) <= 1e-12
+    assert abs(out["rms"] - 0.2) <= 1e-12
+    # the direction is still O
+    assert np.allclose(u / np.linalg.norm(u), out["O"] / np.linalg.norm(out["O"]), atol=1e-12)
