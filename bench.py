@@ -239,6 +239,7 @@ def main():
     ap.add_argument("--ns-steps", type=int, default=5, help="Newton-Schulz iterations (the paper uses 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-adamw", action="store_true", help="skip the AdamW (non-Muon parameters) leg")
     ap.add_argument("--max-count", type=int, default=None,
                     help="cap the matrices per group (small cases for profiler captures)")
     ap.add_argument("--ref-budget", type=float, default=12.0)
@@ -420,6 +421,32 @@ def main():
             one.muon_destroy()
         ctx = binding.MuonContext(groups)
 
+    # ---- AdamW for the parameters Muon does not handle: embedding-sized tensors -------
+    adamw = None
+    if not args.no_adamw and world == 1:
+        torch.cuda.empty_cache()
+        shape = (163840, 2048)  # Moonlight's embedding / LM head
+        ps = [torch.zeros(shape, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        gs = [torch.full(shape, 1e-3, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        ms_ = [torch.zeros(shape, dtype=torch.float32, device=dev) for _ in range(2)]
+        vs = [torch.zeros(shape, dtype=torch.float32, device=dev) for _ in range(2)]
+        for t in range(1, 4):
+            binding.muon_adamw_step(ps, gs, ms_, vs, t, lr=4.2e-4, wd=0.1)
+        torch.cuda.synchronize(dev)
+        e0.record(stream)
+        reps = 5
+        for t in range(4, 4 + reps):
+            binding.muon_adamw_step(ps, gs, ms_, vs, t, lr=4.2e-4, wd=0.1)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        a_ms = e0.elapsed_time(e1) / reps
+        a_bytes = 2 * shape[0] * shape[1] * 22.0
+        adamw = {"kernel": "adamw_kernel", "bound": "hbm", "workload": "2 x 163840x2048 bf16 (embedding, LM head)",
+                 "ms_per_launch": a_ms, "achieved": a_bytes / (a_ms * 1e-3) / 1e9, "peak": float(peaks["hbm_gbs"]),
+                 "unit": "GB/s", "frac": a_bytes / (a_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
+                 "bytes_per_element": 22.0}
+        del ps, gs, ms_, vs
+
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:
         fl, secs, desc, threads = oracle_sample_time(specs, hpd, budget_s=args.ref_budget, max_mats=args.ref_mats)
@@ -442,6 +469,8 @@ def main():
     }
     if shapes is not None:
         line["shapes"] = shapes
+    if adamw is not None:
+        line["roofline_adamw"] = adamw
     print(json.dumps(line))
     ctx.muon_destroy()
     if dist is not None:

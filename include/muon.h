@@ -255,6 +255,45 @@ size_t muon_debug_set_chunk_bytes(size_t bytes);
 int muon_debug_tmem_bases(muon_ctx* ctx, unsigned* out_host, int n);
 
 /*
+ * AdamW step for the parameters Muon does not handle: RMSNorm gains, the LM
+ * head and embeddings (Sec. 2.2 "Matching update RMS of AdamW": they share lr
+ * and wd with the Muon-updated matrices; the appendix notes that weight decay
+ * on the RMSNorm gains matters).  Adam with bias correction and decoupled
+ * weight decay, one fused streaming kernel over all tensors:
+ *
+ *   m <- beta1 m + (1-beta1) g;   v <- beta2 v + (1-beta2) g^2
+ *   p <- p - lr * ( (m/(1-beta1^step)) / (sqrt(v/(1-beta2^step)) + eps) + wd p )
+ *
+ * `tensors` is a HOST array of descriptors with DEVICE pointers: p (bf16 or
+ * fp32) and fp32 m, v are updated in place, g (bf16 or fp32) is read; numel
+ * elements each, any shape, contiguous.  `step` counts from 1.  Asynchronous on
+ * `stream`; needs no context, no workspace and allocates nothing.  16-byte
+ * aligned tensors take the vector path; others a scalar path with the same
+ * results.
+ */
+typedef struct muon_adamw_tensor {
+  void* p;
+  const void* g;
+  float* m;
+  float* v;
+  int64_t numel;
+  int32_t p_dtype;
+  int32_t g_dtype;
+} muon_adamw_tensor;
+
+typedef struct muon_adamw_hparams {
+  float lr;
+  float wd;
+  float beta1;
+  float beta2;
+  float eps;
+  int32_t step;
+} muon_adamw_hparams;
+
+int muon_adamw_step(const muon_adamw_tensor* tensors, int n_tensors, const muon_adamw_hparams* hp,
+                    int device, void* stream);
+
+/*
  * Momentum update and Frobenius norm of ONE matrix with no workspace and no
  * allocation of any kind (the paper has no counterpart; this is a library
  * convenience, not a step of its method):

@@ -34,7 +34,7 @@ EXPORTED = [
     "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
-    "muon_momentum_norm_static",
+    "muon_momentum_norm_static", "muon_adamw_step",
 ]
 MUON_STATIC_MAX_TILES = 65536
 KERNEL_KINDS = ["momentum", "norm", "gram", "poly", "comb", "update"]
@@ -58,6 +58,16 @@ class muon_hparams(C.Structure):
         ("eps", C.c_float), ("rms_scale", C.c_float),
         ("scale_mode", C.c_int32), ("scale_dim", C.c_float),
     ]
+
+
+class muon_adamw_tensor(C.Structure):
+    _fields_ = [("p", C.c_void_p), ("g", C.c_void_p), ("m", C.c_void_p), ("v", C.c_void_p),
+                ("numel", C.c_int64), ("p_dtype", C.c_int32), ("g_dtype", C.c_int32)]
+
+
+class muon_adamw_hparams(C.Structure):
+    _fields_ = [("lr", C.c_float), ("wd", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
+                ("eps", C.c_float), ("step", C.c_int32)]
 
 
 class MuonError(RuntimeError):
@@ -98,6 +108,8 @@ def lib():
     L.muon_momentum_norm_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64,
                                             C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
     L.muon_debug_set_chunk_bytes.argtypes = [C.c_size_t]
+    L.muon_adamw_step.argtypes = [C.POINTER(muon_adamw_tensor), C.c_int, C.POINTER(muon_adamw_hparams), C.c_int,
+                                  C.c_void_p]
     for name in EXPORTED:
         if name == "muon_debug_set_chunk_bytes":
             getattr(L, name).restype = C.c_size_t
@@ -219,6 +231,27 @@ def muon_momentum_norm_static(g, m, mu: float, nesterov: bool, norm_out, stream=
     _check(lib().muon_momentum_norm_static(
         C.c_void_p(g.data_ptr()), C.c_void_p(m.data_ptr()), rows, cols, ld_g, ld_m, _dtype_code(g),
         float(mu), int(bool(nesterov)), C.c_void_p(norm_out.data_ptr()), dev, C.c_void_p(s.cuda_stream)))
+
+
+def muon_adamw_step(params, grads, exp_avgs, exp_avg_sqs, step: int, lr: float, wd: float,
+                    beta1: float = 0.9, beta2: float = 0.95, eps: float = 1e-8, stream=None):
+    """AdamW step over lists of contiguous CUDA tensors (p bf16/fp32, g bf16/fp32,
+    m and v fp32), in place; argument marshalling only."""
+    import torch
+    n = len(params)
+    arr = (muon_adamw_tensor * n)()
+    for i, (p, g, m, v) in enumerate(zip(params, grads, exp_avgs, exp_avg_sqs)):
+        for t in (p, g, m, v):
+            if not t.is_contiguous() or t.numel() != p.numel():
+                raise MuonError(MUON_ERR_INVALID_ARG, "AdamW tensors must be contiguous and equally sized")
+        if m.dtype != torch.float32 or v.dtype != torch.float32:
+            raise MuonError(MUON_ERR_INVALID_ARG, "AdamW moments must be fp32")
+        arr[i] = muon_adamw_tensor(p.data_ptr(), g.data_ptr(), m.data_ptr(), v.data_ptr(), p.numel(),
+                                   _dtype_code(p), _dtype_code(g))
+    dev = params[0].device.index
+    s = torch.cuda.current_stream(dev) if stream is None else stream
+    hp = muon_adamw_hparams(lr, wd, beta1, beta2, eps, int(step))
+    _check(lib().muon_adamw_step(arr, n, C.byref(hp), dev, C.c_void_p(s.cuda_stream)))
 
 
 def muon_debug_set_chunk_bytes(nbytes: int) -> int:

@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmuon_b200.so")
-SOURCES = ["muon_api.cu", "stream_kernels.cu", "stream_tma.cu", "ns_gemm.cu", "no_alloc.cu"]
+SOURCES = ["muon_api.cu", "stream_kernels.cu", "stream_tma.cu", "ns_gemm.cu", "no_alloc.cu", "adamw.cu"]
 HEADERS = ["internal.h", "ptx.cuh", os.path.join("..", "..", "include", "muon.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
