@@ -134,6 +134,20 @@ typedef struct muon_ctx muon_ctx;
 int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_bytes);
 
 /*
+ * Owner-computes partition for data-parallel training (Sec. 2.3, Distributed
+ * Muon: Newton-Schulz needs the whole gradient matrix, so each matrix is given
+ * to ONE rank, which keeps its momentum, runs the step on it and shares the
+ * updated weights afterwards; whole matrices are the unit, so nothing has to
+ * be gathered inside the iteration).  Pure host computation on shapes and
+ * counts: owner_out[i] (HOST, one int per matrix, groups in order) is the rank
+ * in [0, world) that owns matrix i, balanced by the Newton-Schulz work
+ * 3 m^2 n + m^3 with a deterministic longest-first greedy rule, so every rank
+ * derives the same table.  load_out (HOST, world doubles, may be NULL) gets
+ * the per-rank work.
+ */
+int muon_partition(const muon_group* groups, int n_groups, int world, int* owner_out, double* load_out);
+
+/*
  * Build a context: validate the descriptors, form shape buckets, carve the
  * caller's workspace (DEVICE memory, 1024-byte aligned, at least
  * muon_workspace_bytes() long, owned by the caller, alive until destroy),

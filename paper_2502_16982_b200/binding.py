@@ -30,7 +30,7 @@ MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
 MUON_SCALE_ADJUSTED_LR, MUON_SCALE_FIXED_DIM, MUON_SCALE_UPDATE_NORM = 0, 1, 2
 
 EXPORTED = [
-    "muon_workspace_bytes", "muon_init", "muon_step", "muon_step_host", "muon_status",
+    "muon_workspace_bytes", "muon_partition", "muon_init", "muon_step", "muon_step_host", "muon_status",
     "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
@@ -90,6 +90,7 @@ def lib():
             "libmuon_b200.so is not built (%s); run `python -m paper_2502_16982_b200.build`" % LIB_PATH)
     L = C.CDLL(LIB_PATH)
     L.muon_workspace_bytes.argtypes = [C.POINTER(muon_group), C.c_int, C.POINTER(C.c_size_t)]
+    L.muon_partition.argtypes = [C.POINTER(muon_group), C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_double)]
     L.muon_init.argtypes = [C.POINTER(C.c_void_p), C.POINTER(muon_group), C.c_int, C.c_void_p, C.c_size_t, C.c_int]
     L.muon_step.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_void_p]
     L.muon_step_host.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.POINTER(C.POINTER(C.c_void_p)),
@@ -252,6 +253,17 @@ def muon_adamw_step(params, grads, exp_avgs, exp_avg_sqs, step: int, lr: float, 
     s = torch.cuda.current_stream(dev) if stream is None else stream
     hp = muon_adamw_hparams(lr, wd, beta1, beta2, eps, int(step))
     _check(lib().muon_adamw_step(arr, n, C.byref(hp), dev, C.c_void_p(s.cuda_stream)))
+
+
+def muon_partition(shapes, world: int):
+    """Owner rank of every matrix for `world` data-parallel ranks.  ``shapes``
+    is a list of (rows, cols, count); returns (owners, loads)."""
+    arr = shape_only_groups([(r, c, n, MUON_DTYPE_BF16, MUON_DTYPE_BF16) for (r, c, n) in shapes])
+    total = sum(n for (_, _, n) in shapes)
+    owners = (C.c_int * total)()
+    loads = (C.c_double * world)()
+    _check(lib().muon_partition(arr, len(shapes), int(world), owners, loads))
+    return list(owners), list(loads)
 
 
 def muon_debug_set_chunk_bytes(nbytes: int) -> int:

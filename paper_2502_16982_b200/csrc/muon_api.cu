@@ -400,6 +400,36 @@ size_t muon_debug_set_chunk_bytes(size_t bytes) {
   return prev;
 }
 
+int muon_partition(const muon_group* groups, int n_groups, int world, int* owner_out, double* load_out) {
+  if (!owner_out || world <= 0) return fail(MUON_ERR_INVALID_ARG, "owner_out is null or world <= 0");
+  int rc = validate_groups(groups, n_groups, false);
+  if (rc) return rc;
+  // cost of one matrix: the Newton-Schulz work per iteration, 3 m^2 n + m^3
+  struct Item { double cost; int global; };
+  std::vector<Item> items;
+  int global = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    const double m = std::min(groups[g].rows, groups[g].cols), n = std::max(groups[g].rows, groups[g].cols);
+    const double cost = 3.0 * m * m * n + m * m * m;
+    for (int i = 0; i < groups[g].count; ++i) items.push_back(Item{cost, global++});
+  }
+  // longest processing time first: heaviest matrices first, each to the least
+  // loaded rank; ties by matrix order and by rank, so every rank computes the
+  // same assignment
+  std::stable_sort(items.begin(), items.end(), [](const Item& a, const Item& b) { return a.cost > b.cost; });
+  std::vector<double> load(world, 0.0);
+  for (const Item& it : items) {
+    int best = 0;
+    for (int r = 1; r < world; ++r)
+      if (load[r] < load[best]) best = r;
+    owner_out[it.global] = best;
+    load[best] += it.cost;
+  }
+  if (load_out)
+    for (int r = 0; r < world; ++r) load_out[r] = load[r];
+  return MUON_OK;
+}
+
 int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_bytes) {
   if (!out_bytes) return fail(MUON_ERR_INVALID_ARG, "out_bytes is null");
   int rc = validate_groups(groups, n_groups, false);

@@ -350,6 +350,46 @@ def test_fp32_master_weights_with_bf16_shadow():
         b.MuonContext([(wl.views(Wb), wl.views(Gd), wl.views(Md), wl.views(shadow))])
 
 
+def test_owner_computes_shards_give_the_single_context_bits():
+    """Sec. 2.3: each matrix is stepped by its owner rank alone.  A matrix's
+    result must not depend on which other matrices share its launch, so the
+    union of two ranks' shards equals the single-context result bit for bit."""
+    b = _binding()
+    specs = [wl.GroupSpec(328, 200, 5, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
+             wl.GroupSpec(200, 328, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(256, 256, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
+    owners, _ = b.muon_partition([(sp.rows, sp.cols, sp.count) for sp in specs], 2)
+    hp = default_hp(lr=1e-2)
+    single = Case(specs, seed=61)
+    shard = Case(specs, seed=61)  # same bits; stepped by two "ranks", each over its own matrices
+    try:
+        for _ in range(2):
+            assert single.step(hp)[0] == 0
+        ctxs = []
+        for rank in range(2):
+            groups, k = [], 0
+            for gi, sp in enumerate(specs):
+                idx = [i for i in range(sp.count) if owners[k + i] == rank]
+                k += sp.count
+                if idx:
+                    W, G, M = shard.dev[gi]
+                    groups.append(([W[i] for i in idx], [G[i] for i in idx], [M[i] for i in idx]))
+            assert groups
+            ctxs.append(b.MuonContext(groups))
+        for _ in range(2):
+            for c in ctxs:
+                c.muon_step(hp)
+                assert c.muon_status()[0] == 0
+        for gi in range(len(specs)):
+            assert torch.equal(single.dev[gi][0], shard.dev[gi][0])
+            assert torch.equal(single.dev[gi][2], shard.dev[gi][2])
+        for c in ctxs:
+            c.muon_destroy()
+    finally:
+        single.close()
+        shard.close()
+
+
 def test_bitwise_reproducible():
     specs = [wl.GroupSpec(448, 640, 4, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
     outs = []
