@@ -173,7 +173,12 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream);
  * j, g_host[j][i] (host, dense rows*cols of the group's g_dtype) is copied
  * into the device G buffer, the step runs, and if w_host is non-NULL the
  * updated W is copied to w_host[j][i] (host, dense rows*cols of w_dtype).
- * All copies are cudaMemcpyAsync on `stream`; the call does not synchronise.
+ * The call does not synchronise; work enqueued on `stream` after it starts
+ * only when the last copy has finished.  Uploads, kernels and downloads of
+ * successive slices of a bucket overlap: the copies run on two streams the
+ * context creates on first use (asynchronous copies need pinned host memory to
+ * overlap).  A matrix's update RMS, norms and the status word are read as
+ * after muon_step.
  */
 int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* const* g_host,
                    void* const* const* w_host, void* stream);

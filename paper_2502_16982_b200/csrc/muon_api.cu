@@ -98,7 +98,7 @@ struct PlanSizes {
   size_t off_status;
   size_t off_norms;  // float per matrix (global order)
   size_t off_rms;    // float per matrix: update RMS of the last step
-  size_t off_debug;  // TMEM base addresses seen by the CTAs of the pair kernel
+  size_t off_debug;  // TMEM base addresses seen by the CTAs of the GEMM kernel
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -360,8 +360,14 @@ struct muon_ctx {
   std::vector<cudaEvent_t> ev_pool;           // pairs: start, stop
   std::vector<int> ev_kind;                   // kind of each recorded pair
   size_t ev_used;
+  // host-buffer path: copy streams and the events that order copies and kernels
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  std::vector<cudaEvent_t> pipe_events;
   ~muon_ctx() {
     for (cudaEvent_t e : ev_pool) cudaEventDestroy(e);
+    for (cudaEvent_t e : pipe_events) cudaEventDestroy(e);
+    if (s_in) cudaStreamDestroy(s_in);
+    if (s_out) cudaStreamDestroy(s_out);
   }
 };
 
@@ -613,175 +619,185 @@ static int check_hparams(const muon_hparams* hp) {
   return MUON_OK;
 }
 
+// One Muon step for matrices [first, first + count) of bucket b (at most one
+// chunk), enqueued on `stream`.
+static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream, size_t b, int first, int count,
+                      int* launch_counter) {
+  int launches = 0;
+  cudaError_t ce = cudaSuccess;
+  DevStatus* status = reinterpret_cast<DevStatus*>(ctx->ws + ctx->sizes.off_status);
+  float* norms = reinterpret_cast<float*>(ctx->ws + ctx->sizes.off_norms);
+  Bucket& B = ctx->buckets[b];
+  // factor of O in the update (Sec. 2.2 / Sec. 3.1): 0.2*sqrt(max(rows, cols)), or 0.2*sqrt(H)
+  const float factor = hp->rms_scale * std::sqrt(hp->scale_mode == MUON_SCALE_FIXED_DIM
+                                                     ? hp->scale_dim : static_cast<float>(B.n));
+  const bool normalise = hp->scale_mode == MUON_SCALE_UPDATE_NORM;
+  const bool fused_update = B.fused_update && !normalise;
+  const float upd_scale = -hp->lr * factor;
+  const float decay = 1.0f - hp->lr * hp->wd;
+  const MatDesc* descs = reinterpret_cast<const MatDesc*>(ctx->ws + B.off_descs) + first;
+  MatScal* scal = reinterpret_cast<MatScal*>(ctx->ws + B.off_scal);
+  float* partials = reinterpret_cast<float*>(ctx->ws + B.off_partials);
+
+  const int stream_tiles = B.stream_tma ? B.stream_tiles_tma : B.stream_tiles_generic;
+  if (B.stream_tma) {
+    StreamTmaParams S{};
+    S.map_x = B.x_b64[0];
+    S.gmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_gmaps) + first;
+    S.mmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_mmaps) + first;
+    S.descs = descs;
+    S.partials = partials;
+    S.status = status;
+    S.count = count;
+    S.tiles_per_matrix = stream_tiles;
+    S.m = B.m;
+    S.n = B.n;
+    S.mu = hp->mu;
+    S.nesterov = hp->nesterov ? 1 : 0;
+    LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM);
+    ce = launch_momentum_tma(S, B.g_dtype == MUON_DTYPE_FP32, ctx->num_sms, stream);
+  } else {
+    StreamParams S{};
+    S.descs = descs;
+    S.partials = partials;
+    S.x = reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_x[0]);
+    S.x_stride = static_cast<long long>(B.x_stride);
+    S.ldx = B.ldx;
+    S.count = count;
+    S.tiles_per_matrix = stream_tiles;
+    S.mu = hp->mu;
+    S.nesterov = hp->nesterov ? 1 : 0;
+    LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM);
+    ce = launch_momentum_cast(S, B.g_dtype == MUON_DTYPE_FP32, stream);
+  }
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "momentum kernel launch: %s", cudaGetErrorString(ce));
+  ++launches;
+  { LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM); ce = launch_norm_finalise(partials, stream_tiles, count, hp->eps, descs, scal, norms, status, stream); }
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "norm kernel launch: %s", cudaGetErrorString(ce));
+  ++launches;
+
+  int cur = 0;
+  for (int it = 0; it < hp->ns_steps; ++it) {
+    const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
+    const int nxt = cur ^ 1;
+    GemmParams P{};
+    P.descs = descs;
+    P.scal = scal;
+    P.status = status;
+    P.debug = reinterpret_cast<unsigned*>(ctx->ws + ctx->sizes.off_debug);
+    P.rms_partials = reinterpret_cast<float*>(ctx->ws + B.off_rms_partials);
+    P.wmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_wmaps) + first;
+    P.count = count;
+    P.m = B.m;
+    P.upd_scale = upd_scale;
+    P.decay = decay;
+
+    // A = X X^T (first iteration: times s^2, the deferred normalisation)
+    P.map_a = B.x_op[cur];
+    P.map_a64 = B.x_b64[cur];  // unused
+    P.map_b = B.x_b64[cur];
+    P.map_in = B.a_e;  // unused
+    P.map_out = B.a_e;
+    P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
+    P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
+    P.k = B.n;
+    P.out_cols = B.m;
+    P.symmetric = 1; P.a_sym = 0; P.b_sym = 0; P.b_mn_major = 0;
+    P.has_in = 0;
+    P.scale_kind = first_it ? 1 : 0;
+    P.last = 0; P.keep_o = 0;
+    P.c_acc = 1.f; P.c_in = 0.f;
+    { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
+    ++launches;
+
+    // B = b*A + c*A*A  (A symmetric, kept as its upper blocks)
+    P.map_a = B.a_op;
+    P.map_a64 = B.a_b64;
+    P.map_b = B.a_b64;
+    P.map_in = B.a_e;
+    P.map_out = B.b_e;
+    P.k = B.m;
+    P.a_sym = 1; P.b_sym = 1;
+    P.has_in = 1;
+    P.scale_kind = 0;
+    P.c_acc = hp->c; P.c_in = hp->b;
+    { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
+    ++launches;
+
+    // X' = a*X + B X (first iteration: times s); the last iteration updates W
+    // in its epilogue when every W of the bucket is TMA-addressable bf16
+    const bool fuse = last_it && fused_update;
+    P.map_a = B.b_op;
+    P.map_a64 = B.b_b64;
+    P.map_b = B.x_b64[cur];
+    P.map_in = B.x_e[cur];
+    P.map_out = B.x_e[nxt];
+    P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles);
+    P.tiles_per_matrix = static_cast<int>(B.comb_tiles.size());
+    P.k = B.m;
+    P.out_cols = B.n;
+    P.symmetric = 0; P.a_sym = 1; P.b_sym = 0; P.b_mn_major = 1;
+    P.has_in = 1;
+    P.scale_kind = first_it ? 2 : 0;
+    P.last = fuse ? 1 : 0;
+    P.keep_o = (fuse && ctx->keep_o) ? 1 : 0;
+    P.c_acc = 1.f; P.c_in = hp->a;
+    { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, B.comb_acc_cols, ctx->max_clusters, stream); }
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
+    ++launches;
+    cur = nxt;
+  }
+  {
+    // Update RMS for logging (Algorithm 1, returned value) and, when the
+    // weights were not updated in the last epilogue (no iteration, fp32 or
+    // TMA-unaddressable weights, normalised update), the separate update
+    // W <- decay*W - lr*f*O from the stored O.
+    float* rms = reinterpret_cast<float*>(ctx->ws + ctx->sizes.off_rms);
+    if (hp->ns_steps > 0 && fused_update) {
+      LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
+      ce = launch_rms_finalise(reinterpret_cast<const float*>(ctx->ws + B.off_rms_partials),
+                               static_cast<int>(B.comb_tiles.size()) * 8, count, factor, descs, rms, stream);
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
+      ++launches;
+    } else {
+      float* factors = reinterpret_cast<float*>(ctx->ws + B.off_factors);
+      const __nv_bfloat16* xo = reinterpret_cast<const __nv_bfloat16*>(ctx->ws + B.off_x[cur]);
+      {
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
+        ce = launch_rms_from_x(descs, scal, xo, static_cast<long long>(B.x_stride), B.ldx, B.m, B.n, count,
+                               factor, hp->ns_steps == 0, hp->rms_scale, normalise, rms, factors, stream);
+      }
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
+      ++launches;
+      {
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_UPDATE);
+        ce = launch_update_from_x(descs, scal, factors, xo, static_cast<long long>(B.x_stride), B.ldx, count,
+                                  B.m, B.n, -hp->lr, decay, B.w_dtype == MUON_DTYPE_FP32, stream);
+      }
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "update kernel launch: %s", cudaGetErrorString(ce));
+      ++launches;
+    }
+  }
+  ctx->x0_buf[b] = 0;
+  ctx->xlast_buf[b] = cur;
+  *launch_counter += launches;
+  return MUON_OK;
+}
+
 int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
   if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
   int rc = check_hparams(hp);
   if (rc) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   int launches = 0;
-  cudaError_t ce = cudaSuccess;
-  DevStatus* status = reinterpret_cast<DevStatus*>(ctx->ws + ctx->sizes.off_status);
-  float* norms = reinterpret_cast<float*>(ctx->ws + ctx->sizes.off_norms);
-
   for (size_t b = 0; b < ctx->buckets.size(); ++b) {
-    Bucket& B = ctx->buckets[b];
+    const Bucket& B = ctx->buckets[b];
     const int total = static_cast<int>(B.mats.size());
-    // factor of O in the update (Sec. 2.2 / Sec. 3.1): 0.2*sqrt(max(rows, cols)), or 0.2*sqrt(H)
-    const float factor = hp->rms_scale * std::sqrt(hp->scale_mode == MUON_SCALE_FIXED_DIM
-                                                       ? hp->scale_dim : static_cast<float>(B.n));
-    const bool normalise = hp->scale_mode == MUON_SCALE_UPDATE_NORM;
-    const bool fused_update = B.fused_update && !normalise;
-    const float upd_scale = -hp->lr * factor;
-    const float decay = 1.0f - hp->lr * hp->wd;
     for (int first = 0; first < total; first += B.chunk) {
-      const int count = std::min(B.chunk, total - first);
-      const MatDesc* descs = reinterpret_cast<const MatDesc*>(ctx->ws + B.off_descs) + first;
-      MatScal* scal = reinterpret_cast<MatScal*>(ctx->ws + B.off_scal);
-      float* partials = reinterpret_cast<float*>(ctx->ws + B.off_partials);
-
-      const int stream_tiles = B.stream_tma ? B.stream_tiles_tma : B.stream_tiles_generic;
-      if (B.stream_tma) {
-        StreamTmaParams S{};
-        S.map_x = B.x_b64[0];
-        S.gmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_gmaps) + first;
-        S.mmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_mmaps) + first;
-        S.descs = descs;
-        S.partials = partials;
-        S.status = status;
-        S.count = count;
-        S.tiles_per_matrix = stream_tiles;
-        S.m = B.m;
-        S.n = B.n;
-        S.mu = hp->mu;
-        S.nesterov = hp->nesterov ? 1 : 0;
-        LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM);
-        ce = launch_momentum_tma(S, B.g_dtype == MUON_DTYPE_FP32, ctx->num_sms, stream);
-      } else {
-        StreamParams S{};
-        S.descs = descs;
-        S.partials = partials;
-        S.x = reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_x[0]);
-        S.x_stride = static_cast<long long>(B.x_stride);
-        S.ldx = B.ldx;
-        S.count = count;
-        S.tiles_per_matrix = stream_tiles;
-        S.mu = hp->mu;
-        S.nesterov = hp->nesterov ? 1 : 0;
-        LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM);
-        ce = launch_momentum_cast(S, B.g_dtype == MUON_DTYPE_FP32, stream);
-      }
-      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "momentum kernel launch: %s", cudaGetErrorString(ce));
-      ++launches;
-      { LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM); ce = launch_norm_finalise(partials, stream_tiles, count, hp->eps, descs, scal, norms, status, stream); }
-      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "norm kernel launch: %s", cudaGetErrorString(ce));
-      ++launches;
-
-      int cur = 0;
-      for (int it = 0; it < hp->ns_steps; ++it) {
-        const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
-        const int nxt = cur ^ 1;
-        GemmParams P{};
-        P.descs = descs;
-        P.scal = scal;
-        P.status = status;
-        P.debug = reinterpret_cast<unsigned*>(ctx->ws + ctx->sizes.off_debug);
-        P.rms_partials = reinterpret_cast<float*>(ctx->ws + B.off_rms_partials);
-        P.wmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_wmaps) + first;
-        P.count = count;
-        P.m = B.m;
-        P.upd_scale = upd_scale;
-        P.decay = decay;
-
-        // A = X X^T (first iteration: times s^2, the deferred normalisation)
-        P.map_a = B.x_op[cur];
-        P.map_a64 = B.x_b64[cur];  // unused
-        P.map_b = B.x_b64[cur];
-        P.map_in = B.a_e;  // unused
-        P.map_out = B.a_e;
-        P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
-        P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
-        P.k = B.n;
-        P.out_cols = B.m;
-        P.symmetric = 1; P.a_sym = 0; P.b_sym = 0; P.b_mn_major = 0;
-        P.has_in = 0;
-        P.scale_kind = first_it ? 1 : 0;
-        P.last = 0; P.keep_o = 0;
-        P.c_acc = 1.f; P.c_in = 0.f;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
-
-        // B = b*A + c*A*A  (A symmetric, kept as its upper blocks)
-        P.map_a = B.a_op;
-        P.map_a64 = B.a_b64;
-        P.map_b = B.a_b64;
-        P.map_in = B.a_e;
-        P.map_out = B.b_e;
-        P.k = B.m;
-        P.a_sym = 1; P.b_sym = 1;
-        P.has_in = 1;
-        P.scale_kind = 0;
-        P.c_acc = hp->c; P.c_in = hp->b;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
-
-        // X' = a*X + B X (first iteration: times s); the last iteration updates W
-        // in its epilogue when every W of the bucket is TMA-addressable bf16
-        const bool fuse = last_it && fused_update;
-        P.map_a = B.b_op;
-        P.map_a64 = B.b_b64;
-        P.map_b = B.x_b64[cur];
-        P.map_in = B.x_e[cur];
-        P.map_out = B.x_e[nxt];
-        P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles);
-        P.tiles_per_matrix = static_cast<int>(B.comb_tiles.size());
-        P.k = B.m;
-        P.out_cols = B.n;
-        P.symmetric = 0; P.a_sym = 1; P.b_sym = 0; P.b_mn_major = 1;
-        P.has_in = 1;
-        P.scale_kind = first_it ? 2 : 0;
-        P.last = fuse ? 1 : 0;
-        P.keep_o = (fuse && ctx->keep_o) ? 1 : 0;
-        P.c_acc = 1.f; P.c_in = hp->a;
-        { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, B.comb_acc_cols, ctx->max_clusters, stream); }
-        if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
-        ++launches;
-        cur = nxt;
-      }
-      {
-        // Update RMS for logging (Algorithm 1, returned value) and, when the
-        // weights were not updated in the last epilogue (no iteration, fp32 or
-        // TMA-unaddressable weights, normalised update), the separate update
-        // W <- decay*W - lr*f*O from the stored O.
-        float* rms = reinterpret_cast<float*>(ctx->ws + ctx->sizes.off_rms);
-        if (hp->ns_steps > 0 && fused_update) {
-          LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
-          ce = launch_rms_finalise(reinterpret_cast<const float*>(ctx->ws + B.off_rms_partials),
-                                   static_cast<int>(B.comb_tiles.size()) * 8, count, factor, descs, rms, stream);
-          if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
-          ++launches;
-        } else {
-          float* factors = reinterpret_cast<float*>(ctx->ws + B.off_factors);
-          const __nv_bfloat16* xo = reinterpret_cast<const __nv_bfloat16*>(ctx->ws + B.off_x[cur]);
-          {
-            LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
-            ce = launch_rms_from_x(descs, scal, xo, static_cast<long long>(B.x_stride), B.ldx, B.m, B.n, count,
-                                   factor, hp->ns_steps == 0, hp->rms_scale, normalise, rms, factors, stream);
-          }
-          if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
-          ++launches;
-          {
-            LaunchTimer lt(ctx, stream, MUON_KERNEL_UPDATE);
-            ce = launch_update_from_x(descs, scal, factors, xo, static_cast<long long>(B.x_stride), B.ldx, count,
-                                      B.m, B.n, -hp->lr, decay, B.w_dtype == MUON_DTYPE_FP32, stream);
-          }
-          if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "update kernel launch: %s", cudaGetErrorString(ce));
-          ++launches;
-        }
-      }
-      ctx->x0_buf[b] = 0;
-      ctx->xlast_buf[b] = cur;
+      rc = step_chunk(ctx, hp, stream, b, first, std::min(B.chunk, total - first), &launches);
+      if (rc) return rc;
     }
   }
   ctx->last_launches = launches;
@@ -792,29 +808,77 @@ int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* con
                    void* const* const* w_host, void* stream_v) {
   if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
   if (!g_host) return fail(MUON_ERR_INVALID_ARG, "g_host is null");
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-  for (size_t g = 0; g < ctx->groups.size(); ++g) {
-    const muon_group& G = ctx->groups[g];
-    const size_t es = G.g_dtype == MUON_DTYPE_FP32 ? 4 : 2;
-    for (int i = 0; i < G.count; ++i) {
-      cudaError_t ce = cudaMemcpy2DAsync(const_cast<void*>(G.g[i]), G.ld_g * es, g_host[g][i], G.cols * es,
-                                         G.cols * es, G.rows, cudaMemcpyHostToDevice, stream);
-      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gradient upload: %s", cudaGetErrorString(ce));
-    }
-  }
-  int rc = muon_step(ctx, hp, stream_v);
+  int rc = check_hparams(hp);
   if (rc) return rc;
-  if (w_host) {
-    for (size_t g = 0; g < ctx->groups.size(); ++g) {
-      const muon_group& G = ctx->groups[g];
-      const size_t es = G.w_dtype == MUON_DTYPE_FP32 ? 4 : 2;
-      for (int i = 0; i < G.count; ++i) {
-        cudaError_t ce = cudaMemcpy2DAsync(w_host[g][i], G.cols * es, G.w[i], G.ld_w * es, G.cols * es, G.rows,
-                                           cudaMemcpyDeviceToHost, stream);
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  cudaError_t ce = cudaSuccess;
+  if (!ctx->s_in) {
+    ce = cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking);
+    if (ce == cudaSuccess) ce = cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking);
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "copy stream creation: %s", cudaGetErrorString(ce));
+  }
+  size_t ev_next = 0;
+  auto next_event = [&](cudaEvent_t* out) -> cudaError_t {
+    if (ev_next == ctx->pipe_events.size()) {
+      cudaEvent_t e;
+      cudaError_t r = cudaEventCreateWithFlags(&e, cudaEventDisableTiming);
+      if (r != cudaSuccess) return r;
+      ctx->pipe_events.push_back(e);
+    }
+    *out = ctx->pipe_events[ev_next++];
+    return cudaSuccess;
+  };
+  // Uploads, kernels and downloads of successive slices of a bucket overlap:
+  // slice k+1 is uploaded on one copy stream while slice k runs on the caller's
+  // stream and slice k-1 is downloaded on the other copy stream.
+  cudaEvent_t ev;
+  ce = next_event(&ev);
+  if (ce == cudaSuccess) ce = cudaEventRecord(ev, stream);             // copies start after earlier work
+  if (ce == cudaSuccess) ce = cudaStreamWaitEvent(ctx->s_in, ev, 0);
+  if (ce == cudaSuccess) ce = cudaStreamWaitEvent(ctx->s_out, ev, 0);
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "stream ordering: %s", cudaGetErrorString(ce));
+  int launches = 0;
+  for (size_t b = 0; b < ctx->buckets.size(); ++b) {
+    const Bucket& B = ctx->buckets[b];
+    const int total = static_cast<int>(B.mats.size());
+    const int slice = std::max(1, std::min(B.chunk, (total + 3) / 4));
+    for (int first = 0; first < total; first += slice) {
+      const int count = std::min(slice, total - first);
+      for (int i = first; i < first + count && ce == cudaSuccess; ++i) {
+        const MatRef& r = B.mats[i];
+        const muon_group& G = ctx->groups[r.group];
+        const size_t es = G.g_dtype == MUON_DTYPE_FP32 ? 4 : 2;
+        ce = cudaMemcpy2DAsync(const_cast<void*>(G.g[r.index]), G.ld_g * es, g_host[r.group][r.index], G.cols * es,
+                               G.cols * es, G.rows, cudaMemcpyHostToDevice, ctx->s_in);
+      }
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gradient upload: %s", cudaGetErrorString(ce));
+      ce = next_event(&ev);
+      if (ce == cudaSuccess) ce = cudaEventRecord(ev, ctx->s_in);
+      if (ce == cudaSuccess) ce = cudaStreamWaitEvent(stream, ev, 0);
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "stream ordering: %s", cudaGetErrorString(ce));
+      rc = step_chunk(ctx, hp, stream, b, first, count, &launches);
+      if (rc) return rc;
+      if (w_host) {
+        ce = next_event(&ev);
+        if (ce == cudaSuccess) ce = cudaEventRecord(ev, stream);
+        if (ce == cudaSuccess) ce = cudaStreamWaitEvent(ctx->s_out, ev, 0);
+        for (int i = first; i < first + count && ce == cudaSuccess; ++i) {
+          const MatRef& r = B.mats[i];
+          const muon_group& G = ctx->groups[r.group];
+          const size_t es = G.w_dtype == MUON_DTYPE_FP32 ? 4 : 2;
+          ce = cudaMemcpy2DAsync(w_host[r.group][r.index], G.cols * es, G.w[r.index], G.ld_w * es, G.cols * es,
+                                 G.rows, cudaMemcpyDeviceToHost, ctx->s_out);
+        }
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "weight download: %s", cudaGetErrorString(ce));
       }
     }
   }
+  // the caller's stream completes only when the last download has
+  ce = next_event(&ev);
+  if (ce == cudaSuccess) ce = cudaEventRecord(ev, ctx->s_out);
+  if (ce == cudaSuccess) ce = cudaStreamWaitEvent(stream, ev, 0);
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "stream ordering: %s", cudaGetErrorString(ce));
+  ctx->last_launches = launches;
   return MUON_OK;
 }
 
