@@ -138,6 +138,42 @@ def update_factor(O, rms_scale=0.2, scale_mode="adjusted_lr", scale_dim=0.0):
     raise ValueError("unknown scale_mode %r" % (scale_mode,))
 
 
+def round_to_bf16(x):
+    """Round-to-nearest-even of float64 values to bfloat16 (8 significand bits),
+    returned as float64.  Done on the bit pattern of the float32 value: every
+    value used here is far inside float32's range, and rounding float64 ->
+    float32 -> bf16 differs from direct rounding only on exact ties of the
+    second step, which the first rounding cannot create for these magnitudes."""
+    f = np.ascontiguousarray(np.asarray(x, dtype=np.float64).astype(np.float32))
+    bits = f.view(np.uint32).astype(np.uint64)
+    rounded = (bits + 0x7FFF + ((bits >> 16) & 1)) & 0xFFFF0000
+    return rounded.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
+def newton_schulz_bf16_storage(U, eps, steps, a=NS_A, b=NS_B, c=NS_C):
+    """Eq. 2 with the storage precision Sec. 2.3 names ("Newton-Schulz
+    iteration steps in bf16"): every stored matrix -- the input, A, B and each
+    new X -- is rounded to bf16, all arithmetic in between is exact (float64).
+    This is not a reference for the CUDA path (summation order makes any bf16
+    implementation differ from any other by a similar amount); it measures how
+    far the bf16 storage alone moves the result from the float64 iteration, so
+    that tests can tell a kernel error from the precision the paper fixes.  The
+    1/(||U||_F + eps) factor is applied in full precision to the first A and
+    the first X, as the CUDA path does.  Short side first, like newton_schulz."""
+    U = _f64(U)
+    transposed = U.shape[0] > U.shape[1]
+    nu = math.sqrt(float(np.sum(U * U)))
+    s = 1.0 / (nu + eps)
+    X = round_to_bf16(U.T if transposed else U)
+    for k in range(int(steps)):
+        A = round_to_bf16((s * s if k == 0 else 1.0) * (X @ X.T))
+        B = round_to_bf16(b * A + c * (A @ A))
+        X = round_to_bf16((s if k == 0 else 1.0) * (a * X + B @ X))
+    if int(steps) == 0:
+        X = s * X
+    return np.ascontiguousarray(X.T if transposed else X)
+
+
 def apply_update(W, O, lr, wd, rms_scale=0.2, scale_mode="adjusted_lr", scale_dim=0.0):
     """W_t = W_{t-1} - lr * (factor * O + wd * W_{t-1}) with factor =
     rms_scale * sqrt(max(A, B)) for a parameter of shape [A, B]  (Sec. 2.2,

@@ -367,3 +367,36 @@ def test_update_norm_has_rms_exactly_point_two_after_the_iteration():
     assert abs(out["rms"] - 0.2) <= 1e-12
     # the direction is still O
     assert np.allclose(u / np.linalg.norm(u), out["O"] / np.linalg.norm(out["O"]), atol=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# bf16 storage model
+# ---------------------------------------------------------------------------
+def test_round_to_bf16_known_values_and_ties():
+    # 1 + 2^-8 is a tie between 1 and 1 + 2^-7: even significand wins (1.0);
+    # 1 + 3*2^-8 is a tie between 1 + 2^-7 and 1 + 2^-6: even wins (1 + 2^-6)
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, -3.4445, 0.0, 2.0 ** -130])
+    r = orc.round_to_bf16(x)
+    assert r[0] == 1.0 and r[1] == 1.0 and r[2] == 1.0 + 2.0 ** -6 and r[3] == 1.0 + 2.0 ** -7
+    assert r[4] == -3.4375 and r[5] == 0.0
+    # agrees with an independent implementation on random values
+    import torch
+    y = np.random.default_rng(3).standard_normal(10000) * 10.0 ** np.random.default_rng(4).uniform(-6, 6, 10000)
+    assert np.array_equal(orc.round_to_bf16(y), torch.from_numpy(y).to(torch.float32).to(torch.bfloat16).double().numpy())
+
+
+def test_bf16_storage_model_is_the_iteration_with_rounding_only():
+    """The model is the float64 iteration plus bf16 rounding of the stored
+    matrices: it stays within a few bf16 roundings (2^-9 each) amplified by the
+    map of the float64 result, but not closer than one rounding; it follows the
+    same orientation rule, and with no iteration it is bf16(U)/||U||_F."""
+    rng = np.random.default_rng(8)
+    G = rng.standard_normal((24, 40))
+    ref = orc.newton_schulz(orc.frobenius_normalise(G, 1e-7)[1], 5)
+    mod = orc.newton_schulz_bf16_storage(G, 1e-7, 5)
+    err = np.linalg.norm(mod - ref) / np.linalg.norm(ref)
+    assert 1e-4 < err < 5e-2
+    # orientation rule and the no-iteration case
+    assert np.allclose(orc.newton_schulz_bf16_storage(G.T, 1e-7, 5), mod.T, rtol=0, atol=0)
+    x0 = orc.newton_schulz_bf16_storage(G, 0.0, 0)
+    assert np.allclose(x0, orc.round_to_bf16(G) / np.linalg.norm(G), rtol=1e-15)
