@@ -49,6 +49,7 @@ WORKLOAD_NAMES = {
     3: "cfg3: MoE expert bucket, 198 matrices of 2048x1408 / 1408x2048 (0.571 G params)",
     4: "cfg4: shape sweep, 7 single matrices",
     5: "cfg5: Moonlight-shaped full parameter set (5286 matrices, 15.3 G params)",
+    6: "cfg6: the five dense scaling-law models, hidden 1536-2560, MLP [H, 2.6H] (560 matrices, 4.3 G params)",
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
@@ -233,7 +234,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5, 6])
     ap.add_argument("--layers", type=int, default=None, help="shrink configs 2 and 5 (tests only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ns-steps", type=int, default=5, help="Newton-Schulz iterations (the paper uses 5)")

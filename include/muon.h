@@ -105,6 +105,9 @@ typedef struct muon_group {
  *                                       scale_dim = the model's hidden size H),
  *               MUON_SCALE_UPDATE_NORM  rms_scale * O / RMS(O)  ("Update Norm").
  *   scale_dim : H for MUON_SCALE_FIXED_DIM, ignored otherwise.
+ *   coeffs    : NULL, or a HOST array of 3 * ns_steps floats (a_1, b_1, c_1, a_2, ...)
+ *               giving every iteration its own quintic; then a, b, c are ignored.
+ *               (The paper uses one triple for all iterations.)
  */
 enum { MUON_SCALE_ADJUSTED_LR = 0, MUON_SCALE_FIXED_DIM = 1, MUON_SCALE_UPDATE_NORM = 2 };
 typedef struct muon_hparams {
@@ -120,6 +123,7 @@ typedef struct muon_hparams {
   float rms_scale;
   int32_t scale_mode;
   float scale_dim;
+  const float* coeffs;
 } muon_hparams;
 
 typedef struct muon_ctx muon_ctx;

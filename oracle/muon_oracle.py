@@ -63,6 +63,9 @@ class Hyper:
     # (Baseline; scale_dim is the hidden size H) or "update_norm".
     scale_mode: str = "adjusted_lr"
     scale_dim: float = 0.0
+    # Optional list of (a, b, c), one triple per Newton-Schulz step, replacing
+    # the single triple above (the paper uses one triple for all steps).
+    coeffs: object = None
 
 
 def _f64(x):
@@ -96,8 +99,9 @@ def frobenius_normalise(U, eps):
     return nu, U / (nu + eps)
 
 
-def newton_schulz(X0, steps, a=NS_A, b=NS_B, c=NS_C, trace=None):
+def newton_schulz(X0, steps, a=NS_A, b=NS_B, c=NS_C, trace=None, coeffs=None):
     """N steps of Eq. 2:  X_k = a X + b (X X^T) X + c (X X^T)^2 X.
+    With ``coeffs`` (a list of N triples) step k uses its own (a, b, c).
 
     When the matrix has more rows than columns the iteration runs on the
     transpose and the result is transposed back; the polynomial is odd, so in
@@ -110,7 +114,11 @@ def newton_schulz(X0, steps, a=NS_A, b=NS_B, c=NS_C, trace=None):
     if transposed:
         X = X.T
     X = X.copy()
-    for _ in range(int(steps)):
+    if coeffs is not None and len(coeffs) != int(steps):
+        raise ValueError("coeffs must hold one (a, b, c) per step")
+    for k in range(int(steps)):
+        if coeffs is not None:
+            a, b, c = coeffs[k]
         A = X @ X.T
         B = b * A + c * (A @ A)
         X = a * X + B @ X
@@ -217,7 +225,7 @@ def muon_step(W, G, M, hp: Hyper, trace=False):
         out.update(W=W.copy(), X0=None, O=None, rms=float("nan"), nonfinite=True)
         return out
     stages = [] if trace else None
-    O = newton_schulz(X0, hp.ns_steps, hp.a, hp.b, hp.c, trace=stages)
+    O = newton_schulz(X0, hp.ns_steps, hp.a, hp.b, hp.c, trace=stages, coeffs=hp.coeffs)
     out.update(
         W=apply_update(W, O, hp.lr, hp.wd, hp.rms_scale, hp.scale_mode, hp.scale_dim),
         X0=X0,

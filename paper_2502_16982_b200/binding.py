@@ -57,6 +57,7 @@ class muon_hparams(C.Structure):
         ("a", C.c_float), ("b", C.c_float), ("c", C.c_float),
         ("eps", C.c_float), ("rms_scale", C.c_float),
         ("scale_mode", C.c_int32), ("scale_dim", C.c_float),
+        ("coeffs", C.POINTER(C.c_float)),
     ]
 
 
@@ -144,11 +145,19 @@ class Hyper:
     rms_scale: float = 0.2
     scale_mode: int = MUON_SCALE_ADJUSTED_LR
     scale_dim: float = 0.0
+    coeffs: Optional[Sequence] = None  # one (a, b, c) per Newton-Schulz step
 
     def to_c(self) -> muon_hparams:
-        return muon_hparams(self.lr, self.wd, self.mu, int(bool(self.nesterov)), int(self.ns_steps),
-                            self.a, self.b, self.c, self.eps, self.rms_scale, int(self.scale_mode),
-                            float(self.scale_dim))
+        hp = muon_hparams(self.lr, self.wd, self.mu, int(bool(self.nesterov)), int(self.ns_steps),
+                          self.a, self.b, self.c, self.eps, self.rms_scale, int(self.scale_mode),
+                          float(self.scale_dim), None)
+        if self.coeffs is not None:
+            flat = [float(v) for triple in self.coeffs for v in triple]
+            if len(flat) != 3 * int(self.ns_steps):
+                raise MuonError(MUON_ERR_INVALID_ARG, "coeffs must hold one (a, b, c) per Newton-Schulz step")
+            self._coeffs_c = (C.c_float * len(flat))(*flat)  # kept alive by the Hyper object
+            hp.coeffs = C.cast(self._coeffs_c, C.POINTER(C.c_float))
+        return hp
 
 
 def _dtype_code(t):

@@ -613,6 +613,8 @@ static int check_hparams(const muon_hparams* hp) {
     return fail(MUON_ERR_INVALID_ARG, "unknown scale_mode");
   if (hp->scale_mode == MUON_SCALE_FIXED_DIM && !(hp->scale_dim > 0.f))
     return fail(MUON_ERR_INVALID_ARG, "scale_dim must be positive with MUON_SCALE_FIXED_DIM");
+  for (int i = 0; hp->coeffs && i < 3 * hp->ns_steps; ++i)
+    if (!std::isfinite(hp->coeffs[i])) return fail(MUON_ERR_INVALID_ARG, "coefficient schedule must be finite");
   if (!std::isfinite(hp->lr) || !std::isfinite(hp->wd) || !std::isfinite(hp->mu) || !std::isfinite(hp->a) ||
       !std::isfinite(hp->b) || !std::isfinite(hp->c) || !std::isfinite(hp->rms_scale))
     return fail(MUON_ERR_INVALID_ARG, "hyper-parameters must be finite");
@@ -680,6 +682,9 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
   for (int it = 0; it < hp->ns_steps; ++it) {
     const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
     const int nxt = cur ^ 1;
+    const float co_a = hp->coeffs ? hp->coeffs[3 * it] : hp->a;
+    const float co_b = hp->coeffs ? hp->coeffs[3 * it + 1] : hp->b;
+    const float co_c = hp->coeffs ? hp->coeffs[3 * it + 2] : hp->c;
     GemmParams P{};
     P.descs = descs;
     P.scal = scal;
@@ -721,7 +726,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.a_sym = 1; P.b_sym = 1;
     P.has_in = 1;
     P.scale_kind = 0;
-    P.c_acc = hp->c; P.c_in = hp->b;
+    P.c_acc = co_c; P.c_in = co_b;
     { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
     if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
     ++launches;
@@ -743,7 +748,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.scale_kind = first_it ? 2 : 0;
     P.last = fuse ? 1 : 0;
     P.keep_o = (fuse && ctx->keep_o) ? 1 : 0;
-    P.c_acc = 1.f; P.c_in = hp->a;
+    P.c_acc = 1.f; P.c_in = co_a;
     { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, B.comb_acc_cols, ctx->max_clusters, stream); }
     if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
     ++launches;

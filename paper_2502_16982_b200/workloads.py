@@ -18,6 +18,10 @@ parameter sets of the paper's models; no dataset or trained weight is used):
      attention projections 2048x1536, 1536x3072, 2048x576, 512x4096,
      2048x2048; layer 0 dense MLP 2048x11264 (x2) and 11264x2048; layers 1-26
      66 experts x (2048x1408 x2, 1408x2048)
+  6  the five dense Llama-style models of the paper's scaling-law study
+     (hidden 1536 / 1792 / 2048 / 2304 / 2560 with 12 / 14 / 16 / 18 / 20
+     layers): per layer four H x H attention matrices and SwiGLU matrices
+     H x F (x2) and F x H with F = 2.6 H rounded to a multiple of 128
 """
 
 from __future__ import annotations
@@ -80,6 +84,15 @@ def config_groups(cfg: int, layers: Optional[int] = None) -> List[GroupSpec]:
         if moe_layers:
             out.append(GroupSpec(2048, 1408, 2 * 66 * moe_layers, bf, bf, lognormal_scale=True, name="expert_up_gate"))
             out.append(GroupSpec(1408, 2048, 1 * 66 * moe_layers, bf, bf, lognormal_scale=True, name="expert_down"))
+        return out
+    if cfg == 6:
+        out = []
+        for hidden, n_layers in ((1536, 12), (1792, 14), (2048, 16), (2304, 18), (2560, 20)):
+            L = n_layers if layers is None else layers
+            ffn = int(round(2.6 * hidden / 128.0)) * 128
+            out.append(GroupSpec(hidden, hidden, 4 * L, bf, bf, name="attn%d" % hidden))
+            out.append(GroupSpec(hidden, ffn, 2 * L, bf, bf, name="mlp_up_gate%d" % hidden))
+            out.append(GroupSpec(ffn, hidden, 1 * L, bf, bf, name="mlp_down%d" % hidden))
         return out
     raise ValueError("unknown config %r" % (cfg,))
 

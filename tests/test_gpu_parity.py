@@ -52,7 +52,8 @@ SCALE_MODES = {0: "adjusted_lr", 1: "fixed_dim", 2: "update_norm"}
 def to_orc(hp):
     return orc.Hyper(lr=hp.lr, wd=hp.wd, mu=hp.mu, nesterov=hp.nesterov, ns_steps=hp.ns_steps,
                      a=hp.a, b=hp.b, c=hp.c, eps=hp.eps, rms_scale=hp.rms_scale,
-                     scale_mode=SCALE_MODES[hp.scale_mode], scale_dim=hp.scale_dim)
+                     scale_mode=SCALE_MODES[hp.scale_mode], scale_dim=hp.scale_dim,
+                     coeffs=None if hp.coeffs is None else [tuple(t) for t in hp.coeffs])
 
 
 def bf16_ulp_ok_fraction(got_bf16, expect_f64, slack=0.0):
@@ -364,6 +365,20 @@ def test_update_scale_variants(mode, dim, wdt):
             assert all(abs(r - 0.2) < 1e-6 for r in case.ctx.muon_get_update_rms())
     finally:
         case.close()
+
+
+def test_coefficient_schedule():
+    """One (a, b, c) per Newton-Schulz step instead of a single triple."""
+    sched = [(3.4445, -4.7750, 2.0315), (3.0, -3.5, 1.2), (2.0, -1.5, 0.5)]
+    specs = [wl.GroupSpec(328, 200, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(192, 320, 2, torch.float32, torch.float32, 0.02, 1.0)]
+    case = Case(specs, seed=43)
+    try:
+        check_step(case, default_hp(lr=1e-2, ns_steps=3, coeffs=sched))
+    finally:
+        case.close()
+    with pytest.raises(_binding().MuonError):
+        default_hp(ns_steps=5, coeffs=sched).to_c()
 
 
 def test_fp32_master_weights_with_bf16_shadow():

@@ -56,6 +56,24 @@ def test_closed_form_chosen_singular_values(rows, cols, steps):
     assert np.max(np.abs(O - expect)) < 1e-10
 
 
+def test_closed_form_with_a_coefficient_schedule():
+    """One (a, b, c) per step: the singular values go through the composition
+    of the per-step scalar polynomials."""
+    rng = np.random.default_rng(77)
+    rows, cols, k = 10, 14, 10
+    U = householder_orthonormal(rng, rows, k)
+    V = householder_orthonormal(rng, cols, k)
+    s = rng.uniform(0.05, 2.0, size=k)
+    sched = [(3.4445, -4.7750, 2.0315), (3.0, -3.5, 1.2), (2.0, -1.5, 0.5)]
+    x = s / np.linalg.norm(s)
+    for (a, b, c) in sched:
+        x = a * x + b * x**3 + c * x**5
+    O = orc.newton_schulz(((U * s) @ V.T) / np.linalg.norm(s), 3, coeffs=sched)
+    assert np.max(np.abs(O - (U * x) @ V.T)) < 1e-10
+    with pytest.raises(ValueError):
+        orc.newton_schulz(np.eye(3), 2, coeffs=sched)
+
+
 def test_closed_form_full_step_matches_scaled_update():
     rng = np.random.default_rng(7)
     rows, cols = 10, 24
