@@ -29,11 +29,10 @@ cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, cons
                                  const __nv_bfloat16* x, long long x_stride, int ldx, int count, int m,
                                  int n, float neg_lr, float decay, bool w_fp32, cudaStream_t stream);
 cudaError_t launch_rms_finalise(const float* partials, int per_matrix, int count, float factor,
-                                const MatDesc* descs, float* rms, cudaStream_t stream);
-cudaError_t launch_rms_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
-                              long long x_stride, int ldx, int m, int n, int count, float factor,
-                              bool use_inv_norm, float rms_target, bool normalise, float* rms,
-                              float* factors, cudaStream_t stream);
+                                const MatDesc* descs, const MatScal* scal, bool use_inv_norm, float rms_target,
+                                bool normalise, float* rms, float* factors, cudaStream_t stream);
+cudaError_t launch_sumsq_x(const __nv_bfloat16* x, long long x_stride, int ldx, int m, int n, int count,
+                           int per_matrix, float* partials, cudaStream_t stream);
 cudaError_t stream_tma_configure();
 cudaError_t launch_momentum_tma(const StreamTmaParams& P, bool grad_fp32, int num_sms, cudaStream_t stream);
 cudaError_t gemm_configure();
@@ -760,10 +759,12 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     // TMA-unaddressable weights, normalised update), the separate update
     // W <- decay*W - lr*f*O from the stored O.
     float* rms = reinterpret_cast<float*>(ctx->ws + ctx->sizes.off_rms);
+    float* rms_partials = reinterpret_cast<float*>(ctx->ws + B.off_rms_partials);
+    const int per_matrix = static_cast<int>(B.comb_tiles.size()) * 8;
     if (hp->ns_steps > 0 && fused_update) {
       LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
-      ce = launch_rms_finalise(reinterpret_cast<const float*>(ctx->ws + B.off_rms_partials),
-                               static_cast<int>(B.comb_tiles.size()) * 8, count, factor, descs, rms, stream);
+      ce = launch_rms_finalise(rms_partials, per_matrix, count, factor, descs, scal, false, hp->rms_scale, false, rms,
+                               nullptr, stream);
       if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
       ++launches;
     } else {
@@ -771,11 +772,14 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
       const __nv_bfloat16* xo = reinterpret_cast<const __nv_bfloat16*>(ctx->ws + B.off_x[cur]);
       {
         LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
-        ce = launch_rms_from_x(descs, scal, xo, static_cast<long long>(B.x_stride), B.ldx, B.m, B.n, count,
-                               factor, hp->ns_steps == 0, hp->rms_scale, normalise, rms, factors, stream);
+        ce = launch_sumsq_x(xo, static_cast<long long>(B.x_stride), B.ldx, B.m, B.n, count, per_matrix, rms_partials,
+                            stream);
+        if (ce == cudaSuccess)
+          ce = launch_rms_finalise(rms_partials, per_matrix, count, factor, descs, scal, hp->ns_steps == 0,
+                                   hp->rms_scale, normalise, rms, factors, stream);
       }
       if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "rms kernel launch: %s", cudaGetErrorString(ce));
-      ++launches;
+      launches += 2;
       {
         LaunchTimer lt(ctx, stream, MUON_KERNEL_UPDATE);
         ce = launch_update_from_x(descs, scal, factors, xo, static_cast<long long>(B.x_stride), B.ldx, count,

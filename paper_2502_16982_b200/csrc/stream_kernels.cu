@@ -257,31 +257,68 @@ update_from_x_kernel(const MatDesc* __restrict__ descs, const MatScal* __restric
     tile[i][tx] = (xr < x_rows && xc < x_cols) ? __bfloat162float(xm[static_cast<long long>(xr) * ldx + xc]) : 0.f;
   }
   __syncthreads();
-#pragma unroll 4
-  for (int i = ty; i < 64; i += 4) {
-    const int r = r0 + i, c = c0 + tx;
+  // thread: 4 consecutive columns of rows (t / 16) + 16 p
+  const int c4 = (threadIdx.x & 15) * 4;
+  const bool vec_w = d.vec_ok && (d.w_shadow == nullptr || ((reinterpret_cast<uintptr_t>(d.w_shadow) & 7) == 0 && d.ld_ws % 4 == 0));
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    const int i = (threadIdx.x >> 4) + 16 * p;
+    const int r = r0 + i, c = c0 + c4;
     if (r >= d.rows || c >= d.cols) continue;
-    const float o = d.transposed ? tile[tx][i] : tile[i][tx];
+    float o[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o[e] = d.transposed ? tile[c4 + e][i] : tile[i][c4 + e];
     const long long off = static_cast<long long>(r) * d.ld_w + c;
+    const int nv = min(4, d.cols - c);
     if (kWFp32) {
       float* w = reinterpret_cast<float*>(d.w) + off;
-      const float nw = fmaf(decay, *w, f * o);
-      *w = nw;
-      if (d.w_shadow != nullptr)
-        reinterpret_cast<__nv_bfloat16*>(d.w_shadow)[static_cast<long long>(r) * d.ld_ws + c] = __float2bfloat16_rn(nw);
+      __nv_bfloat16* sh = d.w_shadow ? reinterpret_cast<__nv_bfloat16*>(d.w_shadow) + static_cast<long long>(r) * d.ld_ws + c
+                                     : nullptr;
+      if (vec_w && nv == 4) {
+        float4 w4 = *reinterpret_cast<const float4*>(w);
+        w4.x = fmaf(decay, w4.x, f * o[0]);
+        w4.y = fmaf(decay, w4.y, f * o[1]);
+        w4.z = fmaf(decay, w4.z, f * o[2]);
+        w4.w = fmaf(decay, w4.w, f * o[3]);
+        *reinterpret_cast<float4*>(w) = w4;
+        if (sh != nullptr) {
+          __nv_bfloat162 h0 = __floats2bfloat162_rn(w4.x, w4.y), h1 = __floats2bfloat162_rn(w4.z, w4.w);
+          *reinterpret_cast<uint2*>(sh) = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
+        }
+      } else {
+        for (int e = 0; e < nv; ++e) {
+          const float nw = fmaf(decay, w[e], f * o[e]);
+          w[e] = nw;
+          if (sh != nullptr) sh[e] = __float2bfloat16_rn(nw);
+        }
+      }
     } else {
       __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(d.w) + off;
-      *w = __float2bfloat16_rn(fmaf(decay, __bfloat162float(*w), f * o));
+      if (vec_w && nv == 4) {
+        const uint2 w2 = *reinterpret_cast<const uint2*>(w);
+        __nv_bfloat162 h0 = __floats2bfloat162_rn(fmaf(decay, __uint_as_float(w2.x << 16), f * o[0]),
+                                                  fmaf(decay, __uint_as_float(w2.x & 0xFFFF0000u), f * o[1]));
+        __nv_bfloat162 h1 = __floats2bfloat162_rn(fmaf(decay, __uint_as_float(w2.y << 16), f * o[2]),
+                                                  fmaf(decay, __uint_as_float(w2.y & 0xFFFF0000u), f * o[3]));
+        *reinterpret_cast<uint2*>(w) = make_uint2(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1));
+      } else {
+        for (int e = 0; e < nv; ++e) w[e] = __float2bfloat16_rn(fmaf(decay, __bfloat162float(w[e]), f * o[e]));
+      }
     }
   }
 }
 
-// Update RMS from the partial sums the last Newton-Schulz epilogue left:
-// rms = |factor| * sqrt(sum O^2 / (rows * cols)), one warp per matrix, fixed order.
+// Update RMS (Algorithm 1, returned value) from per-matrix partial sums of O^2,
+// one warp per matrix, fixed order: rms = |factor| * sqrt(sum / (rows * cols)).
+// The sums come from the last Newton-Schulz epilogue or from sumsq_x_kernel; in
+// the latter case (separate weight update) the kernel also leaves the factor
+// the update kernel multiplies O by: `factor` * sn, or rms_target / RMS(O) * sn
+// when the update is normalised (Sec. 3.1 "Update Norm"), with sn = 1/(||U||_F +
+// eps) when the stored O is the un-normalised bf16(U) (no iteration).
 __global__ void rms_finalise_kernel(const float* __restrict__ partials, int per_matrix, int count,
                                     float factor, const MatDesc* __restrict__ descs,
-                                    float* __restrict__ rms) {
-  // (fused path: the update factor is fixed by the shape, nothing else to derive)
+                                    const MatScal* __restrict__ scal, int use_inv_norm, float rms_target,
+                                    int normalise, float* __restrict__ rms, float* __restrict__ factors) {
   const int mat = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (mat >= count) return;
   const int lane = threadIdx.x & 31;
@@ -292,29 +329,45 @@ __global__ void rms_finalise_kernel(const float* __restrict__ partials, int per_
   for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
   if (lane == 0) {
     const MatDesc d = descs[mat];
-    rms[d.global_index] = fabsf(factor) * sqrtf(s / (static_cast<float>(d.rows) * static_cast<float>(d.cols)));
+    const float sn = use_inv_norm ? scal[mat].inv_norm : 1.0f;
+    const float o_rms = fabsf(sn) * sqrtf(s / (static_cast<float>(d.rows) * static_cast<float>(d.cols)));
+    if (normalise) {
+      rms[d.global_index] = o_rms > 0.f ? rms_target : 0.f;
+      if (factors != nullptr) factors[mat] = o_rms > 0.f ? sn * rms_target / o_rms : 0.f;
+    } else {
+      rms[d.global_index] = fabsf(factor) * o_rms;
+      if (factors != nullptr) factors[mat] = factor * sn;
+    }
   }
 }
 
-// Update RMS from a stored O (x, short side first, m x n): one CTA per matrix,
-// thread-strided sequential sums and a fixed reduction tree.  Also leaves the
-// per-matrix factor the separate update kernel multiplies O by:
-// `factor` * s, or rms_target / RMS(O) * s when the update is normalised
-// (Sec. 3.1 "Update Norm"); s = 1/(||U||_F + eps) when x is the un-normalised bf16(U).
+// Partial sums of squares of a stored O (x, short side first, m x n): CTA
+// (p, matrix) adds rows p, p + P, ... with 16-byte loads (rows of the workspace
+// are 128-byte aligned) and a fixed reduction tree.
 __global__ void __launch_bounds__(256)
-rms_from_x_kernel(const MatDesc* __restrict__ descs, const MatScal* __restrict__ scal,
-                  const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx, int m, int n,
-                  float factor, int use_inv_norm, float rms_target, int normalise,
-                  float* __restrict__ rms, float* __restrict__ factors) {
+sumsq_x_kernel(const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx, int m, int n,
+               float* __restrict__ partials) {
   __shared__ float warp_sums[8];
-  const int mat = blockIdx.x;
+  const int mat = blockIdx.y;
   const __nv_bfloat16* xm = x + mat * x_stride;
   float s = 0.f;
-  const long long total = static_cast<long long>(m) * n;
-  for (long long i = threadIdx.x; i < total; i += blockDim.x) {
-    const int r = static_cast<int>(i / n), c = static_cast<int>(i - static_cast<long long>(r) * n);
-    const float v = __bfloat162float(xm[static_cast<long long>(r) * ldx + c]);
-    s = fmaf(v, v, s);
+  const int n8 = n / 8;
+  for (int r = blockIdx.x; r < m; r += gridDim.x) {
+    const __nv_bfloat16* row = xm + static_cast<long long>(r) * ldx;
+    for (int c8 = threadIdx.x; c8 < n8; c8 += blockDim.x) {
+      const uint4 v = *reinterpret_cast<const uint4*>(row + c8 * 8);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xFFFF0000u);
+        s = fmaf(lo, lo, s);
+        s = fmaf(hi, hi, s);
+      }
+    }
+    for (int c = n8 * 8 + threadIdx.x; c < n; c += blockDim.x) {
+      const float v = __bfloat162float(row[c]);
+      s = fmaf(v, v, s);
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
@@ -323,37 +376,28 @@ rms_from_x_kernel(const MatDesc* __restrict__ descs, const MatScal* __restrict__
   if (threadIdx.x == 0) {
     float t = 0.f;
     for (int w = 0; w < 8; ++w) t += warp_sums[w];
-    const MatScal sc = scal[mat];
-    const float sn = use_inv_norm ? sc.inv_norm : 1.0f;
-    const float o_rms = fabsf(sn) * sqrtf(t / (static_cast<float>(m) * static_cast<float>(n)));
-    if (normalise) {
-      rms[descs[mat].global_index] = o_rms > 0.f ? rms_target : 0.f;
-      factors[mat] = o_rms > 0.f ? sn * rms_target / o_rms : 0.f;
-    } else {
-      rms[descs[mat].global_index] = fabsf(factor) * o_rms;
-      factors[mat] = factor * sn;
-    }
+    partials[static_cast<long long>(mat) * gridDim.x + blockIdx.x] = t;
   }
 }
 
 }  // namespace
 
 cudaError_t launch_rms_finalise(const float* partials, int per_matrix, int count, float factor,
-                                const MatDesc* descs, float* rms, cudaStream_t stream) {
+                                const MatDesc* descs, const MatScal* scal, bool use_inv_norm, float rms_target,
+                                bool normalise, float* rms, float* factors, cudaStream_t stream) {
   if (count == 0) return cudaSuccess;
   const int warps = 4;
-  rms_finalise_kernel<<<(count + warps - 1) / warps, warps * 32, 0, stream>>>(partials, per_matrix, count, factor,
-                                                                               descs, rms);
+  rms_finalise_kernel<<<(count + warps - 1) / warps, warps * 32, 0, stream>>>(
+      partials, per_matrix, count, factor, descs, scal, use_inv_norm ? 1 : 0, rms_target, normalise ? 1 : 0, rms,
+      factors);
   return cudaGetLastError();
 }
 
-cudaError_t launch_rms_from_x(const MatDesc* descs, const MatScal* scal, const __nv_bfloat16* x,
-                              long long x_stride, int ldx, int m, int n, int count, float factor,
-                              bool use_inv_norm, float rms_target, bool normalise, float* rms,
-                              float* factors, cudaStream_t stream) {
+cudaError_t launch_sumsq_x(const __nv_bfloat16* x, long long x_stride, int ldx, int m, int n, int count,
+                           int per_matrix, float* partials, cudaStream_t stream) {
   if (count == 0) return cudaSuccess;
-  rms_from_x_kernel<<<count, 256, 0, stream>>>(descs, scal, x, x_stride, ldx, m, n, factor, use_inv_norm ? 1 : 0,
-                                               rms_target, normalise ? 1 : 0, rms, factors);
+  sumsq_x_kernel<<<dim3(static_cast<unsigned>(per_matrix), static_cast<unsigned>(count)), 256, 0, stream>>>(
+      x, x_stride, ldx, m, n, partials);
   return cudaGetLastError();
 }
 
