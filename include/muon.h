@@ -261,6 +261,17 @@ int muon_debug_keep(muon_ctx* ctx, int keep);
 int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, size_t dst_bytes);
 
 /*
+ * Test probe for the device-side failure path.  Every wait in the kernels is
+ * bounded: when one expires the kernel records MUON_ERR_TIMEOUT in the status
+ * word, drains and returns instead of hanging.  This call enqueues a one-thread
+ * kernel that waits, for at most limit_ms (1..1000) milliseconds, on a barrier
+ * nothing arrives on, and reports the expiry the same way, naming
+ * `matrix_index`.  muon_status then returns MUON_ERR_TIMEOUT and the context
+ * remains usable.  Nothing faults or hangs.
+ */
+int muon_debug_wait_expiry(muon_ctx* ctx, void* stream, int matrix_index, unsigned limit_ms);
+
+/*
  * Test knob: upper bound, in bytes, on the Newton-Schulz operands (X, A, B) of
  * one bucket chunk; a bucket that needs more is processed in several chunks
  * that reuse the workspace.  Process-wide, read by muon_workspace_bytes and

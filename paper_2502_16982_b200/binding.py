@@ -32,7 +32,7 @@ MUON_SCALE_ADJUSTED_LR, MUON_SCALE_FIXED_DIM, MUON_SCALE_UPDATE_NORM = 0, 1, 2
 EXPORTED = [
     "muon_workspace_bytes", "muon_partition", "muon_init", "muon_step", "muon_step_host", "muon_status",
     "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
-    "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes",
+    "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes", "muon_debug_wait_expiry",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
     "muon_momentum_norm_static", "muon_adamw_step",
 ]
@@ -110,6 +110,7 @@ def lib():
     L.muon_momentum_norm_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64,
                                             C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
     L.muon_debug_set_chunk_bytes.argtypes = [C.c_size_t]
+    L.muon_debug_wait_expiry.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_uint]
     L.muon_adamw_step.argtypes = [C.POINTER(muon_adamw_tensor), C.c_int, C.POINTER(muon_adamw_hparams), C.c_int,
                                   C.c_void_p]
     for name in EXPORTED:
@@ -376,6 +377,11 @@ class MuonContext:
         out = (C.c_uint * n)()
         _check(lib().muon_debug_tmem_bases(self._ctx, out, n))
         return list(out)
+
+    def muon_debug_wait_expiry(self, matrix_index: int, limit_ms: int = 20, stream=None):
+        import torch
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        _check(lib().muon_debug_wait_expiry(self._ctx, C.c_void_p(s.cuda_stream), int(matrix_index), int(limit_ms)))
 
     def muon_debug_keep(self, keep: bool):
         _check(lib().muon_debug_keep(self._ctx, int(keep)))

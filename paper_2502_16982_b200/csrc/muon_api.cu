@@ -35,6 +35,8 @@ cudaError_t launch_sumsq_x(const __nv_bfloat16* x, long long x_stride, int ldx, 
                            int per_matrix, float* partials, cudaStream_t stream);
 cudaError_t stream_tma_configure();
 cudaError_t launch_momentum_tma(const StreamTmaParams& P, bool grad_fp32, int num_sms, cudaStream_t stream);
+cudaError_t launch_wait_expiry_probe(DevStatus* status, int matrix_index, unsigned long long limit_ns,
+                                     cudaStream_t stream);
 cudaError_t gemm_configure();
 cudaError_t gemm_max_clusters(int* out);
 cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream);
@@ -965,6 +967,16 @@ int muon_debug_tmem_bases(muon_ctx* ctx, unsigned* out_host, int n) {
   if (ce == cudaSuccess)
     ce = cudaMemcpy(out_host, ctx->ws + ctx->sizes.off_debug, n * sizeof(unsigned), cudaMemcpyDeviceToHost);
   if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "debug read: %s", cudaGetErrorString(ce));
+  return MUON_OK;
+}
+
+int muon_debug_wait_expiry(muon_ctx* ctx, void* stream_v, int matrix_index, unsigned limit_ms) {
+  if (!ctx || matrix_index < 0 || matrix_index >= ctx->total_mats || limit_ms == 0 || limit_ms > 1000)
+    return fail(MUON_ERR_INVALID_ARG, "bad arguments (limit_ms must be 1..1000)");
+  DevStatus* status = reinterpret_cast<DevStatus*>(ctx->ws + ctx->sizes.off_status);
+  cudaError_t ce = launch_wait_expiry_probe(status, matrix_index, static_cast<unsigned long long>(limit_ms) * 1000000ull,
+                                            static_cast<cudaStream_t>(stream_v));
+  if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "probe launch: %s", cudaGetErrorString(ce));
   return MUON_OK;
 }
 

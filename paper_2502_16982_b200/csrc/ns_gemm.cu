@@ -524,7 +524,30 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
   }
 }
 
+// Test probe for the bounded wait every kernel here relies on: one thread waits
+// on an mbarrier that nothing ever arrives on, with a short limit, and records
+// MUON_ERR_TIMEOUT exactly as the kernels do when a wait expires.  The wait
+// ends by itself; nothing faults or hangs.
+__global__ void wait_expiry_probe_kernel(DevStatus* status, int matrix_index, unsigned long long limit_ns) {
+  __shared__ unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+    if (!ptx::mbar_wait(ptx::smem_u32(&bar), 0u, &abort_flag, limit_ns)) {
+      if (atomicCAS(&status->code, 0, -6 /* MUON_ERR_TIMEOUT */) == 0) status->matrix = matrix_index;
+    }
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_wait_expiry_probe(DevStatus* status, int matrix_index, unsigned long long limit_ns,
+                                     cudaStream_t stream) {
+  wait_expiry_probe_kernel<<<1, 32, 0, stream>>>(status, matrix_index, limit_ns);
+  return cudaGetLastError();
+}
 
 cudaError_t gemm_configure() {
   cudaError_t e = cudaFuncSetAttribute(ns_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,

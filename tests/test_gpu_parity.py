@@ -551,6 +551,23 @@ def test_host_buffer_entry_point():
         ref.close()
 
 
+def test_expired_device_wait_is_reported_and_the_context_survives():
+    """Failure detection without a fault: a bounded wait that nothing satisfies
+    runs out after its limit, the status word carries MUON_ERR_TIMEOUT and the
+    matrix named, and the next step on the same context is correct."""
+    b = _binding()
+    sp = wl.GroupSpec(128, 256, 3, torch.float32, torch.float32, 0.02, 1.0)
+    case = Case([sp], seed=9)
+    try:
+        case.ctx.muon_debug_wait_expiry(2, limit_ms=20)
+        status, which = case.ctx.muon_status()
+        assert status == b.MUON_ERR_TIMEOUT and which == 2
+        assert case.ctx.muon_status()[0] == 0  # cleared by the read
+        check_step(case, default_hp())
+    finally:
+        case.close()
+
+
 def test_invalid_descriptors_are_rejected_on_the_host():
     b = _binding()
     W = torch.zeros(2, 64, 64, device="cuda")
