@@ -47,29 +47,35 @@ namespace muon {
 
 namespace {
 
-constexpr int kStages = 4;
+// Shared memory is split between the operand ring and the epilogue staging.
+// A product whose epilogue loads no input tile (the Gram product) does best
+// with a deeper ring (5 stages, 4 staging buffers per warp); the others with 4
+// stages and 6 buffers (measured on the expert bucket).
+constexpr int kMaxStages = 5;
+constexpr int kMaxSubs = 6;
 constexpr int kTileABytes = 128 * kBK * 2;   // 16 KiB: this CTA's 128 A rows
 constexpr int kTileBBytes = 128 * kBK * 2;   // 16 KiB: up to 128 B rows (half of N = 256)
 constexpr int kStageBytes = kTileABytes + kTileBBytes;
 constexpr int kEpiWarps = 4;
 constexpr int kSubBytes = 32 * 128;          // one warp's 32 rows x 64 bf16 columns
-constexpr int kSubsPerWarp = 6;              // staging buffers per epilogue warp
 constexpr int kNumAcc = 2;
 
 struct Barriers {
-  unsigned long long full[kStages];       // leader's copy is the live one
-  unsigned long long empty[kStages];
+  unsigned long long full[kMaxStages];    // leader's copy is the live one
+  unsigned long long empty[kMaxStages];
   unsigned long long acc_full[kNumAcc];
   unsigned long long acc_empty[kNumAcc];  // leader's copy is the live one
-  unsigned long long io_ready[kEpiWarps][kSubsPerWarp];  // ring entry filled / free to write
+  unsigned long long io_ready[kEpiWarps][kMaxSubs];  // ring entry filled / free to write
   uint32_t tmem_base;
   int abort_flag;
 };
 
 constexpr int kBarrierBytes = 512;
-constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kEpiWarps * kSubsPerWarp * kSubBytes + kBarrierBytes;
+constexpr int smem_bytes(int stages, int subs) {
+  return 1024 + stages * kStageBytes + kEpiWarps * subs * kSubBytes + kBarrierBytes;
+}
 static_assert(sizeof(Barriers) <= kBarrierBytes, "barrier block too large");
-static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared-memory limit");
+static_assert(smem_bytes(5, 4) <= 232448 && smem_bytes(4, 6) <= 232448, "exceeds the 227 KiB shared-memory limit");
 static_assert(kBK == 64, "the issuer loop issues four K = 16 steps per stage");
 
 __device__ __forceinline__ void report_timeout(const GemmParams& P, int mat) {
@@ -123,7 +129,8 @@ struct QuarterCursor {
 };
 
 // kAccCols: fp32 TMEM columns per accumulator stage = widest N (128 or 256).
-template <int kAccCols>
+// kStages: depth of the operand ring; kSubsPerWarp: staging buffers per epilogue warp.
+template <int kAccCols, int kStages, int kSubsPerWarp>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ns_gemm_kernel(const __grid_constant__ GemmParams P) {
   extern __shared__ uint8_t smem_raw[];
@@ -549,38 +556,20 @@ cudaError_t launch_wait_expiry_probe(DevStatus* status, int matrix_index, unsign
   return cudaGetLastError();
 }
 
-cudaError_t gemm_configure() {
-  cudaError_t e = cudaFuncSetAttribute(ns_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kSmemBytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(ns_gemm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+namespace {
+
+template <int kAccCols, int kStages, int kSubs>
+cudaError_t configure_one() {
+  return cudaFuncSetAttribute(ns_gemm_kernel<kAccCols, kStages, kSubs>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              smem_bytes(kStages, kSubs));
 }
 
-// Largest number of co-resident CTA pairs (one CTA per SM).
-cudaError_t gemm_max_clusters(int* out) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2, 1, 1);
-  cfg.blockDim = dim3(kGemmThreads, 1, 1);
-  cfg.dynamicSmemBytes = kSmemBytes;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = 2;
-  attr.val.clusterDim.y = 1;
-  attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  return cudaOccupancyMaxActiveClusters(out, ns_gemm_kernel<256>, &cfg);
-}
-
-// acc_cols: 128 when every tile of the launch is one column block wide, else 256.
-cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream) {
-  const long long total = static_cast<long long>(P.count) * P.tiles_per_matrix;
-  if (total <= 0) return cudaSuccess;
-  const unsigned clusters = static_cast<unsigned>(total < max_clusters ? total : max_clusters);
+template <int kAccCols, int kStages, int kSubs>
+cudaError_t launch_one(const GemmParams& P, unsigned clusters, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * clusters, 1, 1);
   cfg.blockDim = dim3(kGemmThreads, 1, 1);
-  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.dynamicSmemBytes = smem_bytes(kStages, kSubs);
   cfg.stream = stream;
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeClusterDimension;
@@ -589,8 +578,47 @@ cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, 
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  if (acc_cols == 128) return cudaLaunchKernelEx(&cfg, ns_gemm_kernel<128>, P);
-  return cudaLaunchKernelEx(&cfg, ns_gemm_kernel<256>, P);
+  return cudaLaunchKernelEx(&cfg, ns_gemm_kernel<kAccCols, kStages, kSubs>, P);
+}
+
+}  // namespace
+
+cudaError_t gemm_configure() {
+  cudaError_t e = configure_one<128, 4, 6>();
+  if (e == cudaSuccess) e = configure_one<256, 4, 6>();
+  if (e == cudaSuccess) e = configure_one<128, 5, 4>();
+  if (e == cudaSuccess) e = configure_one<256, 5, 4>();
+  return e;
+}
+
+// Largest number of co-resident CTA pairs (one CTA per SM).
+cudaError_t gemm_max_clusters(int* out) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2, 1, 1);
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem_bytes(4, 6);
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaOccupancyMaxActiveClusters(out, ns_gemm_kernel<256, 4, 6>, &cfg);
+}
+
+// acc_cols: 128 when every tile of the launch is one column block wide, else 256.
+cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream) {
+  const long long total = static_cast<long long>(P.count) * P.tiles_per_matrix;
+  if (total <= 0) return cudaSuccess;
+  const unsigned clusters = static_cast<unsigned>(total < max_clusters ? total : max_clusters);
+  const bool deep_ring = !P.has_in && !P.last;  // no epilogue input tiles: the Gram product
+  if (deep_ring) {
+    if (acc_cols == 128) return launch_one<128, 5, 4>(P, clusters, stream);
+    return launch_one<256, 5, 4>(P, clusters, stream);
+  }
+  if (acc_cols == 128) return launch_one<128, 4, 6>(P, clusters, stream);
+  return launch_one<256, 4, 6>(P, clusters, stream);
 }
 
 }  // namespace muon
