@@ -56,7 +56,7 @@ struct PairTile {
 };
 
 // Parameters of one launch of the Newton-Schulz GEMM kernel.  Each output
-// element is  scale * (c_acc * acc + c_in * in).
+// element is  scale * (c_acc * acc + c_in * in) + diag_add * [row == col].
 struct GemmParams {
   CUtensorMap map_a;      // operand A, K-major: box {64 K, 128 rows}, 128B swizzle
   CUtensorMap map_a64;    // operand A, MN-major (transposed read of a symmetric matrix stored
@@ -82,8 +82,9 @@ struct GemmParams {
   int has_in;      // the epilogue reads an input tile through map_in
   int scale_kind;  // 0: none, 1: s^2 of the matrix, 2: s
   int last;        // fused weight update: W is read, updated and written back
+  int last_has_x;  // last iteration: the a*X term is added in this epilogue (an X tile is loaded)
   int keep_o;      // last iteration: also store O through map_out (test tap)
-  float c_acc, c_in;
+  float c_acc, c_in, diag_add;
   float upd_scale, decay;
   const MatDesc* descs;
   const MatScal* scal;

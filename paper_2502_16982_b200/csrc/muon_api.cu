@@ -79,6 +79,7 @@ struct Bucket {
   int stream_tiles_tma;       // tiles per matrix of the TMA streaming kernel (64 x 64)
   bool fused_update;          // every W is bf16 and TMA-addressable: update W in the last epilogue
   bool stream_tma;            // every G and M is TMA-addressable: TMA-pipelined momentum kernel
+  bool fold_identity;         // keep B' = B + a*I so that the combine is the single product B' X
   // workspace offsets (bytes) of the chunk buffers
   size_t off_x[2], off_a, off_b, off_partials, off_scal, off_rms_partials, off_factors;
   // workspace offsets of the persistent per-bucket tables
@@ -250,6 +251,9 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     B.stream_tiles_generic = std::max(t1, t2);
     B.stream_tiles_tma = ceil_div(B.m, 64) * ceil_div(B.n, 64);
     B.stream_tiles = std::max(B.stream_tiles_generic, B.stream_tiles_tma);
+    // Folding a*X into the product rounds B_ii + a to bf16; that is the smaller
+    // error from 128 rows up and the larger one for tiny matrices.
+    B.fold_identity = B.m >= 128;
     const size_t per_mat = 2 * B.x_stride * 2 + 2 * B.a_stride * 2;
     size_t chunk = std::max<size_t>(1, g_chunk_bytes_max / per_mat);
     chunk = std::min<size_t>(chunk, B.mats.size());
@@ -712,7 +716,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.has_in = 0;
     P.scale_kind = first_it ? 1 : 0;
     P.last = 0; P.keep_o = 0;
-    P.c_acc = 1.f; P.c_in = 0.f;
+    P.c_acc = 1.f; P.c_in = 0.f; P.diag_add = 0.f; P.last_has_x = 0;
     { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
     if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
     ++launches;
@@ -728,6 +732,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.has_in = 1;
     P.scale_kind = 0;
     P.c_acc = co_c; P.c_in = co_b;
+    P.diag_add = B.fold_identity ? co_a : 0.f;
     { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
     if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
     ++launches;
@@ -745,11 +750,13 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.k = B.m;
     P.out_cols = B.n;
     P.symmetric = 0; P.a_sym = 1; P.b_sym = 0; P.b_mn_major = 1;
-    P.has_in = 1;
+    P.has_in = (fuse || !B.fold_identity) ? 1 : 0;
     P.scale_kind = first_it ? 2 : 0;
     P.last = fuse ? 1 : 0;
+    P.last_has_x = (fuse && !B.fold_identity) ? 1 : 0;
     P.keep_o = (fuse && ctx->keep_o) ? 1 : 0;
-    P.c_acc = 1.f; P.c_in = co_a;
+    P.c_acc = 1.f; P.c_in = B.fold_identity ? 0.f : co_a;
+    P.diag_add = 0.f;
     { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, B.comb_acc_cols, ctx->max_clusters, stream); }
     if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
     ++launches;

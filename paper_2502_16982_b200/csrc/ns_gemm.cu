@@ -31,7 +31,14 @@
 // diagonal as the transpose of its mirror image (an MN-major UMMA operand), so
 // both triangles are the same bits by construction.
 //
-// Last iteration (Sec. 2.2): the entry holds the W tile and the X tile,
+// The combine is a*X + B X.  For buckets whose short side is at least 128 the
+// polynomial's epilogue adds a to the diagonal of B in fp32 before the one bf16
+// rounding (B' = B + a*I), so that the combine is the single product B' X and
+// its epilogue loads no X tile; smaller matrices keep the a*X term in the
+// combine's epilogue (for them the rounding of B_ii + a is the larger error).
+//
+// Last iteration (Sec. 2.2): the entry holds the W tile (and the X tile when
+// a*X is added here),
 //   O = scale * (acc + a*X),   W <- (1 - lr*wd) * W - lr * rms_scale * sqrt(max(rows, cols)) * O
 // in fp32; O itself never reaches HBM.
 //
@@ -39,6 +46,8 @@
 // MUON_ERR_TIMEOUT, all roles drain, both CTAs meet at the final cluster
 // barrier, TMEM is freed and the kernel returns.
 #include <cuda_bf16.h>
+
+#include <type_traits>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -326,7 +335,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
     unsigned long long* my_bars = bars->io_ready[q];
     // Ring of staging entries: one buffer per quarter, or two (W and X) on the
     // last iteration.
-    const int bufs_per_q = P.last ? 2 : 1;
+    const int bufs_per_q = (P.last && (P.last_has_x || P.keep_o)) ? 2 : 1;
     const uint32_t ring_len = kSubsPerWarp / bufs_per_q;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -355,9 +364,9 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         ptx::mbar_arrive(bar);
       } else if (P.last) {
         const bool tr = P.descs[pre.mat].transposed != 0;
-        ptx::mbar_arrive_expect_tx(bar, 2 * kSubBytes);
+        ptx::mbar_arrive_expect_tx(bar, P.last_has_x ? 2 * kSubBytes : kSubBytes);
         ptx::tma_load_3d(buf, P.wmaps + pre.mat, tr ? row0 : col0, tr ? col0 : row0, 0, bar);
-        ptx::tma_load_3d(buf + kSubBytes, &P.map_in, col0, row0, pre.mat, bar);
+        if (P.last_has_x) ptx::tma_load_3d(buf + kSubBytes, &P.map_in, col0, row0, pre.mat, bar);
         ++loads_in_flight;
       } else if (P.has_in) {
         ptx::mbar_arrive_expect_tx(bar, kSubBytes);
@@ -403,6 +412,9 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           const uint32_t buf = my_base + e * bufs_per_q * kSubBytes;  // in / out (W on the last iteration)
           const uint32_t buf2 = buf + kSubBytes;                        // X tile on the last iteration
           const int col0 = cur.jb * 128 + qd * 64;
+          // column of this lane's row that lies on the matrix diagonal, if the quarter holds it
+          const bool diag_quarter = P.diag_add != 0.f && cur.jb + (qd >> 1) == cur.ib;
+          const int dcol = q * 32 + lane - (qd & 1) * 64;
 
           uint32_t v[64];
           ptx::tmem_ld_32x64(taddr + qd * 64, v);
@@ -415,24 +427,32 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           }
 
           if (!P.last) {
+            // the diagonal add touches one element per row of a diagonal block's
+            // quarter; the warp-uniform branch keeps it out of every other quarter
+            auto combine = [&](auto with_diag) {
 #pragma unroll
-            for (int c8 = 0; c8 < 8; ++c8) {
-              const uint32_t swz = static_cast<uint32_t>(lane * 128 + ((c8 ^ (lane & 7)) << 4));
-              float in[8];
-              if (P.has_in) {
-                uint32_t w0, w1, w2, w3;
-                lds128(buf + swz, w0, w1, w2, w3);
-                unpack8(w0, w1, w2, w3, in);
-              } else {
+              for (int c8 = 0; c8 < 8; ++c8) {
+                const uint32_t swz = static_cast<uint32_t>(lane * 128 + ((c8 ^ (lane & 7)) << 4));
+                float in[8];
+                if (P.has_in) {
+                  uint32_t w0, w1, w2, w3;
+                  lds128(buf + swz, w0, w1, w2, w3);
+                  unpack8(w0, w1, w2, w3, in);
+                } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) in[i] = 0.f;
+                  for (int i = 0; i < 8; ++i) in[i] = 0.f;
+                }
+                float o[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  o[i] = scale * fmaf(P.c_acc, __uint_as_float(v[c8 * 8 + i]), P.c_in * in[i]);
+                  if (decltype(with_diag)::value && c8 * 8 + i == dcol) o[i] += P.diag_add;
+                }
+                sts128(buf + swz, pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
               }
-              float o[8];
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                o[i] = scale * fmaf(P.c_acc, __uint_as_float(v[c8 * 8 + i]), P.c_in * in[i]);
-              sts128(buf + swz, pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
-            }
+            };
+            if (diag_quarter) combine(std::true_type{});
+            else combine(std::false_type{});
           } else {
             // O = scale * (acc + c_in * X);  W <- decay * W + upd_scale * O
             __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(my_ptr + e * bufs_per_q * kSubBytes);
@@ -441,8 +461,13 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
               const uint32_t swz = static_cast<uint32_t>(lane * 128 + ((c8 ^ (lane & 7)) << 4));
               uint32_t w0, w1, w2, w3;
               float x[8], o[8];
-              lds128(buf2 + swz, w0, w1, w2, w3);
-              unpack8(w0, w1, w2, w3, x);
+              if (P.last_has_x) {
+                lds128(buf2 + swz, w0, w1, w2, w3);
+                unpack8(w0, w1, w2, w3, x);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) x[i] = 0.f;
+              }
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 o[i] = scale * fmaf(P.c_acc, __uint_as_float(v[c8 * 8 + i]), P.c_in * x[i]);
