@@ -252,7 +252,7 @@ int muon_profile_read(muon_ctx* ctx, double* ms_by_kernel, int* launches_by_kern
  * NOT yet divided by the norm; valid while ns_steps <= 1), MUON_TAP_A,
  * MUON_TAP_B (last iteration; the kernels keep only the 128x128 blocks on or
  * above the diagonal of these symmetric matrices, the tap fills in the rest by
- * symmetry; when min(rows, cols) >= 128 the stored matrix is B + a*I, B of Eq.
+ * symmetry; when min(rows, cols) >= 16 the stored matrix is B + a*I, B of Eq.
  * 2's factorisation with the coefficient a added on the diagonal, so that
  * a*X + B X is the single product (B + a*I) X) or MUON_TAP_X (last iteration's X).  Only valid for a context with
  * a single shape bucket that fits one chunk (buckets share the chunk buffers).

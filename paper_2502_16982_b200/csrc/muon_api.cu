@@ -252,8 +252,8 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     B.stream_tiles_tma = ceil_div(B.m, 64) * ceil_div(B.n, 64);
     B.stream_tiles = std::max(B.stream_tiles_generic, B.stream_tiles_tma);
     // Folding a*X into the product rounds B_ii + a to bf16; that is the smaller
-    // error from 128 rows up and the larger one for tiny matrices.
-    B.fold_identity = B.m >= 128;
+    // error from 16 rows up (measured with a bf16 storage model) and the larger one below.
+    B.fold_identity = B.m >= 16;
     const size_t per_mat = 2 * B.x_stride * 2 + 2 * B.a_stride * 2;
     size_t chunk = std::max<size_t>(1, g_chunk_bytes_max / per_mat);
     chunk = std::min<size_t>(chunk, B.mats.size());

@@ -31,7 +31,7 @@
 // diagonal as the transpose of its mirror image (an MN-major UMMA operand), so
 // both triangles are the same bits by construction.
 //
-// The combine is a*X + B X.  For buckets whose short side is at least 128 the
+// The combine is a*X + B X.  For buckets whose short side is at least 16 the
 // polynomial's epilogue adds a to the diagonal of B in fp32 before the one bf16
 // rounding (B' = B + a*I), so that the combine is the single product B' X and
 // its epilogue loads no X tile; smaller matrices keep the a*X term in the

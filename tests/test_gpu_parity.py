@@ -146,10 +146,10 @@ def test_config1_full_step():
 
 
 @pytest.mark.parametrize("wdt", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("rows,cols", [(128, 256), (256, 128), (320, 704), (576, 200), (64, 96), (120, 72)])
+@pytest.mark.parametrize("rows,cols", [(128, 256), (256, 128), (320, 704), (576, 200), (64, 96), (120, 72), (12, 40)])
 def test_stagewise_one_iteration(rows, cols, wdt):
     """X0, A, B, X of a single Newton-Schulz iteration against the oracle's.
-    From 128 rows (short side) up the kernels keep B + a*I instead of B."""
+    From 16 rows (short side) up the kernels keep B + a*I instead of B."""
     sp = wl.GroupSpec(rows, cols, 2, wdt, torch.float32, 0.02, 1.0)
     case = Case([sp], seed=42)
     try:
@@ -171,7 +171,7 @@ def test_stagewise_one_iteration(rows, cols, wdt):
             b_gpu = f64(case.ctx.muon_debug_read(i, b.MUON_TAP_B, m, m))
             x_gpu = f64(case.ctx.muon_debug_read(i, b.MUON_TAP_X, m, n))
             assert rel(a_gpu, A) <= TOL_NS, rel(a_gpu, A)
-            if m >= 128:
+            if m >= 16:
                 # off the diagonal it is B; on it, B_ii + a rounded once to bf16
                 off = ~np.eye(m, dtype=bool)
                 assert rel(b_gpu[off], B[off]) <= TOL_NS, rel(b_gpu[off], B[off])
