@@ -246,7 +246,8 @@ int muon_profile_read(muon_ctx* ctx, double* ms_by_kernel, int* launches_by_kern
 
 /*
  * Test taps.  muon_debug_keep(ctx, 1) makes the last Newton-Schulz iteration
- * also store its X (= O) in the workspace.  muon_debug_read copies one stage
+ * store its X (= O) in the workspace; the weights are then updated by the
+ * separate update kernel instead of the last epilogue.  muon_debug_read copies one stage
  * of one matrix to a HOST buffer as dense bf16, short side first (m x n with
  * m = min(rows, cols); m x m for A and B): `which` is MUON_TAP_X0 (bf16(U),
  * NOT yet divided by the norm; valid while ns_steps <= 1), MUON_TAP_A,

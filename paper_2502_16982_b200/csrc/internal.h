@@ -65,13 +65,16 @@ struct GemmParams {
                           // MN-major: {N, K})
   CUtensorMap map_in;     // epilogue input, box {64, 32}, 128B swizzle
   CUtensorMap map_out;    // output (and the O tap of the last iteration), box {64, 32}, 128B swizzle
-  const CUtensorMap* wmaps;  // last iteration: one map per matrix over its W (chunk-relative);
-                             // box {64, 32} swizzled, or {32, 64} plain when rows > cols
+  const CUtensorMap* wmaps;  // last iteration: one map per matrix over its W (chunk-relative),
+                             // box {64, 32}, 128B swizzle
   const PairTile* tiles;  // tile table of one matrix
+  const PairTile* tiles_t;  // last iteration: table of a matrix stored with rows > cols, whose
+                            // product is formed transposed (row pairs along the long side)
   int tiles_per_matrix;
   int count;       // matrices in this launch
   int k;           // contraction length
   int m;           // output rows per matrix (short side of the bucket)
+  int n_long;      // long side of the bucket (output rows of a transposed-formulation tile)
   int out_cols;    // output columns per matrix
   int symmetric;   // the output is symmetric: only blocks on or above the diagonal are
                    // computed and stored
@@ -82,8 +85,6 @@ struct GemmParams {
   int has_in;      // the epilogue reads an input tile through map_in
   int scale_kind;  // 0: none, 1: s^2 of the matrix, 2: s
   int last;        // fused weight update: W is read, updated and written back
-  int last_has_x;  // last iteration: the a*X term is added in this epilogue (an X tile is loaded)
-  int keep_o;      // last iteration: also store O through map_out (test tap)
   float c_acc, c_in, diag_add;
   float upd_scale, decay;
   const MatDesc* descs;

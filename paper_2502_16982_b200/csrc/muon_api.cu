@@ -83,8 +83,9 @@ struct Bucket {
   // workspace offsets (bytes) of the chunk buffers
   size_t off_x[2], off_a, off_b, off_partials, off_scal, off_rms_partials, off_factors;
   // workspace offsets of the persistent per-bucket tables
-  size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_comb_tiles;
+  size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_comb_tiles, off_comb_tiles_t;
   std::vector<PairTile> sym_tiles, comb_tiles;  // tile tables of one matrix
+  std::vector<PairTile> comb_tiles_t;           // combine formed transposed: row pairs along the long side
   int sym_acc_cols, comb_acc_cols;              // widest tile of each table (128 or 256)
   // tensor maps over the chunk buffers (all 128-byte swizzled)
   CUtensorMap x_op[2];   // X as K-major operand A: box {64,128}
@@ -158,11 +159,10 @@ int encode_stream_map(CUtensorMap* out, const void* base, int rows, int cols, lo
 }
 
 // Map over one caller-owned bf16 weight matrix [rows][cols] with row pitch ld.
-// rows <= cols: the tile of the Newton-Schulz orientation, box {64, 32} swizzled;
-// rows > cols: W is the transpose of that orientation, box {32, 64} plain.
+// The last epilogue produces its tiles in W's own orientation, so one box shape
+// serves both orientations: {64, 32}, 128-byte swizzle.
 int encode_w_map(CUtensorMap* out, void* w, int rows, int cols, long long ld) {
-  if (rows <= cols) return encode_map(out, w, cols, rows, 1, static_cast<int>(ld), static_cast<size_t>(rows) * ld, 64, 32, true);
-  return encode_map(out, w, cols, rows, 1, static_cast<int>(ld), static_cast<size_t>(rows) * ld, 32, 64, false);
+  return encode_map(out, w, cols, rows, 1, static_cast<int>(ld), static_cast<size_t>(rows) * ld, 64, 32, true);
 }
 
 int validate_groups(const muon_group* groups, int n_groups, bool need_ptrs) {
@@ -318,6 +318,17 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     off = align_up(off + B.sym_tiles.size() * sizeof(PairTile), 1024);
     B.off_comb_tiles = off;
     off = align_up(off + B.comb_tiles.size() * sizeof(PairTile), 1024);
+    // the same product with the roles of the sides exchanged (as many tiles)
+    B.comb_tiles_t.clear();
+    for (int p = 0; p < ceil_div(ncb, 2); ++p) {
+      for (int jb = 0; jb < nb;) {
+        const int w = std::min(2, nb - jb);
+        B.comb_tiles_t.push_back(PairTile{static_cast<short>(p), static_cast<short>(jb), static_cast<short>(w), 0});
+        jb += w;
+      }
+    }
+    B.off_comb_tiles_t = off;
+    off = align_up(off + B.comb_tiles_t.size() * sizeof(PairTile), 1024);
   }
   sizes->off_debug = off;
   off = align_up(off + 1024 * sizeof(unsigned), 1024);
@@ -560,6 +571,9 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     if (ce == cudaSuccess)
       ce = cudaMemcpy(ctx->ws + B.off_comb_tiles, B.comb_tiles.data(), B.comb_tiles.size() * sizeof(PairTile),
                       cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess)
+      ce = cudaMemcpy(ctx->ws + B.off_comb_tiles_t, B.comb_tiles_t.data(), B.comb_tiles_t.size() * sizeof(PairTile),
+                      cudaMemcpyHostToDevice);
     if (ce == cudaSuccess && B.fused_update) {
       std::vector<CUtensorMap> wmaps(B.mats.size());
       for (size_t i = 0; i < B.mats.size() && rc == MUON_OK; ++i)
@@ -639,7 +653,10 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
   const float factor = hp->rms_scale * std::sqrt(hp->scale_mode == MUON_SCALE_FIXED_DIM
                                                      ? hp->scale_dim : static_cast<float>(B.n));
   const bool normalise = hp->scale_mode == MUON_SCALE_UPDATE_NORM;
-  const bool fused_update = B.fused_update && !normalise;
+  // The last epilogue updates W when every W of the bucket is TMA-addressable
+  // bf16, the update needs no whole-matrix statistic, a*X is folded into the
+  // product and the O tap is off; otherwise O is stored and a second pass applies it.
+  const bool fused_update = B.fused_update && !normalise && B.fold_identity && !ctx->keep_o;
   const float upd_scale = -hp->lr * factor;
   const float decay = 1.0f - hp->lr * hp->wd;
   const MatDesc* descs = reinterpret_cast<const MatDesc*>(ctx->ws + B.off_descs) + first;
@@ -699,6 +716,8 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.wmaps = reinterpret_cast<const CUtensorMap*>(ctx->ws + B.off_wmaps) + first;
     P.count = count;
     P.m = B.m;
+    P.n_long = B.n;
+    P.tiles_t = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles_t);
     P.upd_scale = upd_scale;
     P.decay = decay;
 
@@ -715,8 +734,8 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.symmetric = 1; P.a_sym = 0; P.b_sym = 0; P.b_mn_major = 0;
     P.has_in = 0;
     P.scale_kind = first_it ? 1 : 0;
-    P.last = 0; P.keep_o = 0;
-    P.c_acc = 1.f; P.c_in = 0.f; P.diag_add = 0.f; P.last_has_x = 0;
+    P.last = 0;
+    P.c_acc = 1.f; P.c_in = 0.f; P.diag_add = 0.f;
     { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
     if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
     ++launches;
@@ -750,11 +769,9 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.k = B.m;
     P.out_cols = B.n;
     P.symmetric = 0; P.a_sym = 1; P.b_sym = 0; P.b_mn_major = 1;
-    P.has_in = (fuse || !B.fold_identity) ? 1 : 0;
+    P.has_in = (fuse || !B.fold_identity) ? 1 : 0;  // W when fused, else X for the a*X term
     P.scale_kind = first_it ? 2 : 0;
     P.last = fuse ? 1 : 0;
-    P.last_has_x = (fuse && !B.fold_identity) ? 1 : 0;
-    P.keep_o = (fuse && ctx->keep_o) ? 1 : 0;
     P.c_acc = 1.f; P.c_in = B.fold_identity ? 0.f : co_a;
     P.diag_add = 0.f;
     { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, B.comb_acc_cols, ctx->max_clusters, stream); }

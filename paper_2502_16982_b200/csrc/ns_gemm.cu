@@ -37,10 +37,14 @@
 // its epilogue loads no X tile; smaller matrices keep the a*X term in the
 // combine's epilogue (for them the rounding of B_ii + a is the larger error).
 //
-// Last iteration (Sec. 2.2): the entry holds the W tile (and the X tile when
-// a*X is added here),
-//   O = scale * (acc + a*X),   W <- (1 - lr*wd) * W - lr * rms_scale * sqrt(max(rows, cols)) * O
-// in fp32; O itself never reaches HBM.
+// Last iteration (Sec. 2.2): the entry holds the W tile,
+//   O = scale * acc,   W <- (1 - lr*wd) * W - lr * rms_scale * sqrt(max(rows, cols)) * O
+// in fp32; O itself never reaches HBM.  For a matrix stored with rows > cols
+// (Newton-Schulz ran on its transpose) the last product is formed transposed,
+// O^T = X^T B' with X^T read as an MN-major operand from X and the symmetric B'
+// as the other operand, so that the tile comes out in W's own orientation and
+// no transposition is needed; such tiles follow a second tile table (row pairs
+// along the long side).
 //
 // Every software wait is bounded (ptx::mbar_wait); on expiry the CTA records
 // MUON_ERR_TIMEOUT, all roles drain, both CTAs meet at the final cluster
@@ -118,24 +122,56 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t w0, uint32_t w1, 
 struct QuarterCursor {
   int tile, mat, qd, q_end;
   int ib, jb;
+  int row_limit;  // output rows of the matrix in this tile's orientation
 
   // Quarter range of tile `t` for CTA `rank`; returns false past the last tile.
   __device__ __forceinline__ bool open_tile(const GemmParams& P, int t, int total_tiles, int rank) {
     tile = t;
     if (t >= total_tiles) return false;
     mat = t / P.tiles_per_matrix;
-    const PairTile pt = P.tiles[t - mat * P.tiles_per_matrix];
+    const bool swapped = P.last && P.descs[mat].transposed != 0;
+    const PairTile pt = (swapped ? P.tiles_t : P.tiles)[t - mat * P.tiles_per_matrix];
+    row_limit = swapped ? P.n_long : P.m;
+    const int col_limit = swapped ? P.m : P.out_cols;
     ib = 2 * pt.p + rank;
     jb = pt.jb;
-    const int cols_left = P.out_cols - jb * 128;
+    const int cols_left = col_limit - jb * 128;
     q_end = min(2 * pt.nbw, (cols_left + 63) / 64);
     qd = 0;
-    if (ib * 128 >= P.m) qd = q_end;                     // ragged pair: nothing of ours
+    if (ib * 128 >= row_limit) qd = q_end;               // ragged pair: nothing of ours
     else if (P.symmetric && jb < ib) qd = min(2, q_end);  // below-diagonal block: dropped
     return true;
   }
   __device__ __forceinline__ bool has_quarter() const { return qd < q_end; }
 };
+
+// What one tile of the launch computes: its table entry, whether it is a
+// transposed-formulation tile of the last iteration, and up to which K block
+// each operand is read transposed (MN-major).
+struct TilePlan {
+  PairTile pt;
+  bool swapped;
+  int kb_a, kb_b;  // K blocks [0, kb_a) of A and [0, kb_b) of B are read MN-major
+};
+
+__device__ __forceinline__ TilePlan plan_tile(const GemmParams& P, int tile, int num_kb) {
+  TilePlan t;
+  const int mat = tile / P.tiles_per_matrix;
+  const int idx = tile - mat * P.tiles_per_matrix;
+  t.swapped = P.last && P.descs[mat].transposed != 0;
+  t.pt = (t.swapped ? P.tiles_t : P.tiles)[idx];
+  // a symmetric operand kept as its upper blocks is read transposed up to the
+  // block where some row of the operand tile is still below the diagonal
+  const int sym_b = min(num_kb, 2 * (t.pt.nbw == 2 ? t.pt.jb + 1 : t.pt.jb));
+  if (t.swapped) {  // A = X^T from X (MN-major throughout), B = the symmetric matrix
+    t.kb_a = num_kb;
+    t.kb_b = sym_b;
+  } else {
+    t.kb_a = P.a_sym ? min(num_kb, 2 * (2 * t.pt.p + 1)) : 0;
+    t.kb_b = P.b_mn_major ? num_kb : (P.b_sym ? sym_b : 0);
+  }
+  return t;
+}
 
 // kAccCols: fp32 TMEM columns per accumulator stage = widest N (128 or 256).
 // kStages: depth of the operand ring; kSubsPerWarp: staging buffers per epilogue warp.
@@ -200,15 +236,16 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       const uint32_t leader_full0 = ptx::map_to_cta(full0, 0);  // the rank lives in the upper address bits
       for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
         const int mat = tile / P.tiles_per_matrix;
-        const PairTile pt = P.tiles[tile - mat * P.tiles_per_matrix];
+        const TilePlan tp = plan_tile(P, tile, num_kb);
+        const PairTile pt = tp.pt;
         const int row0 = (2 * pt.p + static_cast<int>(rank)) * 128;
         const int half = 64 * pt.nbw;  // B rows (N columns) staged by each CTA
         const int b0 = pt.jb * 128 + static_cast<int>(rank) * half;
         const uint32_t stage_tx = 2u * static_cast<uint32_t>(kTileABytes + half * 128);
-        // K blocks [0, kb_a) of A and [0, kb_b) of B are read transposed
-        const int kb_a = P.a_sym ? min(num_kb, 2 * (2 * pt.p + 1)) : 0;
-        const int kb_b = P.b_mn_major ? num_kb
-                                      : (P.b_sym ? min(num_kb, 2 * (pt.nbw == 2 ? pt.jb + 1 : pt.jb)) : 0);
+        const int kb_a = tp.kb_a, kb_b = tp.kb_b;
+        // a transposed-formulation tile takes its operands from the other two 64 x 64 maps
+        const CUtensorMap* map_a64 = tp.swapped ? &P.map_b : &P.map_a64;
+        const CUtensorMap* map_b = tp.swapped ? &P.map_a64 : &P.map_b;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = ptx::mbar_wait(empty0 + stage * 8, phase ^ 1u, abort_flag);
           ok = __all_sync(0xFFFFFFFFu, ok);
@@ -225,15 +262,15 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
             if (kb >= kb_a) {
               ptx::tma_load_3d_pair(sa, &P.map_a, k0, row0, mat, leader_full);
             } else {
-              ptx::tma_load_3d_pair(sa, &P.map_a64, row0, k0, mat, leader_full);
-              ptx::tma_load_3d_pair(sa + 8192, &P.map_a64, row0 + 64, k0, mat, leader_full);
+              ptx::tma_load_3d_pair(sa, map_a64, row0, k0, mat, leader_full);
+              ptx::tma_load_3d_pair(sa + 8192, map_a64, row0 + 64, k0, mat, leader_full);
             }
             if (kb >= kb_b) {
-              ptx::tma_load_3d_pair(sb, &P.map_b, k0, b0, mat, leader_full);
-              if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, &P.map_b, k0, b0 + 64, mat, leader_full);
+              ptx::tma_load_3d_pair(sb, map_b, k0, b0, mat, leader_full);
+              if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, map_b, k0, b0 + 64, mat, leader_full);
             } else {
-              ptx::tma_load_3d_pair(sb, &P.map_b, b0, k0, mat, leader_full);
-              if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, &P.map_b, b0 + 64, k0, mat, leader_full);
+              ptx::tma_load_3d_pair(sb, map_b, b0, k0, mat, leader_full);
+              if (pt.nbw == 2) ptx::tma_load_3d_pair(sb + 8192, map_b, b0 + 64, k0, mat, leader_full);
             }
           }
           __syncwarp();
@@ -268,10 +305,9 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       constexpr uint32_t kLboMN = (8192u >> 4) << 16;   // MN-major: LBO 8192 (next 64-element chunk)
       for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
         const int mat = tile / P.tiles_per_matrix;
-        const PairTile pt = P.tiles[tile - mat * P.tiles_per_matrix];
-        const int kb_a = P.a_sym ? min(num_kb, 2 * (2 * pt.p + 1)) : 0;
-        const int kb_b = P.b_mn_major ? num_kb
-                                      : (P.b_sym ? min(num_kb, 2 * (pt.nbw == 2 ? pt.jb + 1 : pt.jb)) : 0);
+        const TilePlan tp = plan_tile(P, tile, num_kb);
+        const PairTile pt = tp.pt;
+        const int kb_a = tp.kb_a, kb_b = tp.kb_b;
         ok = ptx::mbar_wait(ptx::smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) {
@@ -331,12 +367,9 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
     // ----------------------------------------------------------- epilogue ----
     const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the tile
     const uint32_t my_base = ptx::smem_u32(s_epi + q * kSubsPerWarp * kSubBytes);
-    uint8_t* my_ptr = s_epi + q * kSubsPerWarp * kSubBytes;
     unsigned long long* my_bars = bars->io_ready[q];
-    // Ring of staging entries: one buffer per quarter, or two (W and X) on the
-    // last iteration.
-    const int bufs_per_q = (P.last && (P.last_has_x || P.keep_o)) ? 2 : 1;
-    const uint32_t ring_len = kSubsPerWarp / bufs_per_q;
+    // Ring of staging entries, one buffer per quarter.
+    constexpr uint32_t ring_len = kSubsPerWarp;
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t gq = 0;  // quarters processed so far by this warp
@@ -357,16 +390,15 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       if (!pre_valid) return;
       const uint32_t e = pre_g % ring_len;
       const uint32_t bar = ptx::smem_u32(&my_bars[e]);
-      const uint32_t buf = my_base + e * bufs_per_q * kSubBytes;
+      const uint32_t buf = my_base + e * kSubBytes;
       const int row0 = pre.ib * 128 + q * 32;
       const int col0 = pre.jb * 128 + pre.qd * 64;
-      if (row0 >= P.m) {  // this warp's rows lie beyond the matrix: nothing to fetch
+      if (row0 >= pre.row_limit) {  // this warp's rows lie beyond the matrix: nothing to fetch
         ptx::mbar_arrive(bar);
       } else if (P.last) {
-        const bool tr = P.descs[pre.mat].transposed != 0;
-        ptx::mbar_arrive_expect_tx(bar, P.last_has_x ? 2 * kSubBytes : kSubBytes);
-        ptx::tma_load_3d(buf, P.wmaps + pre.mat, tr ? row0 : col0, tr ? col0 : row0, 0, bar);
-        if (P.last_has_x) ptx::tma_load_3d(buf + kSubBytes, &P.map_in, col0, row0, pre.mat, bar);
+        // the tile is in W's own orientation (see the header): W[row0.., col0..]
+        ptx::mbar_arrive_expect_tx(bar, kSubBytes);
+        ptx::tma_load_3d(buf, P.wmaps + pre.mat, col0, row0, 0, bar);
         ++loads_in_flight;
       } else if (P.has_in) {
         ptx::mbar_arrive_expect_tx(bar, kSubBytes);
@@ -399,18 +431,15 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       ptx::tc_fence_after();
       float o_sq = 0.f;  // last iteration: this lane's sum of O^2 over the tile
       if (cur.has_quarter()) {
-        const MatDesc md = P.descs[mat];
         const MatScal sc = P.scal[mat];
         const float scale = P.scale_kind == 1 ? sc.inv_norm_sq : (P.scale_kind == 2 ? sc.inv_norm : 1.0f);
-        const bool w_transposed = P.last && md.transposed;
         const int row0 = cur.ib * 128 + q * 32;  // first of this warp's rows
         const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * kAccCols) +
                                (static_cast<uint32_t>(q * 32) << 16);
 
         for (int qd = cur.qd; qd < cur.q_end && ok; ++qd, ++gq) {
           const uint32_t e = gq % ring_len;
-          const uint32_t buf = my_base + e * bufs_per_q * kSubBytes;  // in / out (W on the last iteration)
-          const uint32_t buf2 = buf + kSubBytes;                        // X tile on the last iteration
+          const uint32_t buf = my_base + e * kSubBytes;  // in / out (W on the last iteration)
           const int col0 = cur.jb * 128 + qd * 64;
           // column of this lane's row that lies on the matrix diagonal, if the quarter holds it
           const bool diag_quarter = P.diag_add != 0.f && cur.jb + (qd >> 1) == cur.ib;
@@ -454,70 +483,43 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
             if (diag_quarter) combine(std::true_type{});
             else combine(std::false_type{});
           } else {
-            // O = scale * (acc + c_in * X);  W <- decay * W + upd_scale * O
-            __nv_bfloat16* wt = reinterpret_cast<__nv_bfloat16*>(my_ptr + e * bufs_per_q * kSubBytes);
+            // O = scale * acc;  W <- decay * W + upd_scale * O
 #pragma unroll
             for (int c8 = 0; c8 < 8; ++c8) {
               const uint32_t swz = static_cast<uint32_t>(lane * 128 + ((c8 ^ (lane & 7)) << 4));
               uint32_t w0, w1, w2, w3;
-              float x[8], o[8];
-              if (P.last_has_x) {
-                lds128(buf2 + swz, w0, w1, w2, w3);
-                unpack8(w0, w1, w2, w3, x);
-              } else {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) x[i] = 0.f;
-              }
+              float w[8];
+              lds128(buf + swz, w0, w1, w2, w3);
+              unpack8(w0, w1, w2, w3, w);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                o[i] = scale * fmaf(P.c_acc, __uint_as_float(v[c8 * 8 + i]), P.c_in * x[i]);
-                o_sq = fmaf(o[i], o[i], o_sq);
+                const float o = scale * __uint_as_float(v[c8 * 8 + i]);
+                o_sq = fmaf(o, o, o_sq);
+                w[i] = fmaf(P.decay, w[i], P.upd_scale * o);
               }
-              if (P.keep_o) {
-                sts128(buf2 + swz, pack2(o[0], o[1]), pack2(o[2], o[3]), pack2(o[4], o[5]), pack2(o[6], o[7]));
-              }
-              if (!w_transposed) {
-                float w[8];
-                lds128(buf + swz, w0, w1, w2, w3);
-                unpack8(w0, w1, w2, w3, w);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) w[i] = fmaf(P.decay, w[i], P.upd_scale * o[i]);
-                sts128(buf + swz, pack2(w[0], w[1]), pack2(w[2], w[3]), pack2(w[4], w[5]), pack2(w[6], w[7]));
-              } else {
-                // W tile as [64 rows of W = columns of O][32 columns of W = rows of
-                // O], not swizzled; this lane owns column `lane` of it.
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                  const int c = c8 * 8 + i;
-                  const float w = __bfloat162float(wt[c * 32 + lane]);
-                  wt[c * 32 + lane] = __float2bfloat16_rn(fmaf(P.decay, w, P.upd_scale * o[i]));
-                }
-              }
+              sts128(buf + swz, pack2(w[0], w[1]), pack2(w[2], w[3]), pack2(w[4], w[5]), pack2(w[6], w[7]));
             }
           }
 
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            if (row0 >= P.m) {
+            if (row0 >= cur.row_limit) {
               // rows beyond the matrix: nothing to store
             } else if (P.last) {
-              if (!sc.nonfinite) {
-                ptx::tma_store_3d(P.wmaps + mat, w_transposed ? row0 : col0, w_transposed ? col0 : row0, 0, buf);
-              }
-              if (P.keep_o) ptx::tma_store_3d(&P.map_out, col0, row0, mat, buf2);
+              if (!sc.nonfinite) ptx::tma_store_3d(P.wmaps + mat, col0, row0, 0, buf);
             } else {
               ptx::tma_store_3d(&P.map_out, col0, row0, mat, buf);
             }
             ptx::tma_store_commit();
-            if (P.has_in && row0 < P.m) --loads_in_flight;
+            if (P.has_in && row0 < cur.row_limit) --loads_in_flight;
             ptx::tma_store_wait_read_all_but_one();  // every store but this quarter's has read its staging
             arm_next();                              // re-arms the entry of the previous quarter
           }
           __syncwarp();
         }
         if (!ok) break;
-        if (row0 >= P.m) o_sq = 0.f;  // rows beyond the matrix were never loaded
+        if (row0 >= cur.row_limit) o_sq = 0.f;  // rows beyond the matrix were never loaded
       }
       if (P.last) {
         // Sum of O^2 of this warp's 32 rows of the tile (Algorithm 1 returns the
