@@ -156,7 +156,9 @@ int muon_partition(const muon_group* groups, int n_groups, int world, int* owner
  * caller's workspace (DEVICE memory, 1024-byte aligned, at least
  * muon_workspace_bytes() long, owned by the caller, alive until destroy),
  * upload pointer tables and encode the TMA descriptors.  `device` is the CUDA
- * device ordinal all pointers live on.  Allocates no device memory itself.
+ * device ordinal all pointers live on; it becomes the calling thread's current
+ * device.  The other calls on the context switch to that device for their
+ * duration and restore the caller's.  Allocates no device memory itself.
  */
 int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* workspace,
               size_t workspace_bytes, int device);

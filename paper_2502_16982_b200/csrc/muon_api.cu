@@ -388,6 +388,19 @@ struct muon_ctx {
 };
 
 namespace {
+// Makes the context's device current for the duration of a call and restores
+// the caller's device afterwards (launches and copies go to the current device).
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int device) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != device) switched = (cudaSetDevice(device) == cudaSuccess);
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
 // Records an event pair around one launch when the context is in measurement mode.
 struct LaunchTimer {
   muon_ctx* ctx;
@@ -823,6 +836,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
 
 int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
   if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
+  DeviceGuard guard(ctx->device);
   int rc = check_hparams(hp);
   if (rc) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
@@ -842,6 +856,7 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
 int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* const* g_host,
                    void* const* const* w_host, void* stream_v) {
   if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
+  DeviceGuard guard(ctx->device);
   if (!g_host) return fail(MUON_ERR_INVALID_ARG, "g_host is null");
   int rc = check_hparams(hp);
   if (rc) return rc;
@@ -919,6 +934,7 @@ int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* con
 
 int muon_status(muon_ctx* ctx, void* stream_v, int* device_status, int* matrix_index) {
   if (!ctx || !device_status) return fail(MUON_ERR_INVALID_ARG, "ctx or device_status is null");
+  DeviceGuard guard(ctx->device);
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   DevStatus st{0, -1};
   cudaError_t ce = cudaMemcpyAsync(&st, ctx->ws + ctx->sizes.off_status, sizeof(st), cudaMemcpyDeviceToHost, stream);
@@ -937,6 +953,7 @@ int muon_status(muon_ctx* ctx, void* stream_v, int* device_status, int* matrix_i
 
 int muon_get_norms(muon_ctx* ctx, void* stream_v, float* out, int n) {
   if (!ctx || !out || n < 0 || n > ctx->total_mats) return fail(MUON_ERR_INVALID_ARG, "bad arguments");
+  DeviceGuard guard(ctx->device);
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   cudaError_t ce = cudaMemcpyAsync(out, ctx->ws + ctx->sizes.off_norms, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
@@ -946,6 +963,7 @@ int muon_get_norms(muon_ctx* ctx, void* stream_v, float* out, int n) {
 
 int muon_get_update_rms(muon_ctx* ctx, void* stream_v, float* out, int n) {
   if (!ctx || !out || n < 0 || n > ctx->total_mats) return fail(MUON_ERR_INVALID_ARG, "bad arguments");
+  DeviceGuard guard(ctx->device);
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   cudaError_t ce = cudaMemcpyAsync(out, ctx->ws + ctx->sizes.off_rms, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
@@ -970,6 +988,7 @@ int muon_profile_enable(muon_ctx* ctx, int enable) {
 
 int muon_profile_read(muon_ctx* ctx, double* ms_by_kernel, int* launches_by_kernel) {
   if (!ctx || !ms_by_kernel || !launches_by_kernel) return fail(MUON_ERR_INVALID_ARG, "null argument");
+  DeviceGuard guard(ctx->device);
   for (int k = 0; k < MUON_KERNEL_KINDS; ++k) { ms_by_kernel[k] = 0.0; launches_by_kernel[k] = 0; }
   cudaError_t ce = cudaDeviceSynchronize();
   if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "synchronise: %s", cudaGetErrorString(ce));
@@ -987,6 +1006,7 @@ int muon_profile_read(muon_ctx* ctx, double* ms_by_kernel, int* launches_by_kern
 
 int muon_debug_tmem_bases(muon_ctx* ctx, unsigned* out_host, int n) {
   if (!ctx || !out_host || n < 0 || n > 1024) return fail(MUON_ERR_INVALID_ARG, "bad arguments");
+  DeviceGuard guard(ctx->device);
   cudaError_t ce = cudaDeviceSynchronize();
   if (ce == cudaSuccess)
     ce = cudaMemcpy(out_host, ctx->ws + ctx->sizes.off_debug, n * sizeof(unsigned), cudaMemcpyDeviceToHost);
@@ -997,6 +1017,7 @@ int muon_debug_tmem_bases(muon_ctx* ctx, unsigned* out_host, int n) {
 int muon_debug_wait_expiry(muon_ctx* ctx, void* stream_v, int matrix_index, unsigned limit_ms) {
   if (!ctx || matrix_index < 0 || matrix_index >= ctx->total_mats || limit_ms == 0 || limit_ms > 1000)
     return fail(MUON_ERR_INVALID_ARG, "bad arguments (limit_ms must be 1..1000)");
+  DeviceGuard guard(ctx->device);
   DevStatus* status = reinterpret_cast<DevStatus*>(ctx->ws + ctx->sizes.off_status);
   cudaError_t ce = launch_wait_expiry_probe(status, matrix_index, static_cast<unsigned long long>(limit_ms) * 1000000ull,
                                             static_cast<cudaStream_t>(stream_v));
@@ -1013,6 +1034,7 @@ int muon_debug_keep(muon_ctx* ctx, int keep) {
 int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, size_t dst_bytes) {
   if (!ctx || !dst_host) return fail(MUON_ERR_INVALID_ARG, "ctx or dst is null");
   if (matrix_index < 0 || matrix_index >= ctx->total_mats) return fail(MUON_ERR_INVALID_ARG, "matrix index out of range");
+  DeviceGuard guard(ctx->device);
   const int b = ctx->where[matrix_index].first, pos = ctx->where[matrix_index].second;
   const Bucket& B = ctx->buckets[b];
   if (ctx->buckets.size() != 1 || static_cast<int>(B.mats.size()) > B.chunk)
