@@ -42,3 +42,33 @@ def test_host_only_calls_work_without_a_gpu():
     except b.MuonError as e:
         assert e.code == b.MUON_ERR_INVALID_ARG
         assert "positive" in str(e)
+
+
+def test_workspace_plan_properties_on_the_host():
+    """The shape-bucketed planner is pure host arithmetic: both orientations of
+    one (min, max) share a bucket, buckets share the chunk buffers (the
+    workspace follows the largest bucket, not the sum), and a bucket above the
+    chunk limit is cut into chunks that reuse them."""
+    from paper_2502_16982_b200 import binding as b
+
+    bf = b.MUON_DTYPE_BF16
+
+    def ws(shapes):
+        return b.muon_workspace_bytes(b.shape_only_groups(shapes), len(shapes))
+
+    one = ws([(2048, 1408, 8, bf, bf)])
+    both = ws([(2048, 1408, 4, bf, bf), (1408, 2048, 4, bf, bf)])
+    assert abs(both - one) <= 4096  # same bucket of 8 matrices (one more group header at most)
+    small = ws([(256, 256, 8, bf, bf)])
+    mixed = ws([(2048, 1408, 8, bf, bf), (256, 256, 8, bf, bf)])
+    assert mixed < one + small and mixed >= one  # chunk buffers shared, per-matrix tables added
+    per_matrix = (2 * 1408 * 2048 + 2 * 1408 * 1408) * 2
+    assert one >= 8 * per_matrix
+    prev = b.muon_debug_set_chunk_bytes(2 * per_matrix + 1024)
+    try:
+        chunked = ws([(2048, 1408, 8, bf, bf)])
+    finally:
+        b.muon_debug_set_chunk_bytes(prev)
+    assert chunked < 4 * per_matrix  # two matrices per chunk instead of eight
+    # fp32 and bf16 weights of one shape are different buckets but still share the buffers
+    assert ws([(512, 512, 2, b.MUON_DTYPE_FP32, bf), (512, 512, 2, bf, bf)]) < 2 * ws([(512, 512, 2, bf, bf)])
