@@ -576,6 +576,38 @@ def test_expired_device_wait_is_reported_and_the_context_survives():
         case.close()
 
 
+def test_host_buffer_entry_point_pipelines_several_buckets():
+    """muon_step_host cuts every bucket into slices whose uploads, kernels and
+    downloads overlap on three streams; the result must be the bits of
+    muon_step on device-resident gradients (two buckets, nine matrices each,
+    two steps so that a second call follows the first on the same stream)."""
+    specs = [wl.GroupSpec(264, 200, 9, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(136, 392, 9, torch.bfloat16, torch.float32, 0.02, 1e-3)]
+    case = Case(specs, seed=71)
+    ref = Case(specs, seed=71)
+    try:
+        hp = default_hp(lr=1e-2)
+        gen = torch.Generator().manual_seed(72)
+        for step in range(2):
+            g_new = [wl.make_grads(sp, gen, "cpu") for sp in specs]
+            g_host = [[g[i].contiguous().pin_memory() for i in range(sp.count)] for g, sp in zip(g_new, specs)]
+            w_host = [[torch.empty(sp.rows, sp.cols, dtype=torch.bfloat16).pin_memory() for _ in range(sp.count)]
+                      for sp in specs]
+            case.ctx.muon_step_host(hp, g_host, w_host)
+            assert case.ctx.muon_status()[0] == 0
+            for gi in range(2):
+                ref.dev[gi][1].copy_(g_new[gi])
+            assert ref.step(hp)[0] == 0
+            for gi, sp in enumerate(specs):
+                for i in range(sp.count):
+                    assert torch.equal(w_host[gi][i], ref.dev[gi][0][i].cpu()), (step, gi, i)
+                assert torch.equal(case.dev[gi][0], ref.dev[gi][0]) and torch.equal(case.dev[gi][2], ref.dev[gi][2])
+        assert case.ctx.muon_get_norms() == ref.ctx.muon_get_norms()
+    finally:
+        case.close()
+        ref.close()
+
+
 def test_invalid_descriptors_are_rejected_on_the_host():
     b = _binding()
     W = torch.zeros(2, 64, 64, device="cuda")
