@@ -174,6 +174,28 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
 int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream);
 
 /*
+ * The shape buckets the planner forms from these groups (pure host
+ * computation, like muon_workspace_bytes): bucket_out[i] (HOST, one int per
+ * matrix, groups in order) is the bucket of matrix i, n_buckets_out the number
+ * of buckets.  A bucket holds every matrix with the same short side, long
+ * side and dtypes, whichever way round it is stored, and is the unit
+ * muon_step_bucket works on.  A context built from the same groups uses the
+ * same numbering.
+ */
+int muon_plan_buckets(const muon_group* groups, int n_groups, int* bucket_out, int* n_buckets_out);
+
+/*
+ * muon_step for the matrices of ONE bucket (numbering of muon_plan_buckets).
+ * Stepping every bucket once, in any order, is one muon_step.  Exists so that
+ * a data-parallel caller can start sharing a bucket's updated weights while the
+ * next bucket is still in its Newton-Schulz iteration (Sec. 2.3 asks for the
+ * gather and the computation to overlap).  Same stream ordering, error
+ * behaviour and asynchrony as muon_step; buckets share the workspace, so the
+ * calls of one context stay on one stream.
+ */
+int muon_step_bucket(muon_ctx* ctx, const muon_hparams* hp, int bucket, void* stream);
+
+/*
  * Same step with HOST gradients and HOST weight read-back, for callers whose
  * gradients arrive in (pinned) host memory: for every matrix i of every group
  * j, g_host[j][i] (host, dense rows*cols of the group's g_dtype) is copied

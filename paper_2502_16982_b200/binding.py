@@ -30,7 +30,8 @@ MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
 MUON_SCALE_ADJUSTED_LR, MUON_SCALE_FIXED_DIM, MUON_SCALE_UPDATE_NORM = 0, 1, 2
 
 EXPORTED = [
-    "muon_workspace_bytes", "muon_partition", "muon_init", "muon_step", "muon_step_host", "muon_status",
+    "muon_workspace_bytes", "muon_partition", "muon_plan_buckets", "muon_init", "muon_step", "muon_step_bucket",
+    "muon_step_host", "muon_status",
     "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes", "muon_debug_wait_expiry",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
@@ -94,6 +95,8 @@ def lib():
     L.muon_partition.argtypes = [C.POINTER(muon_group), C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_double)]
     L.muon_init.argtypes = [C.POINTER(C.c_void_p), C.POINTER(muon_group), C.c_int, C.c_void_p, C.c_size_t, C.c_int]
     L.muon_step.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_void_p]
+    L.muon_plan_buckets.argtypes = [C.POINTER(muon_group), C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+    L.muon_step_bucket.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_int, C.c_void_p]
     L.muon_step_host.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.POINTER(C.POINTER(C.c_void_p)),
                                  C.POINTER(C.POINTER(C.c_void_p)), C.c_void_p]
     L.muon_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
@@ -276,6 +279,17 @@ def muon_partition(shapes, world: int):
     return list(owners), list(loads)
 
 
+def muon_plan_buckets(shapes):
+    """Bucket of every matrix.  ``shapes`` is a list of (rows, cols, count,
+    w_dtype code, g_dtype code); returns (bucket per matrix, number of buckets)."""
+    arr = shape_only_groups(shapes)
+    total = sum(sh[2] for sh in shapes)
+    out = (C.c_int * total)()
+    n = C.c_int(0)
+    _check(lib().muon_plan_buckets(arr, len(shapes), out, C.byref(n)))
+    return list(out), n.value
+
+
 def muon_debug_set_chunk_bytes(nbytes: int) -> int:
     """Test knob: bound on the Newton-Schulz operand bytes of one bucket chunk
     (0 = default).  Returns the previous value."""
@@ -319,6 +333,12 @@ class MuonContext:
         s = torch.cuda.current_stream(self.device) if stream is None else stream
         c_hp = hp.to_c()
         _check(lib().muon_step(self._ctx, C.byref(c_hp), C.c_void_p(s.cuda_stream)))
+
+    def muon_step_bucket(self, hp: Hyper, bucket: int, stream=None):
+        import torch
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        c_hp = hp.to_c()
+        _check(lib().muon_step_bucket(self._ctx, C.byref(c_hp), int(bucket), C.c_void_p(s.cuda_stream)))
 
     def muon_step_host(self, hp: Hyper, g_host, w_host=None, stream=None):
         """g_host / w_host: per group, a list of pinned CPU tensors (dense)."""

@@ -478,6 +478,21 @@ int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_byt
   return MUON_OK;
 }
 
+int muon_plan_buckets(const muon_group* groups, int n_groups, int* bucket_out, int* n_buckets_out) {
+  if (!bucket_out || !n_buckets_out) return fail(MUON_ERR_INVALID_ARG, "bucket_out or n_buckets_out is null");
+  int rc = validate_groups(groups, n_groups, false);
+  if (rc) return rc;
+  std::vector<Bucket> buckets;
+  PlanSizes sizes;
+  int total;
+  rc = make_plan(groups, n_groups, &buckets, &sizes, &total);
+  if (rc) return rc;
+  for (size_t b = 0; b < buckets.size(); ++b)
+    for (const MatRef& r : buckets[b].mats) bucket_out[r.global] = static_cast<int>(b);
+  *n_buckets_out = static_cast<int>(buckets.size());
+  return MUON_OK;
+}
+
 int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* workspace,
               size_t workspace_bytes, int device) {
   if (!out_ctx) return fail(MUON_ERR_INVALID_ARG, "out_ctx is null");
@@ -848,6 +863,25 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream_v) {
       rc = step_chunk(ctx, hp, stream, b, first, std::min(B.chunk, total - first), &launches);
       if (rc) return rc;
     }
+  }
+  ctx->last_launches = launches;
+  return MUON_OK;
+}
+
+int muon_step_bucket(muon_ctx* ctx, const muon_hparams* hp, int bucket, void* stream_v) {
+  if (!ctx) return fail(MUON_ERR_INVALID_ARG, "ctx is null");
+  if (bucket < 0 || bucket >= static_cast<int>(ctx->buckets.size()))
+    return fail(MUON_ERR_INVALID_ARG, "bucket %d out of range (context has %zu)", bucket, ctx->buckets.size());
+  DeviceGuard guard(ctx->device);
+  int rc = check_hparams(hp);
+  if (rc) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  int launches = 0;
+  const Bucket& B = ctx->buckets[bucket];
+  const int total = static_cast<int>(B.mats.size());
+  for (int first = 0; first < total; first += B.chunk) {
+    rc = step_chunk(ctx, hp, stream, bucket, first, std::min(B.chunk, total - first), &launches);
+    if (rc) return rc;
   }
   ctx->last_launches = launches;
   return MUON_OK;

@@ -72,3 +72,23 @@ def test_workspace_plan_properties_on_the_host():
     assert chunked < 4 * per_matrix  # two matrices per chunk instead of eight
     # fp32 and bf16 weights of one shape are different buckets but still share the buffers
     assert ws([(512, 512, 2, b.MUON_DTYPE_FP32, bf), (512, 512, 2, bf, bf)]) < 2 * ws([(512, 512, 2, bf, bf)])
+
+
+def test_bucket_plan_groups_by_sides_and_dtypes_on_the_host():
+    """muon_plan_buckets: matrices share a bucket exactly when short side, long
+    side and both dtypes agree, whatever their orientation; numbering is dense."""
+    from paper_2502_16982_b200 import binding as b
+
+    BF, FP = b.MUON_DTYPE_BF16, b.MUON_DTYPE_FP32
+    shapes = [(2048, 1408, 4, BF, BF), (512, 4096, 2, BF, BF), (1408, 2048, 3, BF, BF),
+              (2048, 1408, 1, FP, BF), (4096, 512, 1, BF, FP), (2048, 2048, 2, BF, BF)]
+    bucket_of, n = b.muon_plan_buckets(shapes)
+    keys = []
+    for r, c, cnt, wd, gd in shapes:
+        keys += [(min(r, c), max(r, c), wd, gd)] * cnt
+    assert len(bucket_of) == len(keys) and sorted(set(bucket_of)) == list(range(n))
+    assert n == len(set(keys)) == 5
+    for i in range(len(keys)):
+        for j in range(len(keys)):
+            assert (bucket_of[i] == bucket_of[j]) == (keys[i] == keys[j])
+    assert b.muon_plan_buckets(shapes) == (bucket_of, n)

@@ -43,20 +43,22 @@ def _free_port():
     return port
 
 
-def _fake_step(local_groups, hp):
+def _fake_step(mats, hp):
     # stand-in for the CUDA step: deterministic, touches owned weights and momentum only
-    for ws, gs, ms in local_groups:
-        for w, g, m in zip(ws, gs, ms):
-            m.mul_(0.5).add_(g.float())
-            w.sub_((hp * m).to(w.dtype))
+    for w, g, m in mats:
+        m.mul_(0.5).add_(g.float())
+        w.sub_((hp * m).to(w.dtype))
 
 
 def _make_groups(seed):
+    # 16x8 and 8x16 share a bucket (same short and long side); the 4x4 bf16 and fp32
+    # groups do not (dtypes differ); the single 32x8 matrix is a bucket only one rank owns
     gen = torch.Generator().manual_seed(seed)
     groups = []
-    for rows, cols, n in ((8, 12, 3), (16, 8, 2), (4, 4, 4)):
-        ws = [torch.randn(rows, cols, generator=gen) for _ in range(n)]
-        gs = [torch.randn(rows, cols, generator=gen) for _ in range(n)]
+    for rows, cols, n, dtype in ((8, 12, 3, torch.float32), (16, 8, 2, torch.float32), (4, 4, 4, torch.bfloat16),
+                                 (8, 16, 3, torch.float32), (32, 8, 1, torch.float32), (4, 4, 2, torch.float32)):
+        ws = [torch.randn(rows, cols, generator=gen).to(dtype) for _ in range(n)]
+        gs = [torch.randn(rows, cols, generator=gen).to(dtype) for _ in range(n)]
         groups.append((ws, gs))
     return groups
 
@@ -73,7 +75,9 @@ def _worker(rank, world, port, out):
         dm.step(0.1)
     n_owned = len(dm.owned)
     n_mom = sum(len(ms) for _, _, ms in dm.local_groups)
-    torch.save({"w": [w.clone() for ws, _ in groups for w in ws], "owned": n_owned, "mom": n_mom}, out % rank)
+    torch.save({"w": [w.clone() for ws, _ in groups for w in ws], "owned": n_owned, "mom": n_mom,
+                "units": dm.n_units, "unit_of": dm.unit_of,
+                "stepped": [len(ms) for ms in dm.unit_mats]}, out % rank)
     dist.barrier()
     dist.destroy_process_group()
 
@@ -92,5 +96,13 @@ def test_two_ranks_end_with_the_single_process_weights(tmp_path):
     single = [w for ws, _ in groups for w in ws]
     assert r0["owned"] + r1["owned"] == len(single) and r0["owned"] > 0 and r1["owned"] > 0
     assert r0["mom"] == r0["owned"] and r1["mom"] == r1["owned"]  # momentum only for owned matrices
+    # the gather's units: five buckets, the same on both ranks; the two orientations share one
+    assert r0["units"] == r1["units"] == 5 and r0["unit_of"] == r1["unit_of"]
+    u = r0["unit_of"]
+    assert u[3] == u[4] == u[9] == u[10] == u[11] and u[5] != u[13] and len(set(u)) == 5
+    # each unit's matrices are stepped by exactly one rank each, and the one-matrix unit by one rank alone
+    both = [a + b_ for a, b_ in zip(r0["stepped"], r1["stepped"])]
+    assert both == [u.count(k) for k in range(5)]
+    assert sorted((r0["stepped"][u[12]], r1["stepped"][u[12]])) == [0, 1]
     for a, b_, c in zip(r0["w"], r1["w"], single):
         assert torch.equal(a, c) and torch.equal(b_, c)

@@ -454,6 +454,65 @@ def test_owner_computes_shards_give_the_single_context_bits():
         shard.close()
 
 
+def test_bucket_by_bucket_step_gives_muon_step_bits():
+    """muon_step_bucket over every bucket, in reverse order, is one muon_step:
+    buckets are independent, and the numbering is muon_plan_buckets' (the two
+    orientations of 328 x 200 share a bucket, so three groups make two buckets)."""
+    b = _binding()
+    specs = [wl.GroupSpec(328, 200, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(256, 256, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(200, 328, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
+    bucket_of, n_buckets = b.muon_plan_buckets(
+        [(sp.rows, sp.cols, sp.count, b.MUON_DTYPE_BF16, b.MUON_DTYPE_BF16) for sp in specs])
+    assert n_buckets == 2 and bucket_of == [0, 0, 0, 1, 1, 0, 0]
+    hp = default_hp(lr=1e-2)
+    whole = Case(specs, seed=71)
+    parts = Case(specs, seed=71)
+    try:
+        for _ in range(2):
+            assert whole.step(hp)[0] == 0
+            for bk in reversed(range(n_buckets)):
+                parts.ctx.muon_step_bucket(hp, bk)
+            assert parts.ctx.muon_status()[0] == 0
+        for gi in range(len(specs)):
+            assert torch.equal(whole.dev[gi][0], parts.dev[gi][0])
+            assert torch.equal(whole.dev[gi][2], parts.dev[gi][2])
+        assert whole.ctx.muon_get_norms() == parts.ctx.muon_get_norms()
+        assert whole.ctx.muon_get_update_rms() == parts.ctx.muon_get_update_rms()
+        with pytest.raises(b.MuonError):
+            parts.ctx.muon_step_bucket(hp, n_buckets)
+    finally:
+        whole.close()
+        parts.close()
+
+
+def test_distributed_wrapper_single_rank_steps_bucket_by_bucket():
+    """The data-parallel wrapper with one rank owns every matrix and must give
+    the plain context's bits (its momentum starts at zero like the plain one's)."""
+    b = _binding()
+    from paper_2502_16982_b200.distributed import DistributedMuon
+    specs = [wl.GroupSpec(328, 200, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(200, 328, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(128, 384, 2, torch.float32, torch.float32, 0.02, 1.0)]
+    hp = default_hp(lr=1e-2)
+    plain = Case(specs, seed=73)
+    other = Case(specs, seed=73)
+    dm = DistributedMuon([([W[i] for i in range(sp.count)], [G[i] for i in range(sp.count)])
+                          for sp, (W, G, M) in zip(specs, other.dev)])
+    try:
+        assert dm.n_units == 2
+        for _ in range(2):
+            assert plain.step(hp)[0] == 0
+            dm.step(hp)
+        torch.cuda.synchronize()
+        for gi in range(len(specs)):
+            assert torch.equal(plain.dev[gi][0], other.dev[gi][0])
+    finally:
+        dm.close()
+        plain.close()
+        other.close()
+
+
 def test_bitwise_reproducible():
     specs = [wl.GroupSpec(448, 640, 4, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
     outs = []
