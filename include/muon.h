@@ -170,6 +170,8 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
  * enqueued, performs no allocation and no host synchronisation.  Device-side
  * problems (expired wait, non-finite input) are reported by muon_status.
  * Calls on one context must be stream-ordered with respect to each other.
+ * Because the call only enqueues kernels, it may be recorded into a CUDA graph
+ * by stream capture; the hyper-parameters are then those of the capture.
  */
 int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream);
 

@@ -513,6 +513,50 @@ def test_distributed_wrapper_single_rank_steps_bucket_by_bucket():
         other.close()
 
 
+def test_step_captured_in_a_cuda_graph_replays_the_eager_bits():
+    """muon_step only enqueues kernels on the caller's stream (no allocation, no
+    host synchronisation), so it can be captured once and replayed: two replays
+    with fresh gradients give the bits of two eager steps."""
+    specs = [wl.GroupSpec(328, 200, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(256, 384, 2, torch.float32, torch.float32, 0.02, 1.0)]
+    hp = default_hp(lr=1e-2)
+    eager = Case(specs, seed=91)
+    graphed = Case(specs, seed=91)
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            graph.capture_begin()
+            graphed.ctx.muon_step(hp, stream=side)
+            graph.capture_end()
+        torch.cuda.current_stream().wait_stream(side)
+        # capture enqueues nothing: weights and momentum are untouched so far
+        fresh = Case(specs, seed=91)
+        for gi in range(len(specs)):
+            assert torch.equal(graphed.dev[gi][0], fresh.dev[gi][0])
+            assert torch.equal(graphed.dev[gi][2], fresh.dev[gi][2])
+        fresh.close()
+        for step in range(2):
+            if step:
+                for gi, sp in enumerate(specs):
+                    gen = torch.Generator().manual_seed(900 + gi)
+                    g_new = wl.make_grads(sp, gen, "cpu").cuda()
+                    eager.dev[gi][1].copy_(g_new)
+                    graphed.dev[gi][1].copy_(g_new)
+            assert eager.step(hp)[0] == 0
+            graph.replay()
+            assert graphed.ctx.muon_status()[0] == 0
+        for gi in range(len(specs)):
+            assert torch.equal(eager.dev[gi][0], graphed.dev[gi][0])
+            assert torch.equal(eager.dev[gi][2], graphed.dev[gi][2])
+        assert eager.ctx.muon_get_norms() == graphed.ctx.muon_get_norms()
+        del graph
+    finally:
+        eager.close()
+        graphed.close()
+
+
 def test_bitwise_reproducible():
     specs = [wl.GroupSpec(448, 640, 4, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
     outs = []
