@@ -187,6 +187,17 @@ int muon_step(muon_ctx* ctx, const muon_hparams* hp, void* stream);
 int muon_plan_buckets(const muon_group* groups, int n_groups, int* bucket_out, int* n_buckets_out);
 
 /*
+ * Newton-Schulz FLOPs of one step over these groups (pure host computation):
+ * *algorithmic_out is Eq. 2 counted with the symmetric products halved,
+ * ns_steps * (3 m^2 n + m^3) per matrix; *planned_out is what the planner's
+ * launch sequence asks of the tensor cores, which is less where it takes the
+ * iterations two at a time (3 m^2 n + 5 m^3 per pair; see
+ * muon_debug_set_pair_fold).  Neither counts tile padding.
+ */
+int muon_plan_flops(const muon_group* groups, int n_groups, int ns_steps, double* algorithmic_out,
+                    double* planned_out);
+
+/*
  * muon_step for the matrices of ONE bucket (numbering of muon_plan_buckets).
  * Stepping every bucket once, in any order, is one muon_step.  Exists so that
  * a data-parallel caller can start sharing a bucket's updated weights while the
@@ -309,6 +320,18 @@ int muon_debug_wait_expiry(muon_ctx* ctx, void* stream, int matrix_index, unsign
  * chunked path on small buckets.
  */
 size_t muon_debug_set_chunk_bytes(size_t bytes);
+
+/*
+ * Test knob: how the planner chooses between the plain iteration sequence and
+ * taking the iterations two at a time (Eq. 2 gives X_{k+1} = P_k X_k with
+ * P_k = a*I + b*A_k + c*A_k^2, so A_{k+1} = P_k^2 A_k and X_{k+2} = P_{k+1} P_k X_k
+ * need no pass over X for every second iteration).  0: by shape (the default:
+ * from 256 rows and a long side of at least twice the short side), 1: never,
+ * 2: whenever the short side is at least 16.  Process-wide, read by
+ * muon_workspace_bytes and muon_init like the chunk bound.  Returns the previous
+ * mode; a value outside 0..2 only queries.
+ */
+int muon_debug_set_pair_fold(int mode);
 
 /*
  * Test tap: the TMEM base address each CTA of the last Newton-Schulz GEMM launch

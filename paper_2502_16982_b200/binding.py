@@ -30,10 +30,11 @@ MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
 MUON_SCALE_ADJUSTED_LR, MUON_SCALE_FIXED_DIM, MUON_SCALE_UPDATE_NORM = 0, 1, 2
 
 EXPORTED = [
-    "muon_workspace_bytes", "muon_partition", "muon_plan_buckets", "muon_init", "muon_step", "muon_step_bucket",
+    "muon_workspace_bytes", "muon_partition", "muon_plan_buckets", "muon_plan_flops", "muon_init", "muon_step", "muon_step_bucket",
     "muon_step_host", "muon_status",
     "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
-    "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes", "muon_debug_wait_expiry",
+    "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes", "muon_debug_set_pair_fold",
+    "muon_debug_wait_expiry",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
     "muon_momentum_norm_static", "muon_adamw_step",
 ]
@@ -96,6 +97,8 @@ def lib():
     L.muon_init.argtypes = [C.POINTER(C.c_void_p), C.POINTER(muon_group), C.c_int, C.c_void_p, C.c_size_t, C.c_int]
     L.muon_step.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_void_p]
     L.muon_plan_buckets.argtypes = [C.POINTER(muon_group), C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+    L.muon_plan_flops.argtypes = [C.POINTER(muon_group), C.c_int, C.c_int, C.POINTER(C.c_double),
+                                  C.POINTER(C.c_double)]
     L.muon_step_bucket.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_int, C.c_void_p]
     L.muon_step_host.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.POINTER(C.POINTER(C.c_void_p)),
                                  C.POINTER(C.POINTER(C.c_void_p)), C.c_void_p]
@@ -113,6 +116,7 @@ def lib():
     L.muon_momentum_norm_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64,
                                             C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
     L.muon_debug_set_chunk_bytes.argtypes = [C.c_size_t]
+    L.muon_debug_set_pair_fold.argtypes = [C.c_int]
     L.muon_debug_wait_expiry.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_uint]
     L.muon_adamw_step.argtypes = [C.POINTER(muon_adamw_tensor), C.c_int, C.POINTER(muon_adamw_hparams), C.c_int,
                                   C.c_void_p]
@@ -277,6 +281,21 @@ def muon_partition(shapes, world: int):
     loads = (C.c_double * world)()
     _check(lib().muon_partition(arr, len(shapes), int(world), owners, loads))
     return list(owners), list(loads)
+
+
+def muon_plan_flops(shapes, ns_steps: int = 5):
+    """(algorithmic, planned) Newton-Schulz FLOPs of one step; ``shapes`` is a
+    list of (rows, cols, count)."""
+    arr = shape_only_groups([(r, c, n, MUON_DTYPE_BF16, MUON_DTYPE_BF16) for (r, c, n) in shapes])
+    alg, planned = C.c_double(0), C.c_double(0)
+    _check(lib().muon_plan_flops(arr, len(shapes), int(ns_steps), C.byref(alg), C.byref(planned)))
+    return alg.value, planned.value
+
+
+def muon_debug_set_pair_fold(mode: int) -> int:
+    """Test knob: 0 = iterations taken in pairs by shape (default), 1 = never,
+    2 = whenever the short side is at least 16.  Returns the previous mode."""
+    return lib().muon_debug_set_pair_fold(int(mode))
 
 
 def muon_plan_buckets(shapes):

@@ -31,6 +31,8 @@ cudaError_t launch_update_from_x(const MatDesc* descs, const MatScal* scal, cons
 cudaError_t launch_rms_finalise(const float* partials, int per_matrix, int count, float factor,
                                 const MatDesc* descs, const MatScal* scal, bool use_inv_norm, float rms_target,
                                 bool normalise, float* rms, float* factors, cudaStream_t stream);
+cudaError_t launch_symmetrise_diag(__nv_bfloat16* s, long long stride, int lda, int m, int count,
+                                   cudaStream_t stream);
 cudaError_t launch_sumsq_x(const __nv_bfloat16* x, long long x_stride, int ldx, int m, int n, int count,
                            int per_matrix, float* partials, cudaStream_t stream);
 cudaError_t stream_tma_configure();
@@ -63,6 +65,26 @@ constexpr size_t kChunkBytesDefault = size_t(8) << 30;
 size_t g_chunk_bytes_max = kChunkBytesDefault;  // process-wide; see muon_debug_set_chunk_bytes
 constexpr int kChunkCountMax = 4096;
 
+// Two iterations per pass over X.  With P_k = a*I + b*A_k + c*A_k^2 (symmetric, a
+// polynomial in A_k = X_k X_k^T) Eq. 2 reads X_{k+1} = P_k X_k, hence
+//   A_{k+1} = P_k A_k P_k = P_k^2 A_k   and   X_{k+2} = (P_{k+1} P_k) X_k:
+// the Gram product and the combine (m^2 n each way) of every second iteration
+// are replaced by three more symmetric m x m x m products, 3 m^2 n + 5 m^3
+// instead of 6 m^2 n + 2 m^3 for the two iterations.  That pays when the long
+// side is well above the short side; with bf16 storage the result is as close
+// to the exact iteration as the plain sequence for n >= 3 m and within 1.4 x of
+// its distance at n = 2 m from 256 rows on (bf16 storage model on the CPU), and
+// further off for small or near-square matrices, which keep the plain sequence.
+constexpr int kPairFoldMinRows = 256;
+constexpr double kPairFoldMinAspect = 2.0;
+int g_pair_fold_mode = 0;  // 0: by shape, 1: never, 2: whenever a*I is folded; see muon_debug_set_pair_fold
+
+bool plan_pair_fold(int m, int n, bool fold_identity) {
+  if (!fold_identity || g_pair_fold_mode == 1) return false;
+  if (g_pair_fold_mode == 2) return true;
+  return m >= kPairFoldMinRows && static_cast<double>(n) >= kPairFoldMinAspect * m;
+}
+
 struct MatRef {
   int group, index, global;
 };
@@ -80,8 +102,10 @@ struct Bucket {
   bool fused_update;          // every W is bf16 and TMA-addressable: update W in the last epilogue
   bool stream_tma;            // every G and M is TMA-addressable: TMA-pipelined momentum kernel
   bool fold_identity;         // keep B' = B + a*I so that the combine is the single product B' X
+  bool pair_fold;             // take two iterations per pass over X (see plan_pair_fold)
   // workspace offsets (bytes) of the chunk buffers
-  size_t off_x[2], off_a, off_b, off_partials, off_scal, off_rms_partials, off_factors;
+  // off_s: the symmetric m x m buffers (A and B; two more when iterations are taken in pairs)
+  size_t off_x[2], off_s[4], off_partials, off_scal, off_rms_partials, off_factors;
   // workspace offsets of the persistent per-bucket tables
   size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_comb_tiles, off_comb_tiles_t;
   std::vector<PairTile> sym_tiles, comb_tiles;  // tile tables of one matrix
@@ -91,9 +115,9 @@ struct Bucket {
   CUtensorMap x_op[2];   // X as K-major operand A: box {64,128}
   CUtensorMap x_b64[2];  // X as operand B (K-major or MN-major): box {64,64}
   CUtensorMap x_e[2];    // X as epilogue input / output: box {64,32}
-  CUtensorMap a_op, b_op;    // A, B as K-major operand A: box {64,128}
-  CUtensorMap a_b64, b_b64;  // A, B as operand B or as transposed (MN-major) operand A: box {64,64}
-  CUtensorMap a_e, b_e;      // A, B as epilogue input / output: box {64,32}
+  CUtensorMap s_op[4];   // symmetric buffer as K-major operand A: box {64,128}
+  CUtensorMap s_b64[4];  // as operand B or as transposed (MN-major) operand A: box {64,64}
+  CUtensorMap s_e[4];    // as epilogue input / output: box {64,32}
 };
 
 struct PlanSizes {
@@ -254,7 +278,9 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     // Folding a*X into the product rounds B_ii + a to bf16; that is the smaller
     // error from 16 rows up (measured with a bf16 storage model) and the larger one below.
     B.fold_identity = B.m >= 16;
-    const size_t per_mat = 2 * B.x_stride * 2 + 2 * B.a_stride * 2;
+    B.pair_fold = plan_pair_fold(B.m, B.n, B.fold_identity);
+    const int n_sym = B.pair_fold ? 4 : 2;
+    const size_t per_mat = 2 * B.x_stride * 2 + n_sym * B.a_stride * 2;
     size_t chunk = std::max<size_t>(1, g_chunk_bytes_max / per_mat);
     chunk = std::min<size_t>(chunk, B.mats.size());
     chunk = std::min<size_t>(chunk, kChunkCountMax);
@@ -269,8 +295,7 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     };
     B.off_x[0] = take(chunk * B.x_stride * 2);
     B.off_x[1] = take(chunk * B.x_stride * 2);
-    B.off_a = take(chunk * B.a_stride * 2);
-    B.off_b = take(chunk * B.a_stride * 2);
+    for (int i = 0; i < 4; ++i) B.off_s[i] = i < n_sym ? take(chunk * B.a_stride * 2) : 0;
     B.off_partials = take(chunk * static_cast<size_t>(B.stream_tiles) * sizeof(float));
     B.off_scal = take(chunk * sizeof(MatScal));
     // sums of O^2 of the last epilogue: per matrix, comb tile, CTA of the pair and epilogue warp
@@ -371,6 +396,7 @@ struct muon_ctx {
   std::vector<std::pair<int, int>> where;
   // debug taps: which X buffer holds X0 / the last X per bucket
   std::vector<int> x0_buf, xlast_buf;
+  std::vector<int> a_last_buf, b_last_buf;  // symmetric buffers holding the last iteration's A and B
   // per-launch timing (measurement mode)
   int profile;
   std::vector<cudaEvent_t> ev_pool;           // pairs: start, stop
@@ -478,6 +504,12 @@ int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_byt
   return MUON_OK;
 }
 
+int muon_debug_set_pair_fold(int mode) {
+  const int prev = g_pair_fold_mode;
+  if (mode >= 0 && mode <= 2) g_pair_fold_mode = mode;
+  return prev;
+}
+
 int muon_plan_buckets(const muon_group* groups, int n_groups, int* bucket_out, int* n_buckets_out) {
   if (!bucket_out || !n_buckets_out) return fail(MUON_ERR_INVALID_ARG, "bucket_out or n_buckets_out is null");
   int rc = validate_groups(groups, n_groups, false);
@@ -490,6 +522,27 @@ int muon_plan_buckets(const muon_group* groups, int n_groups, int* bucket_out, i
   for (size_t b = 0; b < buckets.size(); ++b)
     for (const MatRef& r : buckets[b].mats) bucket_out[r.global] = static_cast<int>(b);
   *n_buckets_out = static_cast<int>(buckets.size());
+  return MUON_OK;
+}
+
+int muon_plan_flops(const muon_group* groups, int n_groups, int ns_steps, double* algorithmic_out,
+                    double* planned_out) {
+  if (!algorithmic_out || !planned_out) return fail(MUON_ERR_INVALID_ARG, "output pointer is null");
+  if (ns_steps < 0 || ns_steps > 64) return fail(MUON_ERR_INVALID_ARG, "ns_steps must be in [0, 64]");
+  int rc = validate_groups(groups, n_groups, false);
+  if (rc) return rc;
+  double alg = 0.0, planned = 0.0;
+  for (int g = 0; g < n_groups; ++g) {
+    const double m = std::min(groups[g].rows, groups[g].cols), n = std::max(groups[g].rows, groups[g].cols);
+    const double one = 3.0 * m * m * n + m * m * m;     // Gram (half), polynomial (half), combine
+    const double two = 3.0 * m * m * n + 5.0 * m * m * m;  // one Gram, five symmetric m^3 products, one combine
+    const bool pairs = plan_pair_fold(static_cast<int>(m), static_cast<int>(n), m >= 16);
+    const int n_pairs = pairs ? ns_steps / 2 : 0;
+    alg += groups[g].count * ns_steps * one;
+    planned += groups[g].count * (n_pairs * two + (ns_steps - 2 * n_pairs) * one);
+  }
+  *algorithmic_out = alg;
+  *planned_out = planned;
   return MUON_OK;
 }
 
@@ -558,6 +611,8 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   ctx->where.assign(ctx->total_mats, std::make_pair(-1, -1));
   ctx->x0_buf.assign(ctx->buckets.size(), 0);
   ctx->xlast_buf.assign(ctx->buckets.size(), 0);
+  ctx->a_last_buf.assign(ctx->buckets.size(), 0);
+  ctx->b_last_buf.assign(ctx->buckets.size(), 1);
 
   // per-bucket: upload matrix descriptors and W maps, encode tensor maps
   for (size_t b = 0; b < ctx->buckets.size(); ++b) {
@@ -629,14 +684,12 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
       if (rc == MUON_OK) rc = encode_map(&B.x_b64[p], xb, B.n, B.m, B.chunk, B.ldx, B.x_stride, 64, 64, true);
       if (rc == MUON_OK) rc = encode_map(&B.x_e[p], xb, B.n, B.m, B.chunk, B.ldx, B.x_stride, 64, 32, true);
     }
-    void* ab = ctx->ws + B.off_a;
-    void* bb = ctx->ws + B.off_b;
-    if (rc == MUON_OK) rc = encode_map(&B.a_op, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 128, true);
-    if (rc == MUON_OK) rc = encode_map(&B.b_op, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 128, true);
-    if (rc == MUON_OK) rc = encode_map(&B.a_b64, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 64, true);
-    if (rc == MUON_OK) rc = encode_map(&B.b_b64, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 64, true);
-    if (rc == MUON_OK) rc = encode_map(&B.a_e, ab, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 32, true);
-    if (rc == MUON_OK) rc = encode_map(&B.b_e, bb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 32, true);
+    for (int i = 0; i < (B.pair_fold ? 4 : 2) && rc == MUON_OK; ++i) {
+      void* sb = ctx->ws + B.off_s[i];
+      rc = encode_map(&B.s_op[i], sb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 128, true);
+      if (rc == MUON_OK) rc = encode_map(&B.s_b64[i], sb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 64, true);
+      if (rc == MUON_OK) rc = encode_map(&B.s_e[i], sb, B.m, B.m, B.chunk, B.lda, B.a_stride, 64, 32, true);
+    }
     if (rc != MUON_OK) { delete ctx; return rc; }
   }
   ce = cudaMemset(ctx->ws + ctx->sizes.off_status, 0, sizeof(DevStatus));
@@ -729,12 +782,8 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
   ++launches;
 
   int cur = 0;
-  for (int it = 0; it < hp->ns_steps; ++it) {
-    const bool first_it = (it == 0), last_it = (it == hp->ns_steps - 1);
-    const int nxt = cur ^ 1;
-    const float co_a = hp->coeffs ? hp->coeffs[3 * it] : hp->a;
-    const float co_b = hp->coeffs ? hp->coeffs[3 * it + 1] : hp->b;
-    const float co_c = hp->coeffs ? hp->coeffs[3 * it + 2] : hp->c;
+  int a_last = 0, b_last = 1;
+  auto base_params = [&]() {
     GemmParams P{};
     P.descs = descs;
     P.scal = scal;
@@ -748,13 +797,16 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.tiles_t = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles_t);
     P.upd_scale = upd_scale;
     P.decay = decay;
-
-    // A = X X^T (first iteration: times s^2, the deferred normalisation)
-    P.map_a = B.x_op[cur];
-    P.map_a64 = B.x_b64[cur];  // unused
-    P.map_b = B.x_b64[cur];
-    P.map_in = B.a_e;  // unused
-    P.map_out = B.a_e;
+    return P;
+  };
+  // S[out] = X X^T (first iteration: times s^2, the deferred normalisation)
+  auto gram = [&](int x, int out, bool first_it) {
+    GemmParams P = base_params();
+    P.map_a = B.x_op[x];
+    P.map_a64 = B.x_b64[x];  // unused
+    P.map_b = B.x_b64[x];
+    P.map_in = B.s_e[out];  // unused
+    P.map_out = B.s_e[out];
     P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
     P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
     P.k = B.n;
@@ -764,34 +816,42 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.scale_kind = first_it ? 1 : 0;
     P.last = 0;
     P.c_acc = 1.f; P.c_in = 0.f; P.diag_add = 0.f;
-    { LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
-    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
+    LaunchTimer lt(ctx, stream, MUON_KERNEL_GRAM);
     ++launches;
-
-    // B = b*A + c*A*A  (A symmetric, kept as its upper blocks)
-    P.map_a = B.a_op;
-    P.map_a64 = B.a_b64;
-    P.map_b = B.a_b64;
-    P.map_in = B.a_e;
-    P.map_out = B.b_e;
+    return launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream);
+  };
+  // S[out] = c_acc * S[left] S[right] + c_in * S[in] + diag * I for symmetric,
+  // commuting operands kept as their upper blocks (in < 0: no input tile)
+  auto sym_product = [&](int left, int right, int in, int out, float c_acc, float c_in, float diag) {
+    GemmParams P = base_params();
+    P.map_a = B.s_op[left];
+    P.map_a64 = B.s_b64[left];
+    P.map_b = B.s_b64[right];
+    P.map_in = B.s_e[in < 0 ? out : in];
+    P.map_out = B.s_e[out];
+    P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
+    P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
     P.k = B.m;
-    P.a_sym = 1; P.b_sym = 1;
-    P.has_in = 1;
+    P.out_cols = B.m;
+    P.symmetric = 1; P.a_sym = 1; P.b_sym = 1; P.b_mn_major = 0;
+    P.has_in = in < 0 ? 0 : 1;
     P.scale_kind = 0;
-    P.c_acc = co_c; P.c_in = co_b;
-    P.diag_add = B.fold_identity ? co_a : 0.f;
-    { LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY); ce = launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream); }
-    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
+    P.last = 0;
+    P.c_acc = c_acc; P.c_in = in < 0 ? 0.f : c_in; P.diag_add = diag;
+    LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY);
     ++launches;
-
-    // X' = a*X + B X (first iteration: times s); the last iteration updates W
-    // in its epilogue when every W of the bucket is TMA-addressable bf16
-    const bool fuse = last_it && fused_update;
-    P.map_a = B.b_op;
-    P.map_a64 = B.b_b64;
-    P.map_b = B.x_b64[cur];
-    P.map_in = B.x_e[cur];
-    P.map_out = B.x_e[nxt];
+    return launch_ns_gemm(P, B.sym_acc_cols, ctx->max_clusters, stream);
+  };
+  // X[nxt] = co_a * X[cur] + S[s] X[cur] (co_a * X only when a*I is not folded into
+  // S; first iteration: times s); the last iteration updates W in its epilogue
+  // when every W of the bucket is TMA-addressable bf16
+  auto combine = [&](int s_buf, int x_cur, int x_nxt, bool first_it, bool fuse, float co_a) {
+    GemmParams P = base_params();
+    P.map_a = B.s_op[s_buf];
+    P.map_a64 = B.s_b64[s_buf];
+    P.map_b = B.x_b64[x_cur];
+    P.map_in = B.x_e[x_cur];
+    P.map_out = B.x_e[x_nxt];
     P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles);
     P.tiles_per_matrix = static_cast<int>(B.comb_tiles.size());
     P.k = B.m;
@@ -802,10 +862,52 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.last = fuse ? 1 : 0;
     P.c_acc = 1.f; P.c_in = B.fold_identity ? 0.f : co_a;
     P.diag_add = 0.f;
-    { LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB); ce = launch_ns_gemm(P, B.comb_acc_cols, ctx->max_clusters, stream); }
-    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
+    LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB);
     ++launches;
+    return launch_ns_gemm(P, B.comb_acc_cols, ctx->max_clusters, stream);
+  };
+  auto coef = [&](int it, int which) {
+    return hp->coeffs ? hp->coeffs[3 * it + which] : (which == 0 ? hp->a : (which == 1 ? hp->b : hp->c));
+  };
+  for (int it = 0; it < hp->ns_steps;) {
+    const bool first_it = (it == 0);
+    const bool pair = B.pair_fold && it + 1 < hp->ns_steps;
+    const bool last_it = it + (pair ? 2 : 1) == hp->ns_steps;
+    const int nxt = cur ^ 1;
+    const float fold_a = B.fold_identity ? coef(it, 0) : 0.f;
+    // A = X X^T;  B' = b*A + c*A*A (+ a*I)
+    ce = gram(cur, 0, first_it);
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gram kernel launch: %s", cudaGetErrorString(ce));
+    ce = sym_product(0, 0, 0, 1, coef(it, 2), coef(it, 1), fold_a);
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
+    int s_comb = 1;
+    a_last = 0;
+    b_last = 1;
+    if (pair) {
+      // the next iteration without X: A' = B'^2 A, B'' = b'*A' + c'*A'^2 + a'*I, then B'' B'
+      // (a product of two different matrices leaves diagonal blocks whose triangles
+      // differ by rounding: they are made equal before anything reads them)
+      auto symmetrise = [&](int buf) {
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY);
+        ++launches;
+        return launch_symmetrise_diag(reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_s[buf]),
+                                      static_cast<long long>(B.a_stride), B.lda, B.m, count, stream);
+      };
+      ce = sym_product(1, 1, -1, 2, 1.f, 0.f, 0.f);
+      if (ce == cudaSuccess) ce = sym_product(2, 0, -1, 3, 1.f, 0.f, 0.f);
+      if (ce == cudaSuccess) ce = symmetrise(3);
+      if (ce == cudaSuccess) ce = sym_product(3, 3, 3, 2, coef(it + 1, 2), coef(it + 1, 1), coef(it + 1, 0));
+      if (ce == cudaSuccess) ce = sym_product(2, 1, -1, 0, 1.f, 0.f, 0.f);
+      if (ce == cudaSuccess) ce = symmetrise(0);
+      if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
+      s_comb = 0;
+      a_last = 3;
+      b_last = 2;
+    }
+    ce = combine(s_comb, cur, nxt, first_it, last_it && fused_update, coef(it, 0));
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "combine kernel launch: %s", cudaGetErrorString(ce));
     cur = nxt;
+    it += pair ? 2 : 1;
   }
   {
     // Update RMS for logging (Algorithm 1, returned value) and, when the
@@ -845,6 +947,8 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
   }
   ctx->x0_buf[b] = 0;
   ctx->xlast_buf[b] = cur;
+  ctx->a_last_buf[b] = a_last;
+  ctx->b_last_buf[b] = b_last;
   *launch_counter += launches;
   return MUON_OK;
 }
@@ -1085,11 +1189,11 @@ int muon_debug_read(muon_ctx* ctx, int matrix_index, int which, void* dst_host, 
       rows = B.m; cols = B.n; ld = B.ldx;
       break;
     case MUON_TAP_A:
-      src = ctx->ws + B.off_a + static_cast<size_t>(pos) * B.a_stride * 2;
+      src = ctx->ws + B.off_s[ctx->a_last_buf[b]] + static_cast<size_t>(pos) * B.a_stride * 2;
       rows = B.m; cols = B.m; ld = B.lda;
       break;
     case MUON_TAP_B:
-      src = ctx->ws + B.off_b + static_cast<size_t>(pos) * B.a_stride * 2;
+      src = ctx->ws + B.off_s[ctx->b_last_buf[b]] + static_cast<size_t>(pos) * B.a_stride * 2;
       rows = B.m; cols = B.m; ld = B.lda;
       break;
     default:

@@ -380,7 +380,38 @@ sumsq_x_kernel(const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx,
   }
 }
 
+// Makes the 128 x 128 diagonal blocks of a symmetric buffer symmetric bit for
+// bit: element (r, c) below the diagonal takes the bits of (c, r).  The product
+// kernels form a diagonal block in full, so for a product of two different
+// matrices its two triangles differ by rounding; the consumers read the block
+// both ways round, and the polynomial of the next iteration, whose terms nearly
+// cancel, would magnify the difference.  One CTA per (block, matrix).
+__global__ void __launch_bounds__(256)
+symmetrise_diag_kernel(__nv_bfloat16* __restrict__ s, long long stride, int lda, int m) {
+  __shared__ unsigned short tile[128][130];
+  unsigned short* base = reinterpret_cast<unsigned short*>(s) + blockIdx.y * stride;
+  const int d0 = blockIdx.x * 128;
+  const int size = min(128, m - d0);
+  for (int idx = threadIdx.x; idx < size * 128; idx += blockDim.x) {
+    const int r = idx >> 7, c = idx & 127;
+    if (c < size && c > r) tile[r][c] = base[static_cast<long long>(d0 + r) * lda + d0 + c];
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < size * 128; idx += blockDim.x) {
+    const int r = idx >> 7, c = idx & 127;
+    if (c < r) base[static_cast<long long>(d0 + r) * lda + d0 + c] = tile[c][r];
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_symmetrise_diag(__nv_bfloat16* s, long long stride, int lda, int m, int count,
+                                   cudaStream_t stream) {
+  if (count == 0) return cudaSuccess;
+  symmetrise_diag_kernel<<<dim3(static_cast<unsigned>((m + 127) / 128), static_cast<unsigned>(count)), 256, 0,
+                           stream>>>(s, stride, lda, m);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_rms_finalise(const float* partials, int per_matrix, int count, float factor,
                                 const MatDesc* descs, const MatScal* scal, bool use_inv_norm, float rms_target,

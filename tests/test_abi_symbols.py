@@ -92,3 +92,32 @@ def test_bucket_plan_groups_by_sides_and_dtypes_on_the_host():
         for j in range(len(keys)):
             assert (bucket_of[i] == bucket_of[j]) == (keys[i] == keys[j])
     assert b.muon_plan_buckets(shapes) == (bucket_of, n)
+
+
+def test_planned_flops_follow_the_pairing_policy_on_the_host():
+    """muon_plan_flops: 3 m^2 n + m^3 per iteration as the algorithmic count; the
+    planned count replaces every two iterations of a wide matrix by
+    3 m^2 n + 5 m^3; the knob switches the pairing off and on."""
+    from paper_2502_16982_b200 import binding as b
+
+    prev = b.muon_debug_set_pair_fold(0)
+    try:
+        one = lambda m, n: 3.0 * m * m * n + float(m) ** 3
+        two = lambda m, n: 3.0 * m * m * n + 5.0 * float(m) ** 3
+        alg, planned = b.muon_plan_flops([(2048, 8192, 2), (1408, 2048, 3), (8192, 2048, 1), (128, 4096, 1)], 5)
+        assert alg == 5 * (3 * one(2048, 8192) + 3 * one(1408, 2048) + one(128, 4096))
+        # wide and at least 256 rows: two pairs and one single; the others plain
+        assert planned == 3 * (2 * two(2048, 8192) + one(2048, 8192)) + 5 * (3 * one(1408, 2048) + one(128, 4096))
+        b.muon_debug_set_pair_fold(1)
+        assert b.muon_plan_flops([(2048, 8192, 2)], 5) == (10 * one(2048, 8192), 10 * one(2048, 8192))
+        b.muon_debug_set_pair_fold(2)
+        assert b.muon_plan_flops([(1408, 2048, 1)], 4)[1] == 2 * two(1408, 2048)
+        # pairs keep two more symmetric buffers per matrix
+        BF = b.MUON_DTYPE_BF16
+        shapes = b.shape_only_groups([(512, 2048, 4, BF, BF)])
+        paired_bytes = b.muon_workspace_bytes(shapes, 1)
+        b.muon_debug_set_pair_fold(1)
+        plain_bytes = b.muon_workspace_bytes(shapes, 1)
+        assert paired_bytes - plain_bytes >= 2 * 4 * 512 * 512 * 2
+    finally:
+        b.muon_debug_set_pair_fold(prev)

@@ -454,6 +454,55 @@ def test_owner_computes_shards_give_the_single_context_bits():
         shard.close()
 
 
+@pytest.fixture
+def pair_fold_knob():
+    b = _binding()
+    prev = b.muon_debug_set_pair_fold(0)
+    yield b
+    b.muon_debug_set_pair_fold(prev)
+
+
+@pytest.mark.parametrize("wdt", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("rows,cols,ns_steps", [(256, 512, 5), (512, 256, 5), (264, 1000, 5), (1100, 392, 5),
+                                               (256, 640, 4), (640, 256, 2), (392, 1100, 3)])
+def test_iterations_taken_in_pairs_match_the_oracle(rows, cols, ns_steps, wdt, pair_fold_knob):
+    """Wide matrices take two iterations per pass over X (A' = B'^2 A,
+    X'' = B'' B' X; Eq. 2 rearranged): same tolerance against the plain fp64
+    iteration, for both orientations, ragged sizes, an odd and an even number of
+    iterations (the last one alone, or the last two as a pair that updates W in
+    its epilogue), with the tap on O and without."""
+    b = pair_fold_knob
+    alg, planned = b.muon_plan_flops([(rows, cols, 3)], ns_steps)
+    assert planned < alg  # the default plan pairs these shapes
+    sp = wl.GroupSpec(rows, cols, 3, wdt, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True)
+    case = Case([sp], seed=rows + 3 * cols)
+    try:
+        hp = default_hp(lr=1e-2, wd=0.05, ns_steps=ns_steps)
+        check_step(case, hp, check_o=True)
+        plain_launches = 2 + 3 * ns_steps + 3   # momentum, norm, three products per iteration, two-pass update
+        assert case.ctx.muon_last_launch_count() > plain_launches
+        check_step(case, hp)
+    finally:
+        case.close()
+
+
+def test_paired_and_plain_sequences_agree_within_tolerance(pair_fold_knob):
+    """The same bucket stepped with the pairing off and forced on: both within
+    the Newton-Schulz tolerance of the oracle, hence of each other twice over."""
+    b = pair_fold_knob
+    sp = wl.GroupSpec(320, 704, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)
+    outs = []
+    for mode in (1, 2):
+        b.muon_debug_set_pair_fold(mode)
+        case = Case([sp], seed=44)
+        try:
+            check_step(case, default_hp(lr=1e-2), check_o=True)
+            outs.append(f64(case.ctx.muon_debug_read(0, b.MUON_TAP_X, 320, 704)))
+        finally:
+            case.close()
+    assert 0 < rel(outs[1], outs[0]) <= 2 * TOL_NS
+
+
 def test_bucket_by_bucket_step_gives_muon_step_bits():
     """muon_step_bucket over every bucket, in reverse order, is one muon_step:
     buckets are independent, and the numbering is muon_plan_buckets' (the two
