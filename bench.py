@@ -292,6 +292,9 @@ def main():
         torch.cuda.synchronize(dev)
 
     alg_flops, dense_flops = wl.ns_flops(specs, hp.ns_steps)
+    # what the launch sequence asks of the tensor cores: less than the algorithmic count
+    # where the library takes two iterations per pass over X (wide matrices)
+    _, planned_flops = binding.muon_plan_flops([(s.rows, s.cols, s.count) for s in specs], hp.ns_steps)
     sbytes = wl.stream_bytes(specs)
 
     # ---- device-resident timing ------------------------------------------------
@@ -374,6 +377,9 @@ def main():
             "dense_equivalent_tflops": dense_flops * args.steps / (gemm_ms * 1e-3) / 1e12,
             "avg_launch_ms": gemm_ms / gemm_launches,
             "flops_per_launch": alg_flops * args.steps / gemm_launches,
+            "planned_tflops": planned_flops * args.steps / (gemm_ms * 1e-3) / 1e12,
+            "frac_planned": planned_flops * args.steps / (gemm_ms * 1e-3) / 1e12 / peak,
+            "planned_over_algorithmic_flops": planned_flops / alg_flops,
             "traffic": None,
         }
         if args.config == 3 and hp.ns_steps == 5:
@@ -412,12 +418,15 @@ def main():
             ms = e0.elapsed_time(e1) / args.steps
             g_ms = sum(pr[k][0] for k in ("gram", "poly", "comb")) / args.steps
             fl, _ = wl.ns_flops([sp], hp.ns_steps)
+            _, fl_planned = binding.muon_plan_flops([(sp.rows, sp.cols, sp.count)], hp.ns_steps)
             m_, n_ = min(sp.rows, sp.cols), max(sp.rows, sp.cols)
             blocks, pairs = -(-m_ // 128), -(-(-(-m_ // 128)) // 2)
             shapes.append({"shape": "%dx%d" % (sp.rows, sp.cols), "ms_per_step": ms,
                            "step_tflops": fl / (ms * 1e-3) / 1e12,
                            "gemm_tflops": fl / (g_ms * 1e-3) / 1e12,
                            "gemm_frac_of_measured_sustained": fl / (g_ms * 1e-3) / 1e12 / float(peaks.get("bf16_tflops_sustained", 1400.0)),
+                           "gemm_planned_tflops": fl_planned / (g_ms * 1e-3) / 1e12,
+                           "iterations_in_pairs": fl_planned < fl,
                            "row_blocks": blocks, "cta_pairs_per_column_tile": pairs})
             one.muon_destroy()
         ctx = binding.MuonContext(groups)

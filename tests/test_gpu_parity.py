@@ -385,6 +385,13 @@ def test_coefficient_schedule():
         check_step(case, default_hp(lr=1e-2, ns_steps=3, coeffs=sched))
     finally:
         case.close()
+    # a wide bucket takes the first two steps as a pair: each keeps its own triple
+    case = Case([wl.GroupSpec(256, 768, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)], seed=47)
+    try:
+        assert _binding().muon_plan_flops([(256, 768, 2)], 3)[1] < _binding().muon_plan_flops([(256, 768, 2)], 3)[0]
+        check_step(case, default_hp(lr=1e-2, ns_steps=3, coeffs=sched), check_o=True)
+    finally:
+        case.close()
     with pytest.raises(_binding().MuonError):
         default_hp(ns_steps=5, coeffs=sched).to_c()
 

@@ -418,3 +418,27 @@ def test_bf16_storage_model_is_the_iteration_with_rounding_only():
     assert np.allclose(orc.newton_schulz_bf16_storage(G.T, 1e-7, 5), mod.T, rtol=0, atol=0)
     x0 = orc.newton_schulz_bf16_storage(G, 0.0, 0)
     assert np.allclose(x0, orc.round_to_bf16(G) / np.linalg.norm(G), rtol=1e-15)
+
+
+@pytest.mark.parametrize("rows,cols", [(6, 20), (12, 12), (9, 40)])
+def test_two_iterations_equal_one_pass_with_the_product_of_their_polynomials(rows, cols):
+    """Eq. 2 is X_{k+1} = P_k X_k with P_k = a I + b A_k + c A_k^2, A_k = X_k X_k^T.
+    P_k is a polynomial in A_k, so A_{k+1} = P_k A_k P_k = P_k^2 A_k, and two
+    iterations are X_{k+2} = P_{k+1} P_k X_k with P_{k+1} formed from A_{k+1}
+    alone.  The GPU path uses this for wide matrices; here the oracle's plain
+    iteration is the reference, with a different coefficient triple per
+    iteration so that a swapped pair of triples would show."""
+    rng = np.random.default_rng(rows * 100 + cols)
+    X0 = orc.frobenius_normalise(rng.standard_normal((rows, cols)), 0.0)[1]
+    coeffs = [(3.4445, -4.7750, 2.0315), (3.0, -4.0, 1.9), (2.5, -3.0, 1.5), (3.4445, -4.7750, 2.0315)]
+    ref = orc.newton_schulz(X0, 4, coeffs=coeffs)
+    I = np.eye(rows)
+    X = X0
+    for k in (0, 2):
+        (a1, b1, c1), (a2, b2, c2) = coeffs[k], coeffs[k + 1]
+        A = X @ X.T
+        P1 = a1 * I + b1 * A + c1 * (A @ A)
+        A1 = P1 @ P1 @ A
+        P2 = a2 * I + b2 * A1 + c2 * (A1 @ A1)
+        X = (P2 @ P1) @ X
+    assert np.linalg.norm(X - ref) <= 1e-11 * np.linalg.norm(ref)
