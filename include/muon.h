@@ -190,7 +190,7 @@ int muon_plan_buckets(const muon_group* groups, int n_groups, int* bucket_out, i
  * Newton-Schulz FLOPs of one step over these groups (pure host computation):
  * *algorithmic_out is Eq. 2 counted with the symmetric products halved,
  * ns_steps * (3 m^2 n + m^3) per matrix; *planned_out is what the planner's
- * launch sequence asks of the tensor cores, which is less where it takes the
+ * launch sequence asks of the tensor cores, which is less where it takes
  * iterations two at a time (3 m^2 n + 5 m^3 per pair; see
  * muon_debug_set_pair_fold).  Neither counts tile padding.
  */
@@ -322,14 +322,19 @@ int muon_debug_wait_expiry(muon_ctx* ctx, void* stream, int matrix_index, unsign
 size_t muon_debug_set_chunk_bytes(size_t bytes);
 
 /*
- * Test knob: how the planner chooses between the plain iteration sequence and
- * taking the iterations two at a time (Eq. 2 gives X_{k+1} = P_k X_k with
- * P_k = a*I + b*A_k + c*A_k^2, so A_{k+1} = P_k^2 A_k and X_{k+2} = P_{k+1} P_k X_k
- * need no pass over X for every second iteration).  0: by shape (the default:
- * from 256 rows and a long side of at least twice the short side), 1: never,
- * 2: whenever the short side is at least 16.  Process-wide, read by
- * muon_workspace_bytes and muon_init like the chunk bound.  Returns the previous
- * mode; a value outside 0..2 only queries.
+ * Knob: where the planner takes two iterations per pass over X (Eq. 2 gives
+ * X_{k+1} = P_k X_k with P_k = a*I + b*A_k + c*A_k^2, so A_{k+1} = P_k^2 A_k and
+ * X_{k+2} = P_{k+1} P_k X_k need no Gram product and no combine for the second
+ * iteration of a pair).  0 (default): the first two iterations, for matrices
+ * of at least 256 rows whose long side is at least 1.25 x the short side (as
+ * accurate as the plain sequence in bf16, and fewer FLOPs); 1: never; 2: the
+ * first two iterations whenever the short side is at least 16; 3: as 0, and
+ * every further pair too when the long side is at least twice the short side
+ * (faster, up to twice the plain sequence's rounding error); 4: every pair
+ * whenever the short side is at least 16.  Process-wide, read by
+ * muon_workspace_bytes, muon_plan_flops and muon_init (a context keeps the
+ * plan it was created with).  Returns the previous mode; a value outside 0..4
+ * only queries.
  */
 int muon_debug_set_pair_fold(int mode);
 

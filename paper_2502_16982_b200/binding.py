@@ -293,8 +293,10 @@ def muon_plan_flops(shapes, ns_steps: int = 5):
 
 
 def muon_debug_set_pair_fold(mode: int) -> int:
-    """Test knob: 0 = iterations taken in pairs by shape (default), 1 = never,
-    2 = whenever the short side is at least 16.  Returns the previous mode."""
+    """Where two iterations are taken per pass over X: 0 = the first two, by
+    shape (default), 1 = never, 2 = the first two whenever the short side is at
+    least 16, 3 = every pair for wide matrices, 4 = every pair whenever the
+    short side is at least 16.  Returns the previous mode."""
     return lib().muon_debug_set_pair_fold(int(mode))
 
 

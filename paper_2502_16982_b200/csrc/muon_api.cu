@@ -68,21 +68,35 @@ constexpr int kChunkCountMax = 4096;
 // Two iterations per pass over X.  With P_k = a*I + b*A_k + c*A_k^2 (symmetric, a
 // polynomial in A_k = X_k X_k^T) Eq. 2 reads X_{k+1} = P_k X_k, hence
 //   A_{k+1} = P_k A_k P_k = P_k^2 A_k   and   X_{k+2} = (P_{k+1} P_k) X_k:
-// the Gram product and the combine (m^2 n each way) of every second iteration
+// the Gram product and the combine (m^2 n each way) of the second iteration
 // are replaced by three more symmetric m x m x m products, 3 m^2 n + 5 m^3
-// instead of 6 m^2 n + 2 m^3 for the two iterations.  That pays when the long
-// side is well above the short side; with bf16 storage the result is as close
-// to the exact iteration as the plain sequence for n >= 3 m and within 1.4 x of
-// its distance at n = 2 m from 256 rows on (bf16 storage model on the CPU), and
-// further off for small or near-square matrices, which keep the plain sequence.
+// instead of 6 m^2 n + 2 m^3 for the two iterations, which pays when the long
+// side is above the short side.
+// By default only the first two iterations are taken as a pair: with bf16
+// storage that is as close to the exact iteration as the plain sequence from
+// 256 rows on, for every spectrum tried on a CPU model (closer for spectra with
+// a wide range, where rounding X_1 to bf16 is what loses the small singular
+// values).  Later pairs work near the band, where the terms of P nearly cancel:
+// they cost accuracy (up to twice the plain sequence's distance on decaying
+// spectra) and are only taken on request (pair-fold mode 3).
 constexpr int kPairFoldMinRows = 256;
-constexpr double kPairFoldMinAspect = 2.0;
-int g_pair_fold_mode = 0;  // 0: by shape, 1: never, 2: whenever a*I is folded; see muon_debug_set_pair_fold
+constexpr double kPairFirstMinAspect = 1.25;
+constexpr double kPairAllMinAspect = 2.0;
+// 0: first pair by shape, 1: never, 2: first pair whenever a*I is folded,
+// 3: every pair by shape, 4: every pair whenever a*I is folded; see muon_debug_set_pair_fold
+int g_pair_fold_mode = 0;
 
-bool plan_pair_fold(int m, int n, bool fold_identity) {
-  if (!fold_identity || g_pair_fold_mode == 1) return false;
-  if (g_pair_fold_mode == 2) return true;
-  return m >= kPairFoldMinRows && static_cast<double>(n) >= kPairFoldMinAspect * m;
+// How many leading pairs of `ns_steps` iterations are taken two per pass in pair-fold mode `mode`.
+int plan_pairs(int mode, int m, int n, bool fold_identity, int ns_steps) {
+  if (!fold_identity || mode == 1 || ns_steps < 2) return 0;
+  const bool big = m >= kPairFoldMinRows;
+  switch (mode) {
+    case 0: return big && n >= kPairFirstMinAspect * m ? 1 : 0;
+    case 2: return 1;
+    case 3: return big && n >= kPairAllMinAspect * m ? ns_steps / 2 : (big && n >= kPairFirstMinAspect * m ? 1 : 0);
+    case 4: return ns_steps / 2;
+    default: return 0;
+  }
 }
 
 struct MatRef {
@@ -102,7 +116,8 @@ struct Bucket {
   bool fused_update;          // every W is bf16 and TMA-addressable: update W in the last epilogue
   bool stream_tma;            // every G and M is TMA-addressable: TMA-pipelined momentum kernel
   bool fold_identity;         // keep B' = B + a*I so that the combine is the single product B' X
-  bool pair_fold;             // take two iterations per pass over X (see plan_pair_fold)
+  bool pair_fold;             // some iterations are taken two per pass over X (see plan_pairs)
+  int pair_mode;              // the pair-fold mode the plan was made with
   // workspace offsets (bytes) of the chunk buffers
   // off_s: the symmetric m x m buffers (A and B; two more when iterations are taken in pairs)
   size_t off_x[2], off_s[4], off_partials, off_scal, off_rms_partials, off_factors;
@@ -278,7 +293,8 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     // Folding a*X into the product rounds B_ii + a to bf16; that is the smaller
     // error from 16 rows up (measured with a bf16 storage model) and the larger one below.
     B.fold_identity = B.m >= 16;
-    B.pair_fold = plan_pair_fold(B.m, B.n, B.fold_identity);
+    B.pair_fold = plan_pairs(g_pair_fold_mode, B.m, B.n, B.fold_identity, 64) > 0;
+    B.pair_mode = g_pair_fold_mode;
     const int n_sym = B.pair_fold ? 4 : 2;
     const size_t per_mat = 2 * B.x_stride * 2 + n_sym * B.a_stride * 2;
     size_t chunk = std::max<size_t>(1, g_chunk_bytes_max / per_mat);
@@ -506,7 +522,7 @@ int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_byt
 
 int muon_debug_set_pair_fold(int mode) {
   const int prev = g_pair_fold_mode;
-  if (mode >= 0 && mode <= 2) g_pair_fold_mode = mode;
+  if (mode >= 0 && mode <= 4) g_pair_fold_mode = mode;
   return prev;
 }
 
@@ -536,8 +552,7 @@ int muon_plan_flops(const muon_group* groups, int n_groups, int ns_steps, double
     const double m = std::min(groups[g].rows, groups[g].cols), n = std::max(groups[g].rows, groups[g].cols);
     const double one = 3.0 * m * m * n + m * m * m;     // Gram (half), polynomial (half), combine
     const double two = 3.0 * m * m * n + 5.0 * m * m * m;  // one Gram, five symmetric m^3 products, one combine
-    const bool pairs = plan_pair_fold(static_cast<int>(m), static_cast<int>(n), m >= 16);
-    const int n_pairs = pairs ? ns_steps / 2 : 0;
+    const int n_pairs = plan_pairs(g_pair_fold_mode, static_cast<int>(m), static_cast<int>(n), m >= 16, ns_steps);
     alg += groups[g].count * ns_steps * one;
     planned += groups[g].count * (n_pairs * two + (ns_steps - 2 * n_pairs) * one);
   }
@@ -869,9 +884,12 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
   auto coef = [&](int it, int which) {
     return hp->coeffs ? hp->coeffs[3 * it + which] : (which == 0 ? hp->a : (which == 1 ? hp->b : hp->c));
   };
+  // the mode the plan was made with, whatever the knob says now
+  int pairs_left = B.pair_fold ? plan_pairs(B.pair_mode, B.m, B.n, B.fold_identity, hp->ns_steps) : 0;
   for (int it = 0; it < hp->ns_steps;) {
     const bool first_it = (it == 0);
-    const bool pair = B.pair_fold && it + 1 < hp->ns_steps;
+    const bool pair = pairs_left > 0 && it + 1 < hp->ns_steps;
+    if (pair) --pairs_left;
     const bool last_it = it + (pair ? 2 : 1) == hp->ns_steps;
     const int nxt = cur ^ 1;
     const float fold_a = B.fold_identity ? coef(it, 0) : 0.f;

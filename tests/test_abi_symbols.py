@@ -104,14 +104,23 @@ def test_planned_flops_follow_the_pairing_policy_on_the_host():
     try:
         one = lambda m, n: 3.0 * m * m * n + float(m) ** 3
         two = lambda m, n: 3.0 * m * m * n + 5.0 * float(m) ** 3
-        alg, planned = b.muon_plan_flops([(2048, 8192, 2), (1408, 2048, 3), (8192, 2048, 1), (128, 4096, 1)], 5)
-        assert alg == 5 * (3 * one(2048, 8192) + 3 * one(1408, 2048) + one(128, 4096))
-        # wide and at least 256 rows: two pairs and one single; the others plain
-        assert planned == 3 * (2 * two(2048, 8192) + one(2048, 8192)) + 5 * (3 * one(1408, 2048) + one(128, 4096))
+        shapes = [(2048, 8192, 2), (1408, 2048, 3), (8192, 2048, 1), (128, 4096, 1), (2048, 2048, 2)]
+        alg, planned = b.muon_plan_flops(shapes, 5)
+        assert alg == 5 * (3 * one(2048, 8192) + 3 * one(1408, 2048) + one(128, 4096) + 2 * one(2048, 2048))
+        # default: from 256 rows and a long side of 1.25 x the short side, the first two iterations
+        first_pair = lambda m, n: two(m, n) + 3 * one(m, n)
+        assert planned == 3 * first_pair(2048, 8192) + 3 * first_pair(1408, 2048) + 5 * (one(128, 4096) + 2 * one(2048, 2048))
         b.muon_debug_set_pair_fold(1)
         assert b.muon_plan_flops([(2048, 8192, 2)], 5) == (10 * one(2048, 8192), 10 * one(2048, 8192))
         b.muon_debug_set_pair_fold(2)
+        assert b.muon_plan_flops([(64, 64, 1)], 4)[1] == two(64, 64) + 2 * one(64, 64)
+        b.muon_debug_set_pair_fold(3)   # wide: every pair; the others as by default
+        assert b.muon_plan_flops([(2048, 8192, 1)], 5)[1] == 2 * two(2048, 8192) + one(2048, 8192)
+        assert b.muon_plan_flops([(1408, 2048, 1)], 5)[1] == first_pair(1408, 2048)
+        b.muon_debug_set_pair_fold(4)
         assert b.muon_plan_flops([(1408, 2048, 1)], 4)[1] == 2 * two(1408, 2048)
+        assert b.muon_plan_flops([(1408, 2048, 1)], 1)[1] == one(1408, 2048)
+        b.muon_debug_set_pair_fold(0)
         # pairs keep two more symmetric buffers per matrix
         BF = b.MUON_DTYPE_BF16
         shapes = b.shape_only_groups([(512, 2048, 4, BF, BF)])
