@@ -54,7 +54,7 @@ WORKLOAD_NAMES = {
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/, taken on 64 matrices of the expert-bucket shapes; it scales with the matrix count.
-NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": 8.236e9, "gemm_launches_per_step": 15,
+NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": 7.930e9, "gemm_launches_per_step": 16,
                "momentum_bytes_per_launch": 2.159e9}
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
@@ -385,7 +385,7 @@ def main():
         if args.config == 3 and hp.ns_steps == 5:
             scale = sum(s.count for s in specs) / NCU_CAPTURE["matrices"]
             roofline["traffic"] = NCU_CAPTURE["gemm_bytes_per_step"] * scale / NCU_CAPTURE["gemm_launches_per_step"]
-            roofline["traffic_note"] = "DRAM bytes per launch (average of the 15 launches of a step), scaled from a 64-matrix ncu capture"
+            roofline["traffic_note"] = "DRAM bytes per launch (average of the 16 launches of a step), scaled from a 64-matrix ncu capture"
     stream_roof = None
     if mom_launches:
         gbs = sbytes * args.steps / (mom_ms * 1e-3) / 1e9

@@ -271,9 +271,9 @@ int muon_last_launch_count(const muon_ctx* ctx);
  */
 enum {
   MUON_KERNEL_MOMENTUM = 0, /* momentum + Nesterov + sum of squares + bf16 cast */
-  MUON_KERNEL_NORM = 1,     /* norm finalisation */
+  MUON_KERNEL_NORM = 1,     /* small helpers: norm and RMS finalisation, diagonal-block symmetrise */
   MUON_KERNEL_GRAM = 2,     /* A = X X^T */
-  MUON_KERNEL_POLY = 3,     /* B = b A + c A A */
+  MUON_KERNEL_POLY = 3,     /* B = b A + c A A and the other symmetric m x m x m products */
   MUON_KERNEL_COMB = 4,     /* X' = a X + B X (last iteration: fused weight update) */
   MUON_KERNEL_UPDATE = 5,   /* separate weight update (ns_steps == 0, fp32 or unaligned W) */
   MUON_KERNEL_KINDS = 6

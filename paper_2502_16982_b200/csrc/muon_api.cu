@@ -906,7 +906,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
       // (a product of two different matrices leaves diagonal blocks whose triangles
       // differ by rounding: they are made equal before anything reads them)
       auto symmetrise = [&](int buf) {
-        LaunchTimer lt(ctx, stream, MUON_KERNEL_POLY);
+        LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);  // counted with the small helper kernels
         ++launches;
         return launch_symmetrise_diag(reinterpret_cast<__nv_bfloat16*>(ctx->ws + B.off_s[buf]),
                                       static_cast<long long>(B.a_stride), B.lda, B.m, count, stream);

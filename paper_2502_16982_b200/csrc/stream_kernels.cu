@@ -388,18 +388,38 @@ sumsq_x_kernel(const __nv_bfloat16* __restrict__ x, long long x_stride, int ldx,
 // cancel, would magnify the difference.  One CTA per (block, matrix).
 __global__ void __launch_bounds__(256)
 symmetrise_diag_kernel(__nv_bfloat16* __restrict__ s, long long stride, int lda, int m) {
-  __shared__ unsigned short tile[128][130];
+  // rows padded to 136 elements: 16-byte aligned for the vector stores, and a
+  // column walk (stride 68 words) touches every bank once
+  __shared__ __align__(16) unsigned short tile[128][136];
   unsigned short* base = reinterpret_cast<unsigned short*>(s) + blockIdx.y * stride;
   const int d0 = blockIdx.x * 128;
   const int size = min(128, m - d0);
-  for (int idx = threadIdx.x; idx < size * 128; idx += blockDim.x) {
-    const int r = idx >> 7, c = idx & 127;
-    if (c < size && c > r) tile[r][c] = base[static_cast<long long>(d0 + r) * lda + d0 + c];
+  // 8-element chunks; rows are 16-byte aligned (lda is a multiple of 64) and
+  // padded at least to the next multiple of 8 beyond m
+  for (int idx = threadIdx.x; idx < size * 16; idx += blockDim.x) {
+    const int r = idx >> 4, c0 = (idx & 15) * 8;
+    if (c0 < size && c0 + 7 >= r) {  // holds elements on or above the diagonal
+      *reinterpret_cast<uint4*>(&tile[r][c0]) =
+          *reinterpret_cast<const uint4*>(base + static_cast<long long>(d0 + r) * lda + d0 + c0);
+    }
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < size * 128; idx += blockDim.x) {
-    const int r = idx >> 7, c = idx & 127;
-    if (c < r) base[static_cast<long long>(d0 + r) * lda + d0 + c] = tile[c][r];
+  for (int idx = threadIdx.x; idx < size * 16; idx += blockDim.x) {
+    const int r = idx >> 4, c0 = (idx & 15) * 8;
+    if (c0 < size && c0 < r) {  // holds elements below the diagonal
+      unsigned short v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int c = c0 + e;
+        v[e] = c < r ? tile[c][r] : tile[r][c];
+      }
+      uint4 out;
+      out.x = v[0] | (static_cast<unsigned>(v[1]) << 16);
+      out.y = v[2] | (static_cast<unsigned>(v[3]) << 16);
+      out.z = v[4] | (static_cast<unsigned>(v[5]) << 16);
+      out.w = v[6] | (static_cast<unsigned>(v[7]) << 16);
+      *reinterpret_cast<uint4*>(base + static_cast<long long>(d0 + r) * lda + d0 + c0) = out;
+    }
   }
 }
 
