@@ -79,6 +79,7 @@ constexpr int kChunkCountMax = 4096;
 // values).  Later pairs work near the band, where the terms of P nearly cancel:
 // they cost accuracy (up to twice the plain sequence's distance on decaying
 // spectra) and are only taken on request (pair-fold mode 3).
+constexpr int kFoldIdentityMinRows = 16;  // from here on B' = B + a*I is kept and the combine is B' X
 constexpr int kPairFoldMinRows = 256;
 constexpr double kPairFirstMinAspect = 1.25;
 constexpr double kPairAllMinAspect = 2.0;
@@ -292,7 +293,7 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     B.stream_tiles = std::max(B.stream_tiles_generic, B.stream_tiles_tma);
     // Folding a*X into the product rounds B_ii + a to bf16; that is the smaller
     // error from 16 rows up (measured with a bf16 storage model) and the larger one below.
-    B.fold_identity = B.m >= 16;
+    B.fold_identity = B.m >= kFoldIdentityMinRows;
     B.pair_fold = plan_pairs(g_pair_fold_mode, B.m, B.n, B.fold_identity, 64) > 0;
     B.pair_mode = g_pair_fold_mode;
     const int n_sym = B.pair_fold ? 4 : 2;
@@ -552,7 +553,8 @@ int muon_plan_flops(const muon_group* groups, int n_groups, int ns_steps, double
     const double m = std::min(groups[g].rows, groups[g].cols), n = std::max(groups[g].rows, groups[g].cols);
     const double one = 3.0 * m * m * n + m * m * m;     // Gram (half), polynomial (half), combine
     const double two = 3.0 * m * m * n + 5.0 * m * m * m;  // one Gram, five symmetric m^3 products, one combine
-    const int n_pairs = plan_pairs(g_pair_fold_mode, static_cast<int>(m), static_cast<int>(n), m >= 16, ns_steps);
+    const int n_pairs = plan_pairs(g_pair_fold_mode, static_cast<int>(m), static_cast<int>(n),
+                                  m >= kFoldIdentityMinRows, ns_steps);
     alg += groups[g].count * ns_steps * one;
     planned += groups[g].count * (n_pairs * two + (ns_steps - 2 * n_pairs) * one);
   }
