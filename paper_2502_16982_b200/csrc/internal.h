@@ -85,6 +85,7 @@ struct GemmParams {
   int has_in;      // the epilogue reads an input tile through map_in
   int scale_kind;  // 0: none, 1: s^2 of the matrix, 2: s
   int last;        // fused weight update: W is read, updated and written back
+  int w_fp32;      // last: the weights are fp32 (maps of box {32, 32}), else bf16 (box {64, 32})
   float c_acc, c_in, diag_add;
   float upd_scale, decay;
   const MatDesc* descs;

@@ -114,7 +114,7 @@ struct Bucket {
   int stream_tiles;           // per-matrix partial sums reserved for the streaming kernels
   int stream_tiles_generic;   // tiles per matrix of the generic streaming kernel (64 x 128)
   int stream_tiles_tma;       // tiles per matrix of the TMA streaming kernel (64 x 64)
-  bool fused_update;          // every W is bf16 and TMA-addressable: update W in the last epilogue
+  bool fused_update;          // every W (and bf16 copy) is TMA-addressable: update W in the last epilogue
   bool stream_tma;            // every G and M is TMA-addressable: TMA-pipelined momentum kernel
   bool fold_identity;         // keep B' = B + a*I so that the combine is the single product B' X
   bool pair_fold;             // some iterations are taken two per pass over X (see plan_pairs)
@@ -205,6 +205,21 @@ int encode_w_map(CUtensorMap* out, void* w, int rows, int cols, long long ld) {
   return encode_map(out, w, cols, rows, 1, static_cast<int>(ld), static_cast<size_t>(rows) * ld, 64, 32, true);
 }
 
+// The same for an fp32 weight matrix: a 128-byte swizzled row holds 32 columns,
+// so the box is {32, 32} and a 64-column quarter of the epilogue takes two.
+int encode_w_map_fp32(CUtensorMap* out, void* w, int rows, int cols, long long ld) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return fail(MUON_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
+  cuuint64_t dims[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows), 1};
+  cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld) * 4, static_cast<cuuint64_t>(ld) * 4 * rows};
+  cuuint32_t box[3] = {32, 32, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, w, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(MUON_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+  return MUON_OK;
+}
+
 int validate_groups(const muon_group* groups, int n_groups, bool need_ptrs) {
   if (!groups || n_groups <= 0) return fail(MUON_ERR_INVALID_ARG, "groups is null or n_groups <= 0");
   for (int g = 0; g < n_groups; ++g) {
@@ -242,9 +257,10 @@ int validate_groups(const muon_group* groups, int n_groups, bool need_ptrs) {
   return MUON_OK;
 }
 
-// True if a bf16 weight matrix can be addressed by a TMA descriptor.
-inline bool w_tma_ok(const void* w, long long ld) {
-  return (reinterpret_cast<uintptr_t>(w) & 15) == 0 && ld % 8 == 0;
+// True if a weight matrix can be addressed by a TMA descriptor (16-byte aligned
+// base and row pitch).
+inline bool w_tma_ok(const void* w, long long ld, bool fp32) {
+  return (reinterpret_cast<uintptr_t>(w) & 15) == 0 && ld % (fp32 ? 4 : 8) == 0;
 }
 
 // Forms the shape buckets and lays out the workspace.  Deterministic in the
@@ -635,7 +651,8 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
   for (size_t b = 0; b < ctx->buckets.size(); ++b) {
     Bucket& B = ctx->buckets[b];
     std::vector<MatDesc> descs(B.mats.size());
-    B.fused_update = (B.w_dtype == MUON_DTYPE_BF16);
+    B.fused_update = true;
+    const bool w_fp32 = B.w_dtype == MUON_DTYPE_FP32;
     B.stream_tma = true;
     const long long g_es = B.g_dtype == MUON_DTYPE_FP32 ? 4 : 2;
     for (size_t i = 0; i < B.mats.size(); ++i) {
@@ -659,7 +676,9 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
       d.vec_ok = (ptr16 && G.ld_w % 8 == 0 && G.ld_g % 8 == 0 && G.ld_m % 8 == 0) ? 1 : 0;
       descs[i] = d;
       ctx->where[r.global] = std::make_pair(static_cast<int>(b), static_cast<int>(i));
-      if (!w_tma_ok(d.w, d.ld_w) || d.ld_w > (1ll << 31)) B.fused_update = false;
+      if (!w_tma_ok(d.w, d.ld_w, w_fp32) || d.ld_w > (1ll << 31)) B.fused_update = false;
+      // the epilogue writes the bf16 copy with 16-byte stores
+      if (d.w_shadow && !w_tma_ok(d.w_shadow, d.ld_ws, false)) B.fused_update = false;
       if ((reinterpret_cast<uintptr_t>(d.g) & 15) || (d.ld_g * g_es) % 16 || (reinterpret_cast<uintptr_t>(d.m) & 15) ||
           (d.ld_m * 4) % 16)
         B.stream_tma = false;
@@ -677,7 +696,8 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     if (ce == cudaSuccess && B.fused_update) {
       std::vector<CUtensorMap> wmaps(B.mats.size());
       for (size_t i = 0; i < B.mats.size() && rc == MUON_OK; ++i)
-        rc = encode_w_map(&wmaps[i], descs[i].w, descs[i].rows, descs[i].cols, descs[i].ld_w);
+        rc = w_fp32 ? encode_w_map_fp32(&wmaps[i], descs[i].w, descs[i].rows, descs[i].cols, descs[i].ld_w)
+                    : encode_w_map(&wmaps[i], descs[i].w, descs[i].rows, descs[i].cols, descs[i].ld_w);
       if (rc != MUON_OK) { delete ctx; return rc; }
       ce = cudaMemcpy(ctx->ws + B.off_wmaps, wmaps.data(), wmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice);
     }
@@ -752,7 +772,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
                                                      ? hp->scale_dim : static_cast<float>(B.n));
   const bool normalise = hp->scale_mode == MUON_SCALE_UPDATE_NORM;
   // The last epilogue updates W when every W of the bucket is TMA-addressable
-  // bf16, the update needs no whole-matrix statistic, a*X is folded into the
+  // (bf16 or fp32), the update needs no whole-matrix statistic, a*X is folded into the
   // product and the O tap is off; otherwise O is stored and a second pass applies it.
   const bool fused_update = B.fused_update && !normalise && B.fold_identity && !ctx->keep_o;
   const float upd_scale = -hp->lr * factor;
@@ -861,7 +881,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
   };
   // X[nxt] = co_a * X[cur] + S[s] X[cur] (co_a * X only when a*I is not folded into
   // S; first iteration: times s); the last iteration updates W in its epilogue
-  // when every W of the bucket is TMA-addressable bf16
+  // when every W of the bucket is TMA-addressable
   auto combine = [&](int s_buf, int x_cur, int x_nxt, bool first_it, bool fuse, float co_a) {
     GemmParams P = base_params();
     P.map_a = B.s_op[s_buf];
@@ -877,6 +897,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.has_in = (fuse || !B.fold_identity) ? 1 : 0;  // W when fused, else X for the a*X term
     P.scale_kind = first_it ? 2 : 0;
     P.last = fuse ? 1 : 0;
+    P.w_fp32 = B.w_dtype == MUON_DTYPE_FP32 ? 1 : 0;
     P.c_acc = 1.f; P.c_in = B.fold_identity ? 0.f : co_a;
     P.diag_add = 0.f;
     LaunchTimer lt(ctx, stream, MUON_KERNEL_COMB);

@@ -39,7 +39,9 @@
 //
 // Last iteration (Sec. 2.2): the entry holds the W tile,
 //   O = scale * acc,   W <- (1 - lr*wd) * W - lr * rms_scale * sqrt(max(rows, cols)) * O
-// in fp32; O itself never reaches HBM.  For a matrix stored with rows > cols
+// in fp32; O itself never reaches HBM.  (W is bf16, or fp32 in the kWFp32
+// instantiation, where an entry is two boxes of 32 fp32 columns and an optional
+// bf16 copy of the new weights is written from the registers.)  For a matrix stored with rows > cols
 // (Newton-Schulz ran on its transpose) the last product is formed transposed,
 // O^T = X^T B' with X^T read as an MN-major operand from X and the symmetric B'
 // as the other operand, so that the tile comes out in W's own orientation and
@@ -84,11 +86,13 @@ struct Barriers {
 };
 
 constexpr int kBarrierBytes = 512;
-constexpr int smem_bytes(int stages, int subs) {
-  return 1024 + stages * kStageBytes + kEpiWarps * subs * kSubBytes + kBarrierBytes;
+constexpr int kSubBytesFp32 = 2 * kSubBytes;  // the same quarter of an fp32 W: two boxes of 32 columns
+constexpr int smem_bytes(int stages, int subs, int entry_bytes = kSubBytes) {
+  return 1024 + stages * kStageBytes + kEpiWarps * subs * entry_bytes + kBarrierBytes;
 }
 static_assert(sizeof(Barriers) <= kBarrierBytes, "barrier block too large");
-static_assert(smem_bytes(5, 4) <= 232448 && smem_bytes(4, 6) <= 232448, "exceeds the 227 KiB shared-memory limit");
+static_assert(smem_bytes(5, 4) <= 232448 && smem_bytes(4, 6) <= 232448 && smem_bytes(4, 3, kSubBytesFp32) <= 232448,
+              "exceeds the 227 KiB shared-memory limit");
 static_assert(kBK == 64, "the issuer loop issues four K = 16 steps per stage");
 
 __device__ __forceinline__ void report_timeout(const GemmParams& P, int mat) {
@@ -175,15 +179,18 @@ __device__ __forceinline__ TilePlan plan_tile(const GemmParams& P, int tile, int
 
 // kAccCols: fp32 TMEM columns per accumulator stage = widest N (128 or 256).
 // kStages: depth of the operand ring; kSubsPerWarp: staging buffers per epilogue warp.
-template <int kAccCols, int kStages, int kSubsPerWarp>
+// kWFp32: the launch is a last iteration over fp32 weights (a staging buffer then
+// holds 32 rows x 64 fp32 columns as two 128-byte-swizzled boxes of 32 columns).
+template <int kAccCols, int kStages, int kSubsPerWarp, bool kWFp32 = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ns_gemm_kernel(const __grid_constant__ GemmParams P) {
+  constexpr int kEntryBytes = kWFp32 ? kSubBytesFp32 : kSubBytes;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
   uint8_t* ring = smem;
   uint8_t* s_epi = smem + kStages * kStageBytes;
-  Barriers* bars = reinterpret_cast<Barriers*>(s_epi + kEpiWarps * kSubsPerWarp * kSubBytes);
+  Barriers* bars = reinterpret_cast<Barriers*>(s_epi + kEpiWarps * kSubsPerWarp * kEntryBytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -366,7 +373,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
   } else {
     // ----------------------------------------------------------- epilogue ----
     const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the tile
-    const uint32_t my_base = ptx::smem_u32(s_epi + q * kSubsPerWarp * kSubBytes);
+    const uint32_t my_base = ptx::smem_u32(s_epi + q * kSubsPerWarp * kEntryBytes);
     unsigned long long* my_bars = bars->io_ready[q];
     // Ring of staging entries, one buffer per quarter.
     constexpr uint32_t ring_len = kSubsPerWarp;
@@ -390,15 +397,16 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       if (!pre_valid) return;
       const uint32_t e = pre_g % ring_len;
       const uint32_t bar = ptx::smem_u32(&my_bars[e]);
-      const uint32_t buf = my_base + e * kSubBytes;
+      const uint32_t buf = my_base + e * kEntryBytes;
       const int row0 = pre.ib * 128 + q * 32;
       const int col0 = pre.jb * 128 + pre.qd * 64;
       if (row0 >= pre.row_limit) {  // this warp's rows lie beyond the matrix: nothing to fetch
         ptx::mbar_arrive(bar);
       } else if (P.last) {
         // the tile is in W's own orientation (see the header): W[row0.., col0..]
-        ptx::mbar_arrive_expect_tx(bar, kSubBytes);
+        ptx::mbar_arrive_expect_tx(bar, kEntryBytes);
         ptx::tma_load_3d(buf, P.wmaps + pre.mat, col0, row0, 0, bar);
+        if (kWFp32) ptx::tma_load_3d(buf + kSubBytes, P.wmaps + pre.mat, col0 + 32, row0, 0, bar);
         ++loads_in_flight;
       } else if (P.has_in) {
         ptx::mbar_arrive_expect_tx(bar, kSubBytes);
@@ -439,7 +447,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
 
         for (int qd = cur.qd; qd < cur.q_end && ok; ++qd, ++gq) {
           const uint32_t e = gq % ring_len;
-          const uint32_t buf = my_base + e * kSubBytes;  // in / out (W on the last iteration)
+          const uint32_t buf = my_base + e * kEntryBytes;  // in / out (W on the last iteration)
           const int col0 = cur.jb * 128 + qd * 64;
           // column of this lane's row that lies on the matrix diagonal, if the quarter holds it
           const bool diag_quarter = P.diag_add != 0.f && cur.jb + (qd >> 1) == cur.ib;
@@ -482,6 +490,50 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
             };
             if (diag_quarter) combine(std::true_type{});
             else combine(std::false_type{});
+          } else if (kWFp32) {
+            // the same update on fp32 weights: 16 chunks of four columns in two boxes;
+            // the bf16 copy of the new weights, if the matrix has one, goes straight
+            // from the registers to global memory (a 128-byte run per row and quarter)
+            const MatDesc& md = P.descs[mat];
+            __nv_bfloat16* shadow = static_cast<__nv_bfloat16*>(md.w_shadow);
+            const int w_cols = md.cols;
+            const bool row_ok = row0 + lane < cur.row_limit && !sc.nonfinite;
+            __nv_bfloat16* srow = shadow == nullptr ? nullptr
+                                                    : shadow + static_cast<long long>(row0 + lane) * md.ld_ws + col0;
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {
+              uint32_t packed[4];
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const int c4 = 2 * c8 + h;
+                const uint32_t addr = buf + static_cast<uint32_t>((c4 >> 3) * kSubBytes + lane * 128 +
+                                                                  (((c4 & 7) ^ (lane & 7)) << 4));
+                uint32_t w0, w1, w2, w3;
+                lds128(addr, w0, w1, w2, w3);
+                float w[4] = {__uint_as_float(w0), __uint_as_float(w1), __uint_as_float(w2), __uint_as_float(w3)};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float o = scale * __uint_as_float(v[c4 * 4 + i]);
+                  o_sq = fmaf(o, o, o_sq);
+                  w[i] = fmaf(P.decay, w[i], P.upd_scale * o);
+                }
+                sts128(addr, __float_as_uint(w[0]), __float_as_uint(w[1]), __float_as_uint(w[2]), __float_as_uint(w[3]));
+                packed[2 * h] = pack2(w[0], w[1]);
+                packed[2 * h + 1] = pack2(w[2], w[3]);
+              }
+              if (srow != nullptr && row_ok) {
+                const int c = col0 + c8 * 8;
+                if (c + 8 <= w_cols) {
+                  *reinterpret_cast<uint4*>(srow + c8 * 8) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                } else {
+                  for (int i = 0; i < 8 && c + i < w_cols; ++i) {
+                    const uint32_t pr = packed[i >> 1];
+                    reinterpret_cast<unsigned short*>(srow + c8 * 8)[i] =
+                        static_cast<unsigned short>((i & 1) ? (pr >> 16) : (pr & 0xFFFFu));
+                  }
+                }
+              }
+            }
           } else {
             // O = scale * acc;  W <- decay * W + upd_scale * O
 #pragma unroll
@@ -507,7 +559,11 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
             if (row0 >= cur.row_limit) {
               // rows beyond the matrix: nothing to store
             } else if (P.last) {
-              if (!sc.nonfinite) ptx::tma_store_3d(P.wmaps + mat, col0, row0, 0, buf);
+              if (!sc.nonfinite) {
+                ptx::tma_store_3d(P.wmaps + mat, col0, row0, 0, buf);
+                if (kWFp32 && col0 + 32 < P.descs[mat].cols)
+                  ptx::tma_store_3d(P.wmaps + mat, col0 + 32, row0, 0, buf + kSubBytes);
+              }
             } else {
               ptx::tma_store_3d(&P.map_out, col0, row0, mat, buf);
             }
@@ -585,18 +641,19 @@ cudaError_t launch_wait_expiry_probe(DevStatus* status, int matrix_index, unsign
 
 namespace {
 
-template <int kAccCols, int kStages, int kSubs>
+template <int kAccCols, int kStages, int kSubs, bool kWFp32 = false>
 cudaError_t configure_one() {
-  return cudaFuncSetAttribute(ns_gemm_kernel<kAccCols, kStages, kSubs>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              smem_bytes(kStages, kSubs));
+  return cudaFuncSetAttribute(ns_gemm_kernel<kAccCols, kStages, kSubs, kWFp32>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              smem_bytes(kStages, kSubs, kWFp32 ? kSubBytesFp32 : kSubBytes));
 }
 
-template <int kAccCols, int kStages, int kSubs>
+template <int kAccCols, int kStages, int kSubs, bool kWFp32 = false>
 cudaError_t launch_one(const GemmParams& P, unsigned clusters, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * clusters, 1, 1);
   cfg.blockDim = dim3(kGemmThreads, 1, 1);
-  cfg.dynamicSmemBytes = smem_bytes(kStages, kSubs);
+  cfg.dynamicSmemBytes = smem_bytes(kStages, kSubs, kWFp32 ? kSubBytesFp32 : kSubBytes);
   cfg.stream = stream;
   cudaLaunchAttribute attr;
   attr.id = cudaLaunchAttributeClusterDimension;
@@ -605,7 +662,7 @@ cudaError_t launch_one(const GemmParams& P, unsigned clusters, cudaStream_t stre
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, ns_gemm_kernel<kAccCols, kStages, kSubs>, P);
+  return cudaLaunchKernelEx(&cfg, ns_gemm_kernel<kAccCols, kStages, kSubs, kWFp32>, P);
 }
 
 }  // namespace
@@ -615,6 +672,8 @@ cudaError_t gemm_configure() {
   if (e == cudaSuccess) e = configure_one<256, 4, 6>();
   if (e == cudaSuccess) e = configure_one<128, 5, 4>();
   if (e == cudaSuccess) e = configure_one<256, 5, 4>();
+  if (e == cudaSuccess) e = configure_one<128, 4, 3, true>();
+  if (e == cudaSuccess) e = configure_one<256, 4, 3, true>();
   return e;
 }
 
@@ -643,6 +702,10 @@ cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, 
   if (deep_ring) {
     if (acc_cols == 128) return launch_one<128, 5, 4>(P, clusters, stream);
     return launch_one<256, 5, 4>(P, clusters, stream);
+  }
+  if (P.last && P.w_fp32) {  // same shared memory: three staging buffers of twice the size
+    if (acc_cols == 128) return launch_one<128, 4, 3, true>(P, clusters, stream);
+    return launch_one<256, 4, 3, true>(P, clusters, stream);
   }
   if (acc_cols == 128) return launch_one<128, 4, 6>(P, clusters, stream);
   return launch_one<256, 4, 6>(P, clusters, stream);

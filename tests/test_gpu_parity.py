@@ -459,6 +459,53 @@ def test_fp32_master_weights_with_bf16_shadow():
         b.MuonContext([(wl.views(Wb), wl.views(Gd), wl.views(Md), wl.views(shadow))])
 
 
+@pytest.mark.parametrize("rows,cols", [(200, 332), (332, 200), (384, 1028)])
+@pytest.mark.parametrize("with_shadow", [False, True])
+def test_fp32_weights_updated_in_the_last_epilogue(rows, cols, with_shadow):
+    """fp32 weights that TMA can address (16-byte aligned rows) are updated in the
+    last combine's epilogue like bf16 ones, the bf16 copy written from the same
+    registers.  Column counts that are a multiple of 4 but not of 8 or 64 leave
+    a ragged last box and a scalar tail in the copy; the copy's rows are padded
+    so that its pitch is a multiple of 8.  The launch count shows that no
+    separate update pass ran; a second step checks the path from non-zero
+    momentum."""
+    b = _binding()
+    sp = wl.GroupSpec(rows, cols, 2, torch.float32, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True)
+    W, G, M = wl.make_group(sp, rows + cols, "cpu")
+    Wd, Gd, Md = W.cuda(), G.cuda(), M.cuda()
+    groups = [wl.views(Wd), wl.views(Gd), wl.views(Md)]
+    pitch = (cols + 7) // 8 * 8
+    backing = torch.full((2, rows, pitch), 7.0, dtype=torch.bfloat16, device="cuda")
+    shadow = backing[:, :, :cols]
+    if with_shadow:
+        groups.append([shadow[i] for i in range(2)])
+    ctx = b.MuonContext([tuple(groups)])
+    try:
+        hp = default_hp(lr=1e-2, wd=0.1)
+        gen = torch.Generator().manual_seed(5)
+        Wc, Mc = W.clone(), M.clone()
+        for step in range(2):
+            if step:
+                G = wl.make_grads(sp, gen, "cpu")
+                Gd.copy_(G)
+            ctx.muon_step(hp)
+            assert ctx.muon_status()[0] == 0
+            alg, planned = b.muon_plan_flops([(rows, cols, 2)], hp.ns_steps)
+            products = 3 * hp.ns_steps + (3 if planned < alg else 0)  # a leading pair: 7 products + 2 helpers for 6
+            assert ctx.muon_last_launch_count() == 2 + products + 1
+            for i in range(2):
+                ref = orc.muon_step(f64(Wc[i]), f64(G[i]), f64(Mc[i]), to_orc(hp))
+                assert rel(f64(Wd[i]) - f64(Wc[i]), ref["W"] - f64(Wc[i])) <= TOL_NS
+                assert rel(f64(Md[i]), ref["M"]) <= TOL_FP32
+                if with_shadow:
+                    assert torch.equal(shadow[i], Wd[i].to(torch.bfloat16))
+            Wc, Mc = Wd.cpu().clone(), Md.cpu().clone()
+        # the padding columns of the copy's rows were never written
+        assert bool((backing[:, :, cols:] == 7.0).all())
+    finally:
+        ctx.muon_destroy()
+
+
 def test_owner_computes_shards_give_the_single_context_bits():
     """Sec. 2.3: each matrix is stepped by its owner rank alone.  A matrix's
     result must not depend on which other matrices share its launch, so the
