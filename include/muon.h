@@ -275,7 +275,7 @@ enum {
   MUON_KERNEL_GRAM = 2,     /* A = X X^T */
   MUON_KERNEL_POLY = 3,     /* B = b A + c A A and the other symmetric m x m x m products */
   MUON_KERNEL_COMB = 4,     /* X' = a X + B X (last iteration: fused weight update) */
-  MUON_KERNEL_UPDATE = 5,   /* separate weight update (ns_steps == 0, fp32 or unaligned W) */
+  MUON_KERNEL_UPDATE = 5,   /* separate weight update (ns_steps == 0, unaligned W, normalised update) */
   MUON_KERNEL_KINDS = 6
 };
 int muon_profile_enable(muon_ctx* ctx, int enable);

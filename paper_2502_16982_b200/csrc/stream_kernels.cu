@@ -395,18 +395,25 @@ symmetrise_diag_kernel(__nv_bfloat16* __restrict__ s, long long stride, int lda,
   const int d0 = blockIdx.x * 128;
   const int size = min(128, m - d0);
   // 8-element chunks; rows are 16-byte aligned (lda is a multiple of 64) and
-  // padded at least to the next multiple of 8 beyond m
-  for (int idx = threadIdx.x; idx < size * 16; idx += blockDim.x) {
-    const int r = idx >> 4, c0 = (idx & 15) * 8;
-    if (c0 < size && c0 + 7 >= r) {  // holds elements on or above the diagonal
-      *reinterpret_cast<uint4*>(&tile[r][c0]) =
-          *reinterpret_cast<const uint4*>(base + static_cast<long long>(d0 + r) * lda + d0 + c0);
-    }
+  // padded at least to the next multiple of 8 beyond m.  Thread t owns half a
+  // row (8 chunks); all its loads are issued before the first is used.
+  const int r = threadIdx.x >> 1, half = (threadIdx.x & 1) * 64;
+  unsigned short* grow = base + static_cast<long long>(d0 + r) * lda + d0 + half;
+  uint4 in[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int c0 = half + k * 8;
+    in[k] = make_uint4(0u, 0u, 0u, 0u);
+    if (r < size && c0 < size && c0 + 7 >= r)  // holds elements on or above the diagonal
+      in[k] = *reinterpret_cast<const uint4*>(grow + k * 8);
   }
+#pragma unroll
+  for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(&tile[r][half + k * 8]) = in[k];
   __syncthreads();
-  for (int idx = threadIdx.x; idx < size * 16; idx += blockDim.x) {
-    const int r = idx >> 4, c0 = (idx & 15) * 8;
-    if (c0 < size && c0 < r) {  // holds elements below the diagonal
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int c0 = half + k * 8;
+    if (r < size && c0 < size && c0 < r) {  // holds elements below the diagonal
       unsigned short v[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
@@ -418,7 +425,7 @@ symmetrise_diag_kernel(__nv_bfloat16* __restrict__ s, long long stride, int lda,
       out.y = v[2] | (static_cast<unsigned>(v[3]) << 16);
       out.z = v[4] | (static_cast<unsigned>(v[5]) << 16);
       out.w = v[6] | (static_cast<unsigned>(v[7]) << 16);
-      *reinterpret_cast<uint4*>(base + static_cast<long long>(d0 + r) * lda + d0 + c0) = out;
+      *reinterpret_cast<uint4*>(grow + k * 8) = out;
     }
   }
 }
