@@ -54,7 +54,7 @@ WORKLOAD_NAMES = {
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/, taken on 64 matrices of the expert-bucket shapes; it scales with the matrix count.
-NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": 7.930e9, "gemm_launches_per_step": 16,
+NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": 7.921e9, "gemm_launches_per_step": 16,
                "momentum_bytes_per_launch": 2.159e9}
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
