@@ -493,19 +493,22 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           } else if (kWFp32) {
             // the same update on fp32 weights: 16 chunks of four columns in two boxes;
             // the bf16 copy of the new weights, if the matrix has one, goes straight
-            // from the registers to global memory (a 128-byte run per row and quarter)
+            // from the registers to global memory (a 128-byte run per row and quarter,
+            // in 32-byte stores where the row is aligned for them)
             const MatDesc& md = P.descs[mat];
             __nv_bfloat16* shadow = static_cast<__nv_bfloat16*>(md.w_shadow);
             const int w_cols = md.cols;
             const bool row_ok = row0 + lane < cur.row_limit && !sc.nonfinite;
             __nv_bfloat16* srow = shadow == nullptr ? nullptr
                                                     : shadow + static_cast<long long>(row0 + lane) * md.ld_ws + col0;
+            // two 8-column chunks at a time: a 32-byte store per lane fills a whole sector
+            const bool wide = srow != nullptr && ((reinterpret_cast<uintptr_t>(srow) & 31) == 0);
 #pragma unroll
-            for (int c8 = 0; c8 < 8; ++c8) {
-              uint32_t packed[4];
+            for (int c16 = 0; c16 < 4; ++c16) {
+              uint32_t packed[8];
 #pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                const int c4 = 2 * c8 + h;
+              for (int h = 0; h < 4; ++h) {
+                const int c4 = 4 * c16 + h;
                 const uint32_t addr = buf + static_cast<uint32_t>((c4 >> 3) * kSubBytes + lane * 128 +
                                                                   (((c4 & 7) ^ (lane & 7)) << 4));
                 uint32_t w0, w1, w2, w3;
@@ -522,14 +525,26 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
                 packed[2 * h + 1] = pack2(w[2], w[3]);
               }
               if (srow != nullptr && row_ok) {
-                const int c = col0 + c8 * 8;
-                if (c + 8 <= w_cols) {
-                  *reinterpret_cast<uint4*>(srow + c8 * 8) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                const int c = col0 + c16 * 16;
+                __nv_bfloat16* dst = srow + c16 * 16;
+                if (wide && c + 16 <= w_cols) {
+                  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(packed[0]),
+                               "r"(packed[1]), "r"(packed[2]), "r"(packed[3]), "r"(packed[4]), "r"(packed[5]),
+                               "r"(packed[6]), "r"(packed[7])
+                               : "memory");
                 } else {
-                  for (int i = 0; i < 8 && c + i < w_cols; ++i) {
-                    const uint32_t pr = packed[i >> 1];
-                    reinterpret_cast<unsigned short*>(srow + c8 * 8)[i] =
-                        static_cast<unsigned short>((i & 1) ? (pr >> 16) : (pr & 0xFFFFu));
+#pragma unroll
+                  for (int h8 = 0; h8 < 2; ++h8) {
+                    if (c + 8 * h8 + 8 <= w_cols) {
+                      *reinterpret_cast<uint4*>(dst + 8 * h8) =
+                          make_uint4(packed[4 * h8], packed[4 * h8 + 1], packed[4 * h8 + 2], packed[4 * h8 + 3]);
+                    } else {
+                      for (int i = 0; i < 8 && c + 8 * h8 + i < w_cols; ++i) {
+                        const uint32_t pr = packed[4 * h8 + (i >> 1)];
+                        reinterpret_cast<unsigned short*>(dst + 8 * h8)[i] =
+                            static_cast<unsigned short>((i & 1) ? (pr >> 16) : (pr & 0xFFFFu));
+                      }
+                    }
                   }
                 }
               }
