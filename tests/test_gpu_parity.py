@@ -370,14 +370,21 @@ def test_dimensions_above_the_limit_are_rejected():
     assert e.value.code == b.MUON_ERR_UNSUPPORTED
 
 
-def test_chunked_bucket_matches_the_oracle():
+@pytest.mark.parametrize("m,n", [(200, 264), (264, 384)])
+def test_chunked_bucket_matches_the_oracle(m, n):
     """A bucket larger than the chunk limit is processed in several chunks that
     reuse the workspace (as the 3432-matrix expert buckets of the full
-    Moonlight-shaped set are): 7 matrices, 3 per chunk, both orientations."""
+    Moonlight-shaped set are): 7 matrices, 3 per chunk, both orientations; the
+    second shape takes its first two iterations as a pair (four symmetric
+    buffers per matrix)."""
     b = _binding()
-    specs = [wl.GroupSpec(264, 200, 4, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
-             wl.GroupSpec(200, 264, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True)]
-    per_matrix = (2 * 200 * 320 + 2 * 200 * 256) * 2  # two X buffers, A and B, bf16, padded pitches
+    specs = [wl.GroupSpec(n, m, 4, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
+             wl.GroupSpec(m, n, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True)]
+    alg, planned = b.muon_plan_flops([(m, n, 1)], 5)
+    n_sym = 4 if planned < alg else 2
+    assert n_sym == (4 if m >= 256 else 2)
+    pad = lambda v: (v + 63) // 64 * 64
+    per_matrix = (2 * m * pad(n) + n_sym * m * pad(m)) * 2  # X buffers and symmetric buffers, bf16, padded pitches
     prev = b.muon_debug_set_chunk_bytes(3 * per_matrix + 64)
     try:
         case = Case(specs, seed=31)
