@@ -939,7 +939,9 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
       if (ce == cudaSuccess) ce = symmetrise(3);
       if (ce == cudaSuccess) ce = sym_product(3, 3, 3, 2, coef(it + 1, 2), coef(it + 1, 1), coef(it + 1, 0));
       if (ce == cudaSuccess) ce = sym_product(2, 1, -1, 0, 1.f, 0.f, 0.f);
-      if (ce == cudaSuccess) ce = symmetrise(0);
+      // B'' B' only multiplies X; in the first pair its mismatch stays at rounding level
+      // (no polynomial is formed from it), later pairs are near the band and keep the fix
+      if (ce == cudaSuccess && !first_it) ce = symmetrise(0);
       if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "poly kernel launch: %s", cudaGetErrorString(ce));
       s_comb = 0;
       a_last = 3;

@@ -498,7 +498,7 @@ def test_fp32_weights_updated_in_the_last_epilogue(rows, cols, with_shadow):
             ctx.muon_step(hp)
             assert ctx.muon_status()[0] == 0
             alg, planned = b.muon_plan_flops([(rows, cols, 2)], hp.ns_steps)
-            products = 3 * hp.ns_steps + (3 if planned < alg else 0)  # a leading pair: 7 products + 2 helpers for 6
+            products = 3 * hp.ns_steps + (2 if planned < alg else 0)  # a leading pair: 7 products + 1 helper for 6
             assert ctx.muon_last_launch_count() == 2 + products + 1
             for i in range(2):
                 ref = orc.muon_step(f64(Wc[i]), f64(G[i]), f64(Mc[i]), to_orc(hp))
