@@ -238,6 +238,9 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="shrink configs 2 and 5 (tests only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ns-steps", type=int, default=5, help="Newton-Schulz iterations (the paper uses 5)")
+    ap.add_argument("--weights", default="config", choices=["config", "fp32", "fp32+bf16copy"],
+                    help="weight dtype: the configuration's own (default), fp32 master weights, or fp32 "
+                         "master weights with a bf16 copy written by the step (Sec. 2.3 keeps fp32 parameters)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-adamw", action="store_true", help="skip the AdamW (non-Muon parameters) leg")
@@ -273,6 +276,9 @@ def main():
     if args.max_count is not None:
         import dataclasses
         specs = [dataclasses.replace(s, count=min(s.count, args.max_count)) for s in specs]
+    if args.weights != "config":
+        import dataclasses
+        specs = [dataclasses.replace(s, w_dtype=torch.float32) for s in specs]
     hpd = hp_dict_default()
     hpd["ns_steps"] = args.ns_steps
     hp = binding.Hyper(**hpd)
@@ -282,7 +288,12 @@ def main():
     for gi, sp in enumerate(specs):
         W, G, M = wl.make_group(sp, rank_seed(args.config, gi, rank), dev)
         state.append((W, G, M))
-        groups.append((wl.views(W), wl.views(G), wl.views(M)))
+        if args.weights == "fp32+bf16copy":
+            copy = torch.zeros(W.shape, dtype=torch.bfloat16, device=dev)
+            state.append((copy,))  # kept alive with the rest
+            groups.append((wl.views(W), wl.views(G), wl.views(M), wl.views(copy)))
+        else:
+            groups.append((wl.views(W), wl.views(G), wl.views(M)))
     ctx = binding.MuonContext(groups)
     stream = torch.cuda.current_stream(dev)
 
@@ -332,7 +343,7 @@ def main():
     if not args.no_e2e:
         g_host, w_host = [], []
         h2d = d2h = 0
-        for sp, (W, G, M) in zip(specs, state):
+        for sp, (W, G, M) in zip(specs, [st for st in state if len(st) == 3]):
             gh = [G[i].cpu().pin_memory() for i in range(sp.count)]
             wh = [torch.empty((sp.rows, sp.cols), dtype=sp.w_dtype).pin_memory() for _ in range(sp.count)]
             g_host.append(gh)
@@ -468,7 +479,7 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD_NAMES[args.config], "matrices": sum(s.count for s in specs),
-                   "params": wl.group_params(specs), "ns_steps": hp.ns_steps,
+                   "params": wl.group_params(specs), "ns_steps": hp.ns_steps, "weights": args.weights,
                    "l2": "inputs exceed L2" if wl.group_params(specs) * 8 > 126e6 else "inputs fit L2",
                    "algorithmic_tflop_per_step": alg_flops / 1e12},
         "pct_bf16_peak_measured_sustained": 100.0 * value / world / float(peaks.get("bf16_tflops_sustained", 1400.0)),
