@@ -131,7 +131,8 @@ typedef struct muon_ctx muon_ctx;
 /*
  * Bytes of device workspace muon_init needs for these groups (pure host
  * computation; only rows/cols/count/dtypes are read).  The workspace holds the
- * bf16 Newton-Schulz operands X, A, B of one bucket chunk, pointer tables,
+ * bf16 Newton-Schulz operands of one bucket chunk (two X buffers, A and B, and
+ * two more symmetric buffers where iterations are taken in pairs), pointer tables,
  * per-matrix scalars and the status word.  Large buckets are processed in
  * chunks so that the workspace stays bounded.
  */
