@@ -158,7 +158,7 @@ def round_to_bf16(x):
     return rounded.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
 
 
-def newton_schulz_bf16_storage(U, eps, steps, a=NS_A, b=NS_B, c=NS_C):
+def newton_schulz_bf16_storage(U, eps, steps, a=NS_A, b=NS_B, c=NS_C, trace=None):
     """Eq. 2 with the storage precision Sec. 2.3 names ("Newton-Schulz
     iteration steps in bf16"): every stored matrix -- the input, A, B and each
     new X -- is rounded to bf16, all arithmetic in between is exact (float64).
@@ -167,16 +167,26 @@ def newton_schulz_bf16_storage(U, eps, steps, a=NS_A, b=NS_B, c=NS_C):
     far the bf16 storage alone moves the result from the float64 iteration, so
     that tests can tell a kernel error from the precision the paper fixes.  The
     1/(||U||_F + eps) factor is applied in full precision to the first A and
-    the first X, as the CUDA path does.  Short side first, like newton_schulz."""
+    the first X, as the CUDA path does.  Short side first, like newton_schulz.
+    If ``trace`` is a list, the stored input and then every iteration's stored
+    (A, B, X) are appended to it (short side first).
+
+    Pinned by a hand-derived two-iteration 2x2 example
+    (tests/golden/bf16_storage_2x2_two_steps.txt) that a missing, doubled or
+    misplaced rounding changes."""
     U = _f64(U)
     transposed = U.shape[0] > U.shape[1]
     nu = math.sqrt(float(np.sum(U * U)))
     s = 1.0 / (nu + eps)
     X = round_to_bf16(U.T if transposed else U)
+    if trace is not None:
+        trace.append(X.copy())
     for k in range(int(steps)):
         A = round_to_bf16((s * s if k == 0 else 1.0) * (X @ X.T))
         B = round_to_bf16(b * A + c * (A @ A))
         X = round_to_bf16((s if k == 0 else 1.0) * (a * X + B @ X))
+        if trace is not None:
+            trace.append((A, B, X.copy()))
     if int(steps) == 0:
         X = s * X
     return np.ascontiguousarray(X.T if transposed else X)

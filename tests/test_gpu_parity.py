@@ -1,12 +1,19 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU fp64
 oracle on the same seeded inputs.
 
-Tolerances (relative Frobenius error):
+Tolerances (relative Frobenius error), the one rule of this suite:
   * fp32 element-wise parts (momentum, norm):            <= 1e-5
-  * bf16 Newton-Schulz path (A, B, X stages, O, delta W): <= 2e-2
-The 2e-2 bound is the one stated for the paper's N = 5 iterations; inside the
-band the quintic map amplifies a perturbation by up to |f'| ~ 3.9 per step, so
-for N > 5 the tests allow 5e-2.
+  * bf16 Newton-Schulz path (A, B, X stages, O, delta W): <= 2e-2 (TOL_NS), on
+    every input shaped and distributed like the benchmark configurations and on
+    every Gaussian test input, for the paper's N = 5 and fewer iterations.
+  * stress inputs only (more than five iterations; max/min in the thousands;
+    spectra spanning orders of magnitude): bf16 storage, the precision the
+    paper fixes (Sec. 2.3), by itself moves the result more than 2e-2 from the
+    float64 iteration there.  ``ns_bound`` then measures that distance with the
+    oracle's storage model (exact arithmetic, only the stored X, A, B rounded;
+    pinned by a hand-derived example) and allows max(2e-2, 1.1 x that
+    distance): the CUDA path may be at most a tenth worse than bf16 storage
+    alone.  The pair (GPU distance, model distance) is printed.
 For bf16 weights the per-step change is about one bf16 ulp of the weight, so
 the weight itself is compared element-wise with the oracle's result: >= 99.9 %
 of elements within one bf16 ulp plus the Newton-Schulz tolerance expressed per
@@ -26,7 +33,17 @@ pytestmark = pytest.mark.gpu
 
 TOL_FP32 = 1e-5
 TOL_NS = 2e-2
-TOL_NS_LONG = 5e-2
+STRESS_SLACK = 1.10
+
+
+def ns_bound(U, eps, ns_steps, o_ref=None, label=""):
+    """(bound, model distance) for a stress input U (the Newton-Schulz input in
+    float64): the larger of TOL_NS and STRESS_SLACK x the distance of the bf16
+    storage model from the float64 iteration on this very input."""
+    if o_ref is None:
+        o_ref = orc.newton_schulz(orc.frobenius_normalise(U, eps)[1], ns_steps)
+    model = rel(orc.newton_schulz_bf16_storage(U, eps, ns_steps), o_ref)
+    return max(TOL_NS, STRESS_SLACK * model), model
 
 
 def _binding():
@@ -101,12 +118,17 @@ def check_step(case, hp, check_w=True, check_o=False):
     rms = case.ctx.muon_get_update_rms()
     gidx = 0
     ohp = to_orc(hp)
-    tol_ns = TOL_NS if hp.ns_steps <= 5 else TOL_NS_LONG
     for gi, sp in enumerate(case.specs):
         W, G, M = case.dev[gi]
         W0, G0, M0 = before[gi]
         for i in range(sp.count):
             ref = orc.muon_step(W0[i], G0[i], M0[i], ohp)
+            tol_ns = TOL_NS
+            if hp.ns_steps > 5:  # a stress input: see the module docstring
+                U = ref["X0"] * (ref["nu"] + hp.eps)
+                tol_ns, model = ns_bound(U, hp.eps, hp.ns_steps, ref["O"])
+                print("N=%d %dx%d: bf16 storage model %.3e from the float64 iteration, bound %.3e"
+                      % (hp.ns_steps, sp.rows, sp.cols, model, tol_ns))
             assert rel(f64(M[i]), ref["M"]) <= TOL_FP32, ("M", gi, i)
             assert abs(norms[gidx] - ref["nu"]) <= TOL_FP32 * ref["nu"] + 1e-30, ("nu", gi, i)
             # update RMS returned for logging (Algorithm 1): follows O, so the Newton-Schulz tolerance
@@ -300,9 +322,8 @@ def test_extreme_aspect_ratios(rows, cols):
     the quintic map is steep, so the bf16 storage the paper prescribes moves the
     result further from the float64 iteration than elsewhere: a CPU model that
     only rounds the stored X, A, B to bf16 (exact arithmetic otherwise) is
-    2.6e-2 away at 48x16400.  The bound here is therefore the larger of 2e-2 and
-    1.25 times that model's own distance, still measured against the float64
-    oracle."""
+    2.6e-2 away at 48x16400.  A stress input: the bound is ``ns_bound``'s, still
+    measured against the float64 oracle."""
     sp = wl.GroupSpec(rows, cols, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)
     case = Case([sp], seed=rows + cols)
     try:
@@ -315,11 +336,12 @@ def test_extreme_aspect_ratios(rows, cols):
         for i in range(sp.count):
             U = (hp.mu + 1.0) * G0[i]  # Nesterov-style input at step 1 from zero momentum
             o_ref = orc.newton_schulz(orc.frobenius_normalise(U, hp.eps)[1], hp.ns_steps)
-            o_model = orc.newton_schulz_bf16_storage(U, hp.eps, hp.ns_steps)
-            bound = max(TOL_NS, 1.25 * rel(o_model, o_ref))
+            bound, model = ns_bound(U, hp.eps, hp.ns_steps, o_ref)
             o_gpu = f64(case.ctx.muon_debug_read(i, case.b.MUON_TAP_X, m, n))
             o_gpu = o_gpu.T if rows > cols else o_gpu
-            assert rel(o_gpu, o_ref) <= bound, (i, rel(o_gpu, o_ref), bound)
+            print("%dx%d matrix %d: GPU %.3e, bf16 storage model %.3e from the float64 iteration (bound %.3e)"
+                  % (rows, cols, i, rel(o_gpu, o_ref), model, bound))
+            assert rel(o_gpu, o_ref) <= bound, (i, rel(o_gpu, o_ref), model, bound)
             assert rel(f64(M[i]), G0[i]) <= TOL_FP32
     finally:
         case.close()
@@ -332,9 +354,9 @@ def test_decaying_and_low_rank_spectra(rows, cols, spectrum):
     have a narrow one): power-law decays and eight directions on a 1e-3 floor.
     Small singular values sit near the rounding noise of bf16 storage, which the
     iteration amplifies up to a^5, so here the bf16 model itself is 1e-2 to
-    1.6e-1 from the float64 iteration; the bound is the larger of 2e-2 and 1.25
-    times the model's distance, as for the extreme aspect ratios.  256 x 512
-    takes its first two iterations as a pair, 192 x 320 the plain sequence."""
+    1.6e-1 from the float64 iteration: stress inputs, bounded by ``ns_bound`` as
+    the extreme aspect ratios are.  256 x 512 takes its first two iterations as
+    a pair, 192 x 320 the plain sequence."""
     b = _binding()
     rng = np.random.default_rng(rows + len(spectrum))
     m = min(rows, cols)
@@ -355,10 +377,11 @@ def test_decaying_and_low_rank_spectra(rows, cols, spectrum):
         assert ctx.muon_status()[0] == 0
         U = (hp.mu + 1.0) * f64(G[0])
         o_ref = orc.newton_schulz(orc.frobenius_normalise(U, hp.eps)[1], hp.ns_steps)
-        o_model = orc.newton_schulz_bf16_storage(U, hp.eps, hp.ns_steps)
-        bound = max(TOL_NS, 1.25 * rel(o_model, o_ref))
+        bound, model = ns_bound(U, hp.eps, hp.ns_steps, o_ref)
         o_gpu = f64(ctx.muon_debug_read(0, b.MUON_TAP_X, m, max(rows, cols)))
-        assert rel(o_gpu, o_ref) <= bound, (rel(o_gpu, o_ref), bound)
+        print("%s %dx%d: GPU %.3e, bf16 storage model %.3e from the float64 iteration (bound %.3e)"
+              % (spectrum, rows, cols, rel(o_gpu, o_ref), model, bound))
+        assert rel(o_gpu, o_ref) <= bound, (rel(o_gpu, o_ref), model, bound)
     finally:
         ctx.muon_destroy()
 

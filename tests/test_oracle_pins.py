@@ -420,6 +420,92 @@ def test_bf16_storage_model_is_the_iteration_with_rounding_only():
     assert np.allclose(x0, orc.round_to_bf16(G) / np.linalg.norm(G), rtol=1e-15)
 
 
+def test_bf16_storage_model_against_the_hand_derived_2x2_example(golden):
+    """Two iterations on a 2x2 input whose every stored value was rounded to 8
+    significant bits by hand (exact rational arithmetic, each decision listed in
+    the fixture): the model must reproduce every stored matrix exactly, also when
+    the input is embedded in a wide or a tall matrix (orientation rule)."""
+    g = golden("bf16_storage_2x2_two_steps.txt")
+    tr = []
+    out = orc.newton_schulz_bf16_storage(g["U"], 0.0, 2, trace=tr)
+    assert np.array_equal(tr[0], g["XB"])
+    for k, names in ((1, ("A", "B", "X1")), (2, ("A2", "B2", "X2"))):
+        for got, name in zip(tr[k], names):
+            assert np.array_equal(got, g[name]), name
+    assert np.array_equal(out, g["X2"])
+    assert np.array_equal(orc.newton_schulz_bf16_storage(g["U"], 0.0, 1), g["X1"])
+    # a wide (2 x 3) and a tall (3 x 2) embedding of the same input: a zero column (row) changes no
+    # stored value, and the tall one must come back transposed
+    wide = np.concatenate([g["U"], np.zeros((2, 1))], axis=1)
+    assert np.array_equal(orc.newton_schulz_bf16_storage(wide, 0.0, 2)[:, :2], g["X2"])
+    tall = np.ascontiguousarray(np.concatenate([g["U"].T, np.zeros((1, 2))], axis=0))
+    assert np.array_equal(orc.newton_schulz_bf16_storage(tall, 0.0, 2)[:2, :], g["X2"].T)
+
+
+def _bf16_model_with_a_planted_mistake(U, kind):
+    """One iteration of the bf16 storage model with one plausible mistake planted
+    (a copy of the model's few lines, each variant changing one of them)."""
+    r = orc.round_to_bf16
+    a, b, c = A_, B_, C_
+    s = 1.0 / math.sqrt(float(np.sum(U * U)))
+    if kind == "s_before_rounding":
+        X, sa, sx = r(s * U), 1.0, 1.0
+    else:
+        X, sa, sx = r(U), s * s, s
+    gram = X.T @ X if kind == "transposed_gram" else X @ X.T
+    A = sa * gram if kind == "A_not_rounded" else r(sa * gram)
+    if kind == "bA_rounded_first":
+        B = r(r(b * A) + c * (A @ A))
+    elif kind == "B_not_rounded":
+        B = b * A + c * (A @ A)
+    elif kind == "b_and_c_swapped":
+        B = r(c * A + b * (A @ A))
+    else:
+        B = r(b * A + c * (A @ A))
+    Y = a * X + B @ X
+    if kind == "rounded_then_scaled":
+        return B, r(sx * r(Y))
+    if kind == "X_not_rounded":
+        return B, sx * Y
+    if kind == "s_squared_on_X":
+        return B, r(sa * Y)
+    return B, r(sx * Y)
+
+
+def test_bf16_storage_pin_notices_planted_mistakes(golden, monkeypatch):
+    """The 2x2 example separates the model from its plausible wrong versions:
+    a rounding left out (A, B, X), done twice or too early (b*A, s*U), the factor
+    s misapplied, a transposed Gram product, swapped coefficients.  The values a
+    wrong model stores are the ones listed in the fixture's comment."""
+    g = golden("bf16_storage_2x2_two_steps.txt")
+    B, X1 = _bf16_model_with_a_planted_mistake(g["U"], "none")
+    assert np.array_equal(B, g["B"]) and np.array_equal(X1, g["X1"])  # the copy itself is faithful
+    for kind in ("A_not_rounded", "s_before_rounding", "bA_rounded_first", "B_not_rounded", "rounded_then_scaled",
+                 "transposed_gram", "X_not_rounded", "s_squared_on_X", "b_and_c_swapped"):
+        B, X1 = _bf16_model_with_a_planted_mistake(g["U"], kind)
+        assert not np.array_equal(X1, g["X1"]), kind
+    B, X1 = _bf16_model_with_a_planted_mistake(g["U"], "A_not_rounded")
+    assert B[0, 1] == -1.2890625 and np.array_equal(X1, [[0.51171875, 0.1904296875], [0.06494140625, 0.609375]])
+    B, X1 = _bf16_model_with_a_planted_mistake(g["U"], "s_before_rounding")
+    assert X1[0, 1] == 0.19140625 and X1[1, 0] == 0.0625
+    B, X1 = _bf16_model_with_a_planted_mistake(g["U"], "rounded_then_scaled")
+    assert X1[1, 0] == 0.068359375
+    # the same, planted in the oracle itself: leaving out its n-th rounding (input, A, B, X1, A2, B2, X2)
+    real = orc.round_to_bf16
+    for skip in range(7):
+        calls = {"n": 0}
+
+        def skipping(x, _skip=skip):
+            calls["n"] += 1
+            return np.asarray(x, dtype=np.float64) if calls["n"] - 1 == _skip else real(x)
+
+        monkeypatch.setattr(orc, "round_to_bf16", skipping)
+        out = orc.newton_schulz_bf16_storage(g["U"], 0.0, 2)
+        monkeypatch.setattr(orc, "round_to_bf16", real)
+        assert calls["n"] == 7
+        assert not np.array_equal(out, g["X2"]), skip
+
+
 @pytest.mark.parametrize("rows,cols", [(6, 20), (12, 12), (9, 40)])
 def test_two_iterations_equal_one_pass_with_the_product_of_their_polynomials(rows, cols):
     """Eq. 2 is X_{k+1} = P_k X_k with P_k = a I + b A_k + c A_k^2, A_k = X_k X_k^T.

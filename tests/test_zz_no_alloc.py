@@ -8,16 +8,21 @@ The check: on the same seeded gradients, two optimizer steps in a row through
 muon_step (workspace path; momentum and ||U||_F read back through
 muon_get_norms) and two calls in a row of the no-workspace entry point must give
 the same momentum and the same norm, within the fp32 tolerance of the GPU parity
-tests.  Two calls matter because the built-in array still holds the first
-call's partial sums when the second one starts.
+tests; both are also held against the CPU oracle's momentum update and
+Frobenius norm directly.  Two calls matter because the built-in array still
+holds the first call's partial sums when the second one starts.  The cases
+cover the kernel's four load paths: 16-byte vector loads and element-wise loads,
+each for bf16 and for fp32 gradients.
 
 This file sorts last on purpose, so a run that stops at the first failure has
 already been through every other test.
 """
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import muon_oracle as orc
 from paper_2502_16982_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -32,8 +37,10 @@ def _rel(a, b):
 
 
 @pytest.mark.parametrize("rows,cols,gdt,nesterov", [
-    (320, 704, torch.bfloat16, True),     # several tiles, vector path
-    (200, 331, torch.float32, False),     # ragged: scalar path, partial tiles
+    (320, 704, torch.bfloat16, True),     # several tiles, bf16 vector loads
+    (256, 512, torch.float32, True),      # fp32 vector loads
+    (200, 331, torch.float32, False),     # ragged: fp32 element-wise loads, partial tiles
+    (136, 203, torch.bfloat16, False),    # ragged: bf16 element-wise loads, partial tiles
     (1408, 2048, torch.bfloat16, True),   # an expert-sized matrix: 352 tiles
 ])
 def test_static_scratch_matches_workspace_path_twice(rows, cols, gdt, nesterov):
@@ -51,6 +58,7 @@ def test_static_scratch_matches_workspace_path_twice(rows, cols, gdt, nesterov):
     # the new entry point's own tensors, all created before its first call
     Gs, Ms = G.cuda()[0].contiguous(), M.cuda()[0].contiguous()
     norm_out = torch.zeros(1, dtype=torch.float32, device="cuda")
+    m_oracle = M[0].double().numpy()
 
     for step, grad in enumerate((G, G2)):
         Gd.copy_(grad)
@@ -65,6 +73,14 @@ def test_static_scratch_matches_workspace_path_twice(rows, cols, gdt, nesterov):
         nu = float(norm_out.item())
         assert abs(nu - nu_ref) <= TOL_FP32 * nu_ref, (step, nu, nu_ref)
         assert _rel(Ms, Md[0]) <= TOL_FP32, (step, _rel(Ms, Md[0]))
+
+        # first hand: the oracle's momentum update, Newton-Schulz input and its Frobenius norm
+        g64 = grad[0].double().numpy()
+        m_oracle = orc.momentum_update(m_oracle, g64, 0.95)
+        nu_oracle, _ = orc.frobenius_normalise(orc.newton_schulz_input(m_oracle, g64, 0.95, nesterov), 0.0)
+        assert abs(nu - nu_oracle) <= TOL_FP32 * nu_oracle, (step, nu, nu_oracle)
+        m_gpu = Ms.double().cpu().numpy()
+        assert np.linalg.norm(m_gpu - m_oracle) <= TOL_FP32 * np.linalg.norm(m_oracle), step
     ctx.muon_destroy()
 
 
