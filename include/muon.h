@@ -70,6 +70,14 @@ enum { MUON_DTYPE_BF16 = 0, MUON_DTYPE_FP32 = 1 };
  *             cols.  The fast vector paths need 16-byte aligned pointers and
  *             ld_* that are multiples of 8; anything else takes a slower
  *             scalar path with the same results.
+ *   Magnitudes: the sum of squares behind ||U||_F and the first Gram product
+ *             (formed from the un-normalised bf16(U) and scaled by 1/||U||_F^2
+ *             in its epilogue) are fp32, so ||U||_F must stay within fp32's
+ *             comfortable range: between about 1e-15 and 1e+18.  Above it the
+ *             sums overflow and a finite input is reported as
+ *             MUON_ERR_NONFINITE; far below it they underflow, the norm reads
+ *             0 and the step only decays W.  Gradients of any loss scale used
+ *             in practice are many orders of magnitude inside these limits.
  */
 typedef struct muon_group {
   int32_t rows;
@@ -157,9 +165,9 @@ int muon_partition(const muon_group* groups, int n_groups, int world, int* owner
  * caller's workspace (DEVICE memory, 1024-byte aligned, at least
  * muon_workspace_bytes() long, owned by the caller, alive until destroy),
  * upload pointer tables and encode the TMA descriptors.  `device` is the CUDA
- * device ordinal all pointers live on; it becomes the calling thread's current
- * device.  The other calls on the context switch to that device for their
- * duration and restore the caller's.  Allocates no device memory itself.
+ * device ordinal all pointers live on.  This call and every other call on the
+ * context switch to that device for their duration and restore the caller's
+ * current device before returning.  Allocates no device memory itself.
  */
 int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* workspace,
               size_t workspace_bytes, int device);
@@ -230,8 +238,12 @@ int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* con
  * MUON_ERR_TIMEOUT or MUON_ERR_NONFINITE; *matrix_index (may be NULL) is the
  * global index (groups in order, matrices in order) of the first matrix that
  * reported it, or -1.  The status word is cleared.  A matrix with a non-finite
- * Newton-Schulz input keeps its W; its M has been updated (and now holds the
- * non-finite values).
+ * Newton-Schulz input keeps its W; its M has been updated by the first line of
+ * the rule and now holds the non-finite values (the momentum pass runs before
+ * the norm is known).  Before the next step the caller must repair that
+ * matrix's M - zero it, or restore it from a copy - or every later step of the
+ * matrix reports MUON_ERR_NONFINITE again and leaves its W unchanged; the
+ * other matrices of the context are not affected.
  */
 int muon_status(muon_ctx* ctx, void* stream, int* device_status, int* matrix_index);
 

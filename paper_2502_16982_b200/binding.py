@@ -326,7 +326,11 @@ class MuonContext:
     gradients, fp32 momenta).  Tensors must outlive the context.
     """
 
-    def __init__(self, groups: Sequence[Sequence[Sequence["torch.Tensor"]]], device: Optional[int] = None):
+    def __init__(self, groups: Sequence[Sequence[Sequence["torch.Tensor"]]], device: Optional[int] = None,
+                 workspace: Optional["torch.Tensor"] = None):
+        """``workspace``: an optional uint8 CUDA tensor to carve the library's
+        workspace from (at least ``muon_workspace_bytes`` + 1023 bytes, so that a
+        1024-byte aligned start fits); by default one is allocated here."""
         import torch
         if not torch.cuda.is_available():
             raise MuonError(MUON_ERR_CUDA, "no CUDA device: this library has no CPU path")
@@ -341,9 +345,15 @@ class MuonContext:
         self.device = dev.index if device is None else device
         nbytes = muon_workspace_bytes(self._groups_c, n)
         self.workspace_bytes = nbytes
-        self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+        if workspace is None:
+            workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+        elif workspace.dtype != torch.uint8 or not workspace.is_contiguous() or workspace.device != dev:
+            raise MuonError(MUON_ERR_WORKSPACE, "workspace must be a contiguous uint8 tensor on the matrices' device")
+        self.workspace = workspace
         base = self.workspace.data_ptr()
         self._ws_ptr = (base + 1023) // 1024 * 1024
+        if self._ws_ptr + nbytes > base + workspace.numel():
+            raise MuonError(MUON_ERR_WORKSPACE, "workspace too small: need %d bytes after alignment" % nbytes)
         ctx = C.c_void_p()
         _check(L.muon_init(C.byref(ctx), self._groups_c, n, C.c_void_p(self._ws_ptr), nbytes, self.device))
         self._ctx = ctx

@@ -606,8 +606,15 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     return fail(MUON_ERR_WORKSPACE, "workspace too small: need %zu bytes, got %zu", need, workspace_bytes);
   }
 
-  cudaError_t ce = cudaSetDevice(device);
+  // `device` is current for the rest of the call; the guard restores the caller's on every return
+  int caller_device = -1;
+  cudaError_t ce = cudaGetDevice(&caller_device);
+  if (ce == cudaSuccess) ce = cudaSetDevice(device);
   if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "cudaSetDevice: %s", cudaGetErrorString(ce)); }
+  struct Restore {
+    int prev, cur;
+    ~Restore() { if (prev >= 0 && prev != cur) cudaSetDevice(prev); }
+  } restore{caller_device, device};
   cudaDeviceProp prop;
   ce = cudaGetDeviceProperties(&prop, device);
   if (ce != cudaSuccess) { delete ctx; return fail(MUON_ERR_CUDA, "cudaGetDeviceProperties: %s", cudaGetErrorString(ce)); }
