@@ -158,7 +158,7 @@ def round_to_bf16(x):
     return rounded.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
 
 
-def newton_schulz_bf16_storage(U, eps, steps, a=NS_A, b=NS_B, c=NS_C, trace=None):
+def newton_schulz_bf16_storage(U, eps, steps, a=NS_A, b=NS_B, c=NS_C, trace=None, fold_identity=False):
     """Eq. 2 with the storage precision Sec. 2.3 names ("Newton-Schulz
     iteration steps in bf16"): every stored matrix -- the input, A, B and each
     new X -- is rounded to bf16, all arithmetic in between is exact (float64).
@@ -170,6 +170,13 @@ def newton_schulz_bf16_storage(U, eps, steps, a=NS_A, b=NS_B, c=NS_C, trace=None
     the first X, as the CUDA path does.  Short side first, like newton_schulz.
     If ``trace`` is a list, the stored input and then every iteration's stored
     (A, B, X) are appended to it (short side first).
+
+    The paper does not say which intermediates are the stored ones.  Eq. 2's
+    a X + B X is also the single product (B + a I) X; ``fold_identity`` selects
+    that reading: the stored polynomial is bf16(b A + c A^2 + a I) and the new X
+    is bf16 of its product with X.  Identical in exact arithmetic; in bf16 the
+    rounding of B_ii + a replaces that of B_ii, which is the smaller error on
+    most inputs and the larger one on a few.
 
     Pinned by a hand-derived two-iteration 2x2 example
     (tests/golden/bf16_storage_2x2_two_steps.txt) that a missing, doubled or
@@ -183,8 +190,12 @@ def newton_schulz_bf16_storage(U, eps, steps, a=NS_A, b=NS_B, c=NS_C, trace=None
         trace.append(X.copy())
     for k in range(int(steps)):
         A = round_to_bf16((s * s if k == 0 else 1.0) * (X @ X.T))
-        B = round_to_bf16(b * A + c * (A @ A))
-        X = round_to_bf16((s if k == 0 else 1.0) * (a * X + B @ X))
+        if fold_identity:
+            B = round_to_bf16(b * A + c * (A @ A) + a * np.eye(A.shape[0]))
+            X = round_to_bf16((s if k == 0 else 1.0) * (B @ X))
+        else:
+            B = round_to_bf16(b * A + c * (A @ A))
+            X = round_to_bf16((s if k == 0 else 1.0) * (a * X + B @ X))
         if trace is not None:
             trace.append((A, B, X.copy()))
     if int(steps) == 0:

@@ -434,6 +434,14 @@ def test_bf16_storage_model_against_the_hand_derived_2x2_example(golden):
             assert np.array_equal(got, g[name]), name
     assert np.array_equal(out, g["X2"])
     assert np.array_equal(orc.newton_schulz_bf16_storage(g["U"], 0.0, 1), g["X1"])
+    # the reading with a*I folded into the stored polynomial
+    tr = []
+    out = orc.newton_schulz_bf16_storage(g["U"], 0.0, 2, trace=tr, fold_identity=True)
+    assert np.array_equal(tr[0], g["XB"])
+    for k, names in ((1, ("A", "BI", "X1F")), (2, ("A2F", "BI2", "X2F"))):
+        for got, name in zip(tr[k], names):
+            assert np.array_equal(got, g[name]), name
+    assert np.array_equal(out, g["X2F"]) and not np.array_equal(g["X2F"], g["X2"])
     # a wide (2 x 3) and a tall (3 x 2) embedding of the same input: a zero column (row) changes no
     # stored value, and the tall one must come back transposed
     wide = np.concatenate([g["U"], np.zeros((2, 1))], axis=1)
