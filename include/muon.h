@@ -207,6 +207,21 @@ int muon_plan_flops(const muon_group* groups, int n_groups, int ns_steps, double
                     double* planned_out);
 
 /*
+ * The same per kernel kind (arrays of MUON_KERNEL_KINDS doubles, indexed by
+ * MUON_KERNEL_*; pure host computation).  planned_by_kind: the FLOPs the launch
+ * sequence asks for, without padding (Gram m^2 n, every symmetric m x m x m
+ * product m^3, combine 2 m^2 n; their sum is muon_plan_flops' planned figure).
+ * executed_by_kind: the FLOPs the tensor cores execute, tile by tile - every
+ * tile is 256 rows by 128 or 256 columns by the contraction length in whole
+ * 64-element stages - so padding at ragged edges and the blocks that are
+ * computed and dropped (below the diagonal of a symmetric result, the cross
+ * terms of a tile shared by two matrices) are included: the figure to hold
+ * against a tensor-pipe utilisation counter.
+ */
+int muon_plan_work(const muon_group* groups, int n_groups, int ns_steps, double* planned_by_kind,
+                   double* executed_by_kind);
+
+/*
  * muon_step for the matrices of ONE bucket (numbering of muon_plan_buckets).
  * Stepping every bucket once, in any order, is one muon_step.  Exists so that
  * a data-parallel caller can start sharing a bucket's updated weights while the
@@ -350,6 +365,19 @@ size_t muon_debug_set_chunk_bytes(size_t bytes);
  * only queries.
  */
 int muon_debug_set_pair_fold(int mode);
+
+/*
+ * Test tap (pure host computation): the tile table the Newton-Schulz products
+ * of a rows x cols matrix use.  which = 0: products with a symmetric result,
+ * table of one unit of *unit_mats matrices; 1: the same for a last matrix
+ * without a partner (empty when units are single matrices); 2: the combine;
+ * 3: the combine formed transposed.  Every tile is nine int16 in `out` (room
+ * for cap_tiles tiles; NULL only queries the count): row block of CTA 0 and of
+ * CTA 1, column block of the first and of the second 128 accumulator columns,
+ * width in column blocks (1 or 2), matrix of CTA 0 and of CTA 1 within the unit,
+ * and per CTA a mask of the column halves whose 128 x 128 block is stored.
+ */
+int muon_debug_tile_table(int rows, int cols, int which, int16_t* out, int cap_tiles, int* n_tiles, int* unit_mats);
 
 /*
  * Test tap: the TMEM base address each CTA of the last Newton-Schulz GEMM launch

@@ -30,7 +30,7 @@ MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
 MUON_SCALE_ADJUSTED_LR, MUON_SCALE_FIXED_DIM, MUON_SCALE_UPDATE_NORM = 0, 1, 2
 
 EXPORTED = [
-    "muon_workspace_bytes", "muon_partition", "muon_plan_buckets", "muon_plan_flops", "muon_init", "muon_step", "muon_step_bucket",
+    "muon_workspace_bytes", "muon_partition", "muon_plan_buckets", "muon_plan_flops", "muon_plan_work", "muon_debug_tile_table", "muon_init", "muon_step", "muon_step_bucket",
     "muon_step_host", "muon_status",
     "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes", "muon_debug_set_pair_fold",
@@ -99,6 +99,10 @@ def lib():
     L.muon_plan_buckets.argtypes = [C.POINTER(muon_group), C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     L.muon_plan_flops.argtypes = [C.POINTER(muon_group), C.c_int, C.c_int, C.POINTER(C.c_double),
                                   C.POINTER(C.c_double)]
+    L.muon_plan_work.argtypes = [C.POINTER(muon_group), C.c_int, C.c_int, C.POINTER(C.c_double),
+                                 C.POINTER(C.c_double)]
+    L.muon_debug_tile_table.argtypes = [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int16), C.c_int,
+                                        C.POINTER(C.c_int), C.POINTER(C.c_int)]
     L.muon_step_bucket.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_int, C.c_void_p]
     L.muon_step_host.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.POINTER(C.POINTER(C.c_void_p)),
                                  C.POINTER(C.POINTER(C.c_void_p)), C.c_void_p]
@@ -290,6 +294,33 @@ def muon_plan_flops(shapes, ns_steps: int = 5):
     alg, planned = C.c_double(0), C.c_double(0)
     _check(lib().muon_plan_flops(arr, len(shapes), int(ns_steps), C.byref(alg), C.byref(planned)))
     return alg.value, planned.value
+
+
+def muon_plan_work(shapes, ns_steps: int = 5):
+    """({kind: planned FLOPs}, {kind: executed FLOPs}) of one step per kernel
+    kind; ``shapes`` is a list of (rows, cols, count).  Executed counts whole
+    tiles: padding and dropped blocks included."""
+    arr = shape_only_groups([(r, c, n, MUON_DTYPE_BF16, MUON_DTYPE_BF16) for (r, c, n) in shapes])
+    planned = (C.c_double * len(KERNEL_KINDS))()
+    executed = (C.c_double * len(KERNEL_KINDS))()
+    _check(lib().muon_plan_work(arr, len(shapes), int(ns_steps), planned, executed))
+    return ({k: planned[i] for i, k in enumerate(KERNEL_KINDS)},
+            {k: executed[i] for i, k in enumerate(KERNEL_KINDS)})
+
+
+def muon_debug_tile_table(rows: int, cols: int, which: int):
+    """(tiles, matrices per unit): every tile is a dict with the row blocks
+    ``i`` and matrices ``dm`` of the two CTAs, the column blocks ``j`` of the
+    two accumulator halves, the width ``nbw`` and the ``keep`` masks."""
+    n, unit = C.c_int(0), C.c_int(0)
+    _check(lib().muon_debug_tile_table(rows, cols, which, None, 0, C.byref(n), C.byref(unit)))
+    buf = (C.c_int16 * (9 * max(1, n.value)))()
+    _check(lib().muon_debug_tile_table(rows, cols, which, buf, n.value, C.byref(n), C.byref(unit)))
+    tiles = []
+    for k in range(n.value):
+        v = buf[9 * k:9 * k + 9]
+        tiles.append({"i": (v[0], v[1]), "j": (v[2], v[3]), "nbw": v[4], "dm": (v[5], v[6]), "keep": (v[7], v[8])})
+    return tiles, unit.value
 
 
 def muon_debug_set_pair_fold(mode: int) -> int:

@@ -48,12 +48,29 @@ struct DevStatus {
   int matrix;
 };
 
-// One entry of a tile table: the CTA pair covers row blocks 2*p and 2*p+1
-// (128 rows each, one per CTA) and `nbw` (1 or 2) column blocks of 128
-// starting at block `jb`.
+// One entry of a tile table.  For rank r in {0, 1} the CTA pair computes the 128
+// output rows of row block i[r] of matrix (first matrix of the unit + dm[r])
+// against N = 128 * nbw output columns:
+//   nbw == 2: accumulator columns [0, 128) are column block j[0], [128, 256)
+//             column block j[1]; CTA r stages the operand-B rows of block j[r],
+//             taken from ITS matrix;
+//   nbw == 1: the columns are block j[0]; each CTA stages 64 of its rows.
+// keep[r] bit h set: the 128 x 128 block (rows of CTA r, column half h) is
+// stored.  The other blocks of the product are computed and dropped: a block
+// below the diagonal of a symmetric result, or the cross terms of a tile whose
+// two CTAs work on different matrices.
+// The row blocks (and, for a symmetric operand B, the column blocks) of one
+// entry are equal or neighbours, because one instruction reads an operand of
+// both CTAs in one layout (see TilePlan in ns_gemm.cu).
 struct PairTile {
-  short p, jb, nbw, pad_;
+  short i[2];
+  short j[2];
+  unsigned char nbw;
+  unsigned char dm[2];
+  unsigned char keep[2];
+  unsigned char pad_[3];
 };
+static_assert(sizeof(PairTile) == 16, "PairTile is read as one 16-byte entry");
 
 // Parameters of one launch of the Newton-Schulz GEMM kernel.  Each output
 // element is  scale * (c_acc * acc + c_in * in) + diag_add * [row == col].
@@ -67,19 +84,20 @@ struct GemmParams {
   CUtensorMap map_out;    // output (and the O tap of the last iteration), box {64, 32}, 128B swizzle
   const CUtensorMap* wmaps;  // last iteration: one map per matrix over its W (chunk-relative),
                              // box {64, 32}, 128B swizzle
-  const PairTile* tiles;  // tile table of one matrix
+  const PairTile* tiles;    // tile table of one unit of `unit_mats` consecutive matrices
+  const PairTile* tiles_tail;  // unit_mats == 2 and an odd count: table of the last matrix alone
   const PairTile* tiles_t;  // last iteration: table of a matrix stored with rows > cols, whose
                             // product is formed transposed (row pairs along the long side)
-  int tiles_per_matrix;
+  int tiles_per_unit;
+  int tiles_per_tail;
+  int unit_mats;   // 1, or 2 where the table pairs blocks of two matrices in one tile
   int count;       // matrices in this launch
   int k;           // contraction length
   int m;           // output rows per matrix (short side of the bucket)
   int n_long;      // long side of the bucket (output rows of a transposed-formulation tile)
   int out_cols;    // output columns per matrix
-  int symmetric;   // the output is symmetric: only blocks on or above the diagonal are
-                   // computed and stored
-  int a_sym;       // operand A is such a matrix: blocks below the diagonal are read as the
-                   // transposes of their mirror images
+  int a_sym;       // operand A is a symmetric matrix kept as its 128-blocks on or above the
+                   // diagonal: blocks below it are read as the transposes of their mirror images
   int b_sym;       // the same for operand B
   int b_mn_major;  // operand B is read MN-major throughout (X in X' = a X + B X)
   int has_in;      // the epilogue reads an input tile through map_in

@@ -123,10 +123,13 @@ struct Bucket {
   // off_s: the symmetric m x m buffers (A and B; two more when iterations are taken in pairs)
   size_t off_x[2], off_s[4], off_partials, off_scal, off_rms_partials, off_factors;
   // workspace offsets of the persistent per-bucket tables
-  size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_comb_tiles, off_comb_tiles_t;
-  std::vector<PairTile> sym_tiles, comb_tiles;  // tile tables of one matrix
-  std::vector<PairTile> comb_tiles_t;           // combine formed transposed: row pairs along the long side
-  int sym_acc_cols, comb_acc_cols;              // widest tile of each table (128 or 256)
+  size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_sym_tiles_tail, off_comb_tiles, off_comb_tiles_t;
+  std::vector<PairTile> sym_tiles;       // symmetric products: table of one unit of sym_unit_mats matrices
+  std::vector<PairTile> sym_tiles_tail;  // sym_unit_mats == 2: table of a last matrix without a partner
+  int sym_unit_mats;
+  std::vector<PairTile> comb_tiles;      // combine: table of one matrix
+  std::vector<PairTile> comb_tiles_t;    // combine formed transposed: row pairs along the long side
+  int sym_acc_cols, comb_acc_cols;       // widest tile of each table (128 or 256)
   // tensor maps over the chunk buffers (all 128-byte swizzled)
   CUtensorMap x_op[2];   // X as K-major operand A: box {64,128}
   CUtensorMap x_b64[2];  // X as operand B (K-major or MN-major): box {64,64}
@@ -263,6 +266,91 @@ inline bool w_tma_ok(const void* w, long long ld, bool fp32) {
   return (reinterpret_cast<uintptr_t>(w) & 15) == 0 && ld % (fp32 ? 4 : 8) == 0;
 }
 
+PairTile make_tile(int i0, int i1, int j0, int j1, int nbw, int dm0, int dm1, unsigned keep0, unsigned keep1) {
+  PairTile t{};
+  t.i[0] = static_cast<short>(i0);
+  t.i[1] = static_cast<short>(i1);
+  t.j[0] = static_cast<short>(j0);
+  t.j[1] = static_cast<short>(j1);
+  t.nbw = static_cast<unsigned char>(nbw);
+  t.dm[0] = static_cast<unsigned char>(dm0);
+  t.dm[1] = static_cast<unsigned char>(dm1);
+  t.keep[0] = static_cast<unsigned char>(keep0);
+  t.keep[1] = static_cast<unsigned char>(keep1);
+  return t;
+}
+
+// Tiles of the symmetric products (only the 128-blocks on or above the diagonal
+// are produced) for matrix `dm` of a unit, nb row blocks.  A tile is two
+// neighbouring row blocks times two neighbouring column blocks.
+//  * nb even: row pair (r, r+1), r even, takes columns r, r+1, then r+2, r+3, ...:
+//    every tile is full width; the first one holds the block (r+1, r) below the
+//    diagonal, which is computed and dropped (nb/2 blocks of nb(nb+1)/2 + nb/2).
+//  * nb odd: row pair (r, r+1) takes columns r+1, r+2, then r+3, r+4, ...: an even
+//    number of columns, every block of every tile is kept.  That leaves the
+//    diagonal blocks (r, r), r even, which no full tile can hold (the block
+//    below it in the pair lies under the diagonal).  `lone` receives them.
+void sym_tiles_of_matrix(int nb, int dm, std::vector<PairTile>* tiles, std::vector<int>* lone) {
+  if (nb % 2 == 0) {
+    for (int r = 0; r < nb; r += 2)
+      for (int c = r; c < nb; c += 2)
+        tiles->push_back(make_tile(r, r + 1, c, c + 1, 2, dm, dm, 3u, c == r ? 2u : 3u));
+    return;
+  }
+  for (int r = 0; r + 1 < nb; r += 2)
+    for (int c = r + 1; c + 1 < nb; c += 2) tiles->push_back(make_tile(r, r + 1, c, c + 1, 2, dm, dm, 3u, 3u));
+  for (int r = 0; r < nb; r += 2) lone->push_back(r);
+}
+
+// Tile tables of a bucket.  Symmetric products with an odd number of row blocks
+// work on units of two matrices: the lone diagonal blocks (r, r) of the two
+// share a full-width tile, one CTA per matrix, whose two cross blocks are
+// dropped; a matrix alone takes them as half-width tiles instead.
+void build_tile_tables(Bucket* Bp) {
+  Bucket& B = *Bp;
+  const int nb = ceil_div(B.m, 128), ncb = ceil_div(B.n, 128), np = ceil_div(nb, 2);
+  B.sym_tiles.clear();
+  B.sym_tiles_tail.clear();
+  B.comb_tiles.clear();
+  B.comb_tiles_t.clear();
+  B.sym_acc_cols = B.comb_acc_cols = 128;
+  std::vector<int> lone;
+  if (nb % 2 == 0) {
+    B.sym_unit_mats = 1;
+    sym_tiles_of_matrix(nb, 0, &B.sym_tiles, &lone);
+  } else {
+    B.sym_unit_mats = 2;
+    sym_tiles_of_matrix(nb, 0, &B.sym_tiles, &lone);
+    lone.clear();
+    sym_tiles_of_matrix(nb, 1, &B.sym_tiles, &lone);
+    for (int r : lone) B.sym_tiles.push_back(make_tile(r, r, r, r, 2, 0, 1, 1u, 2u));
+    lone.clear();
+    sym_tiles_of_matrix(nb, 0, &B.sym_tiles_tail, &lone);
+    // half width: rows (r, r+1) against column block r; the second CTA's block is under the diagonal
+    for (int r : lone) B.sym_tiles_tail.push_back(make_tile(r, r + 1, r, r, 1, 0, 0, 1u, 0u));
+  }
+  for (const PairTile& t : B.sym_tiles)
+    if (t.nbw == 2) B.sym_acc_cols = 256;
+  // combine: row pair p covers row blocks 2p, 2p+1; column tiles are two 128-blocks
+  // wide, with one single block at the end of an odd run
+  for (int p = 0; p < np; ++p) {
+    for (int jb = 0; jb < ncb;) {
+      const int w = std::min(2, ncb - jb);
+      B.comb_tiles.push_back(make_tile(2 * p, 2 * p + 1, jb, jb + 1, w, 0, 0, w == 2 ? 3u : 1u, w == 2 ? 3u : 1u));
+      if (w == 2) B.comb_acc_cols = 256;
+      jb += w;
+    }
+  }
+  // the same product with the roles of the sides exchanged (as many tiles)
+  for (int p = 0; p < ceil_div(ncb, 2); ++p) {
+    for (int jb = 0; jb < nb;) {
+      const int w = std::min(2, nb - jb);
+      B.comb_tiles_t.push_back(make_tile(2 * p, 2 * p + 1, jb, jb + 1, w, 0, 0, w == 2 ? 3u : 1u, w == 2 ? 3u : 1u));
+      jb += w;
+    }
+  }
+}
+
 // Forms the shape buckets and lays out the workspace.  Deterministic in the
 // group list (pointers are not consulted), so muon_workspace_bytes and
 // muon_init agree.
@@ -352,39 +440,13 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
     off = align_up(off + B.mats.size() * sizeof(CUtensorMap), 1024);
     B.off_mmaps = off;
     off = align_up(off + B.mats.size() * sizeof(CUtensorMap), 1024);
-    // tile tables: row pair p covers row blocks 2p, 2p+1; column tiles are two
-    // 128-blocks wide, with one single block at the end of an odd run
-    B.sym_tiles.clear();
-    B.comb_tiles.clear();
-    B.sym_acc_cols = B.comb_acc_cols = 128;
-    const int nb = ceil_div(B.m, 128), ncb = ceil_div(B.n, 128), np = ceil_div(nb, 2);
-    for (int p = 0; p < np; ++p) {
-      for (int jb = 2 * p; jb < nb;) {
-        const int w = std::min(2, nb - jb);
-        B.sym_tiles.push_back(PairTile{static_cast<short>(p), static_cast<short>(jb), static_cast<short>(w), 0});
-        if (w == 2) B.sym_acc_cols = 256;
-        jb += w;
-      }
-      for (int jb = 0; jb < ncb;) {
-        const int w = std::min(2, ncb - jb);
-        B.comb_tiles.push_back(PairTile{static_cast<short>(p), static_cast<short>(jb), static_cast<short>(w), 0});
-        if (w == 2) B.comb_acc_cols = 256;
-        jb += w;
-      }
-    }
+    build_tile_tables(&B);
     B.off_sym_tiles = off;
     off = align_up(off + B.sym_tiles.size() * sizeof(PairTile), 1024);
+    B.off_sym_tiles_tail = off;
+    off = align_up(off + B.sym_tiles_tail.size() * sizeof(PairTile), 1024);
     B.off_comb_tiles = off;
     off = align_up(off + B.comb_tiles.size() * sizeof(PairTile), 1024);
-    // the same product with the roles of the sides exchanged (as many tiles)
-    B.comb_tiles_t.clear();
-    for (int p = 0; p < ceil_div(ncb, 2); ++p) {
-      for (int jb = 0; jb < nb;) {
-        const int w = std::min(2, nb - jb);
-        B.comb_tiles_t.push_back(PairTile{static_cast<short>(p), static_cast<short>(jb), static_cast<short>(w), 0});
-        jb += w;
-      }
-    }
     B.off_comb_tiles_t = off;
     off = align_up(off + B.comb_tiles_t.size() * sizeof(PairTile), 1024);
   }
@@ -579,6 +641,69 @@ int muon_plan_flops(const muon_group* groups, int n_groups, int ns_steps, double
   return MUON_OK;
 }
 
+int muon_plan_work(const muon_group* groups, int n_groups, int ns_steps, double* planned_by_kind,
+                   double* executed_by_kind) {
+  if (!planned_by_kind || !executed_by_kind) return fail(MUON_ERR_INVALID_ARG, "output pointer is null");
+  if (ns_steps < 0 || ns_steps > 64) return fail(MUON_ERR_INVALID_ARG, "ns_steps must be in [0, 64]");
+  int rc = validate_groups(groups, n_groups, false);
+  if (rc) return rc;
+  std::vector<Bucket> buckets;
+  PlanSizes sizes;
+  int total;
+  rc = make_plan(groups, n_groups, &buckets, &sizes, &total);
+  if (rc) return rc;
+  for (int k = 0; k < MUON_KERNEL_KINDS; ++k) planned_by_kind[k] = executed_by_kind[k] = 0.0;
+  // FLOPs one table executes: every tile is 256 rows x (128 or 256) columns x the
+  // contraction length in whole 64-element pipeline stages
+  auto table_flops = [](const std::vector<PairTile>& t, int k) {
+    double f = 0.0;
+    for (const PairTile& e : t) f += 2.0 * 256.0 * (128.0 * e.nbw) * (static_cast<double>(ceil_div(k, kBK)) * kBK);
+    return f;
+  };
+  for (const Bucket& B : buckets) {
+    const double m = B.m, n = B.n;
+    const int n_pairs = plan_pairs(B.pair_mode, B.m, B.n, B.fold_identity, ns_steps);
+    const int n_gram = ns_steps - n_pairs, n_comb = ns_steps - n_pairs;  // a pair has one of each
+    const int n_poly = (ns_steps - 2 * n_pairs) + 5 * n_pairs;
+    const int total_mats = static_cast<int>(B.mats.size());
+    planned_by_kind[MUON_KERNEL_GRAM] += total_mats * n_gram * (m * m * n);
+    planned_by_kind[MUON_KERNEL_POLY] += total_mats * n_poly * (m * m * m);
+    planned_by_kind[MUON_KERNEL_COMB] += total_mats * n_comb * (2.0 * m * m * n);
+    for (int first = 0; first < total_mats; first += B.chunk) {
+      const int count = std::min(B.chunk, total_mats - first);
+      const int units = count / B.sym_unit_mats, tail = count % B.sym_unit_mats;
+      executed_by_kind[MUON_KERNEL_GRAM] +=
+          n_gram * (units * table_flops(B.sym_tiles, B.n) + tail * table_flops(B.sym_tiles_tail, B.n));
+      executed_by_kind[MUON_KERNEL_POLY] +=
+          n_poly * (units * table_flops(B.sym_tiles, B.m) + tail * table_flops(B.sym_tiles_tail, B.m));
+      // both orientations of the combine have as many tiles of the same widths
+      executed_by_kind[MUON_KERNEL_COMB] += n_comb * (count * table_flops(B.comb_tiles, B.m));
+    }
+  }
+  return MUON_OK;
+}
+
+int muon_debug_tile_table(int rows, int cols, int which, int16_t* out, int cap_tiles, int* n_tiles, int* unit_mats) {
+  if (!n_tiles || !unit_mats || rows <= 0 || cols <= 0 || rows > 65536 || cols > 65536 || which < 0 || which > 3)
+    return fail(MUON_ERR_INVALID_ARG, "bad arguments");
+  Bucket B{};
+  B.m = std::min(rows, cols);
+  B.n = std::max(rows, cols);
+  build_tile_tables(&B);
+  const std::vector<PairTile>& t = which == 0 ? B.sym_tiles : (which == 1 ? B.sym_tiles_tail : (which == 2 ? B.comb_tiles : B.comb_tiles_t));
+  *n_tiles = static_cast<int>(t.size());
+  *unit_mats = which == 0 ? B.sym_unit_mats : 1;
+  if (out) {
+    if (cap_tiles < *n_tiles) return fail(MUON_ERR_INVALID_ARG, "table has %d tiles, room for %d", *n_tiles, cap_tiles);
+    for (size_t k = 0; k < t.size(); ++k) {
+      int16_t* o = out + 9 * k;
+      o[0] = t[k].i[0]; o[1] = t[k].i[1]; o[2] = t[k].j[0]; o[3] = t[k].j[1]; o[4] = t[k].nbw;
+      o[5] = t[k].dm[0]; o[6] = t[k].dm[1]; o[7] = t[k].keep[0]; o[8] = t[k].keep[1];
+    }
+  }
+  return MUON_OK;
+}
+
 int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* workspace,
               size_t workspace_bytes, int device) {
   if (!out_ctx) return fail(MUON_ERR_INVALID_ARG, "out_ctx is null");
@@ -694,6 +819,9 @@ int muon_init(muon_ctx** out_ctx, const muon_group* groups, int n_groups, void* 
     if (ce == cudaSuccess)
       ce = cudaMemcpy(ctx->ws + B.off_sym_tiles, B.sym_tiles.data(), B.sym_tiles.size() * sizeof(PairTile),
                       cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess && !B.sym_tiles_tail.empty())
+      ce = cudaMemcpy(ctx->ws + B.off_sym_tiles_tail, B.sym_tiles_tail.data(),
+                      B.sym_tiles_tail.size() * sizeof(PairTile), cudaMemcpyHostToDevice);
     if (ce == cudaSuccess)
       ce = cudaMemcpy(ctx->ws + B.off_comb_tiles, B.comb_tiles.data(), B.comb_tiles.size() * sizeof(PairTile),
                       cudaMemcpyHostToDevice);
@@ -843,6 +971,14 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.decay = decay;
     return P;
   };
+  // tile tables of the products with a symmetric result
+  auto set_sym_tiles = [&](GemmParams& P) {
+    P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
+    P.tiles_tail = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles_tail);
+    P.tiles_per_unit = static_cast<int>(B.sym_tiles.size());
+    P.tiles_per_tail = static_cast<int>(B.sym_tiles_tail.size());
+    P.unit_mats = B.sym_unit_mats;
+  };
   // S[out] = X X^T (first iteration: times s^2, the deferred normalisation)
   auto gram = [&](int x, int out, bool first_it) {
     GemmParams P = base_params();
@@ -851,11 +987,10 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.map_b = B.x_b64[x];
     P.map_in = B.s_e[out];  // unused
     P.map_out = B.s_e[out];
-    P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
-    P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
+    set_sym_tiles(P);
     P.k = B.n;
     P.out_cols = B.m;
-    P.symmetric = 1; P.a_sym = 0; P.b_sym = 0; P.b_mn_major = 0;
+    P.a_sym = 0; P.b_sym = 0; P.b_mn_major = 0;
     P.has_in = 0;
     P.scale_kind = first_it ? 1 : 0;
     P.last = 0;
@@ -873,11 +1008,10 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.map_b = B.s_b64[right];
     P.map_in = B.s_e[in < 0 ? out : in];
     P.map_out = B.s_e[out];
-    P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_sym_tiles);
-    P.tiles_per_matrix = static_cast<int>(B.sym_tiles.size());
+    set_sym_tiles(P);
     P.k = B.m;
     P.out_cols = B.m;
-    P.symmetric = 1; P.a_sym = 1; P.b_sym = 1; P.b_mn_major = 0;
+    P.a_sym = 1; P.b_sym = 1; P.b_mn_major = 0;
     P.has_in = in < 0 ? 0 : 1;
     P.scale_kind = 0;
     P.last = 0;
@@ -897,10 +1031,13 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     P.map_in = B.x_e[x_cur];
     P.map_out = B.x_e[x_nxt];
     P.tiles = reinterpret_cast<const PairTile*>(ctx->ws + B.off_comb_tiles);
-    P.tiles_per_matrix = static_cast<int>(B.comb_tiles.size());
+    P.tiles_tail = P.tiles;
+    P.tiles_per_unit = static_cast<int>(B.comb_tiles.size());
+    P.tiles_per_tail = 0;
+    P.unit_mats = 1;
     P.k = B.m;
     P.out_cols = B.n;
-    P.symmetric = 0; P.a_sym = 1; P.b_sym = 0; P.b_mn_major = 1;
+    P.a_sym = 1; P.b_sym = 0; P.b_mn_major = 1;
     P.has_in = (fuse || !B.fold_identity) ? 1 : 0;  // W when fused, else X for the a*X term
     P.scale_kind = first_it ? 2 : 0;
     P.last = fuse ? 1 : 0;

@@ -121,61 +121,108 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t w0, uint32_t w1, 
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
 }
 
-// Walks the stream of 64-column quarters one CTA's epilogue processes: tiles in
-// the CTA pair's order, within a tile the quarters that hold output of this CTA.
-struct QuarterCursor {
-  int tile, mat, qd, q_end;
-  int ib, jb;
-  int row_limit;  // output rows of the matrix in this tile's orientation
-
-  // Quarter range of tile `t` for CTA `rank`; returns false past the last tile.
-  __device__ __forceinline__ bool open_tile(const GemmParams& P, int t, int total_tiles, int rank) {
-    tile = t;
-    if (t >= total_tiles) return false;
-    mat = t / P.tiles_per_matrix;
-    const bool swapped = P.last && P.descs[mat].transposed != 0;
-    const PairTile pt = (swapped ? P.tiles_t : P.tiles)[t - mat * P.tiles_per_matrix];
-    row_limit = swapped ? P.n_long : P.m;
-    const int col_limit = swapped ? P.m : P.out_cols;
-    ib = 2 * pt.p + rank;
-    jb = pt.jb;
-    const int cols_left = col_limit - jb * 128;
-    q_end = min(2 * pt.nbw, (cols_left + 63) / 64);
-    qd = 0;
-    if (ib * 128 >= row_limit) qd = q_end;               // ragged pair: nothing of ours
-    else if (P.symmetric && jb < ib) qd = min(2, q_end);  // below-diagonal block: dropped
-    return true;
-  }
-  __device__ __forceinline__ bool has_quarter() const { return qd < q_end; }
-};
-
-// What one tile of the launch computes: its table entry, whether it is a
-// transposed-formulation tile of the last iteration, and up to which K block
-// each operand is read transposed (MN-major).
+// What one tile of the launch computes: its table entry, the first matrix of
+// its unit, whether it is a transposed-formulation tile of the last iteration,
+// and up to which K block each operand is read transposed (MN-major).
 struct TilePlan {
   PairTile pt;
+  int base_mat;
   bool swapped;
   int kb_a, kb_b;  // K blocks [0, kb_a) of A and [0, kb_b) of B are read MN-major
 };
 
+// Field of CTA `rank` of a table entry, without indexing an array at run time
+// (which would put the entry in local memory).
+template <typename T>
+__device__ __forceinline__ int of_rank(const T (&v)[2], int rank) {
+  return rank ? static_cast<int>(v[1]) : static_cast<int>(v[0]);
+}
+
+// Table entry and first matrix of tile `tile` of the launch: whole units first,
+// then the tiles of a last matrix that has no partner.
+__device__ __forceinline__ void locate_tile(const GemmParams& P, int tile, PairTile& pt, int& base_mat, bool& swapped) {
+  const int unit = tile / P.tiles_per_unit;
+  const int full_units = P.count / P.unit_mats;
+  swapped = false;
+  if (unit < full_units) {
+    base_mat = unit * P.unit_mats;
+    const int idx = tile - unit * P.tiles_per_unit;
+    swapped = P.last && P.descs[base_mat].transposed != 0;  // the last product has one matrix per unit
+    pt = (swapped ? P.tiles_t : P.tiles)[idx];
+  } else {
+    base_mat = full_units * P.unit_mats;
+    pt = P.tiles_tail[tile - full_units * P.tiles_per_unit];
+  }
+}
+
 __device__ __forceinline__ TilePlan plan_tile(const GemmParams& P, int tile, int num_kb) {
   TilePlan t;
-  const int mat = tile / P.tiles_per_matrix;
-  const int idx = tile - mat * P.tiles_per_matrix;
-  t.swapped = P.last && P.descs[mat].transposed != 0;
-  t.pt = (t.swapped ? P.tiles_t : P.tiles)[idx];
-  // a symmetric operand kept as its upper blocks is read transposed up to the
-  // block where some row of the operand tile is still below the diagonal
-  const int sym_b = min(num_kb, 2 * (t.pt.nbw == 2 ? t.pt.jb + 1 : t.pt.jb));
+  locate_tile(P, tile, t.pt, t.base_mat, t.swapped);
+  // A symmetric operand kept as its upper blocks is read transposed up to the
+  // K block where a row of the operand tile is still below the diagonal.  One
+  // instruction reads the tiles of both CTAs in one layout, so their blocks
+  // are equal or neighbours and the later switch point serves both: the block
+  // the other CTA then reads "the wrong way round" is a diagonal block, which
+  // is the same bits either way.
+  const int sym_a = min(num_kb, 2 * max(t.pt.i[0], t.pt.i[1]));
+  const int sym_b = min(num_kb, 2 * (t.pt.nbw == 2 ? max(t.pt.j[0], t.pt.j[1]) : t.pt.j[0]));
   if (t.swapped) {  // A = X^T from X (MN-major throughout), B = the symmetric matrix
     t.kb_a = num_kb;
     t.kb_b = sym_b;
   } else {
-    t.kb_a = P.a_sym ? min(num_kb, 2 * (2 * t.pt.p + 1)) : 0;
+    t.kb_a = P.a_sym ? sym_a : 0;
     t.kb_b = P.b_mn_major ? num_kb : (P.b_sym ? sym_b : 0);
   }
   return t;
 }
+
+// Walks the stream of 64-column quarters one CTA's epilogue processes: tiles in
+// the CTA pair's order, within a tile the quarters that hold output of this CTA
+// (`qmask`: bit qd set = quarter qd, accumulator columns [64 qd, 64 qd + 64),
+// is still to be stored).
+struct QuarterCursor {
+  int tile, mat;
+  unsigned qmask;
+  int ib;
+  int jb0, jb1;   // column blocks of the two accumulator halves
+  int row_limit;  // output rows of the matrix in this tile's orientation
+
+  // Quarters of tile `t` for CTA `rank`; returns false past the last tile.
+  __device__ __forceinline__ bool open_tile(const GemmParams& P, int t, int total_tiles, int rank) {
+    tile = t;
+    if (t >= total_tiles) {
+      qmask = 0;
+      return false;
+    }
+    PairTile pt;
+    int base_mat;
+    bool swapped;
+    locate_tile(P, t, pt, base_mat, swapped);
+    mat = base_mat + of_rank(pt.dm, rank);
+    row_limit = swapped ? P.n_long : P.m;
+    const int col_limit = swapped ? P.m : P.out_cols;
+    ib = of_rank(pt.i, rank);
+    jb0 = pt.j[0];
+    jb1 = pt.j[1];
+    qmask = 0;
+    if (ib * 128 < row_limit) {  // else a ragged pair: nothing of ours
+      const unsigned keep = static_cast<unsigned>(of_rank(pt.keep, rank));
+#pragma unroll
+      for (int qd = 0; qd < 4; ++qd) {
+        const int h = qd >> 1;
+        const bool on = qd < 2 * pt.nbw && ((keep >> h) & 1u) && (h ? jb1 : jb0) * 128 + (qd & 1) * 64 < col_limit;
+        qmask |= on ? (1u << qd) : 0u;
+      }
+    }
+    return true;
+  }
+  __device__ __forceinline__ bool has_quarter() const { return qmask != 0; }
+  __device__ __forceinline__ int quarter() const { return __ffs(qmask) - 1; }
+  __device__ __forceinline__ void pop_quarter() { qmask &= qmask - 1; }
+  // first output column of quarter qd
+  __device__ __forceinline__ int col_block(int qd) const { return (qd >> 1) ? jb1 : jb0; }
+  __device__ __forceinline__ int col0(int qd) const { return col_block(qd) * 128 + (qd & 1) * 64; }
+};
 
 // kAccCols: fp32 TMEM columns per accumulator stage = widest N (128 or 256).
 // kStages: depth of the operand ring; kSubsPerWarp: staging buffers per epilogue warp.
@@ -197,7 +244,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
   const uint32_t rank = ptx::cluster_ctarank();      // 0 = leader
   const int cluster = static_cast<int>(ptx::cluster_id_x());
   const int num_clusters = static_cast<int>(ptx::num_clusters_x());
-  const int total_tiles = P.count * P.tiles_per_matrix;
+  const int total_tiles = (P.count / P.unit_mats) * P.tiles_per_unit + (P.count % P.unit_mats ? P.tiles_per_tail : 0);
   const int num_kb = (P.k + kBK - 1) / kBK;
   volatile int* abort_flag = &bars->abort_flag;
   constexpr uint32_t kTmemCols = kNumAcc * kAccCols;
@@ -242,12 +289,13 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       const uint32_t empty0 = ptx::smem_u32(&bars->empty[0]);
       const uint32_t leader_full0 = ptx::map_to_cta(full0, 0);  // the rank lives in the upper address bits
       for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
-        const int mat = tile / P.tiles_per_matrix;
         const TilePlan tp = plan_tile(P, tile, num_kb);
         const PairTile pt = tp.pt;
-        const int row0 = (2 * pt.p + static_cast<int>(rank)) * 128;
+        const int r = static_cast<int>(rank);
+        const int mat = tp.base_mat + of_rank(pt.dm, r);  // this CTA's matrix (its own A rows and B rows)
+        const int row0 = of_rank(pt.i, r) * 128;
         const int half = 64 * pt.nbw;  // B rows (N columns) staged by each CTA
-        const int b0 = pt.jb * 128 + static_cast<int>(rank) * half;
+        const int b0 = pt.nbw == 2 ? of_rank(pt.j, r) * 128 : pt.j[0] * 128 + r * 64;
         const uint32_t stage_tx = 2u * static_cast<uint32_t>(kTileABytes + half * 128);
         const int kb_a = tp.kb_a, kb_b = tp.kb_b;
         // a transposed-formulation tile takes its operands from the other two 64 x 64 maps
@@ -311,9 +359,9 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       constexpr uint32_t kLboK = (16u >> 4) << 16;      // K-major: LBO 16
       constexpr uint32_t kLboMN = (8192u >> 4) << 16;   // MN-major: LBO 8192 (next 64-element chunk)
       for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
-        const int mat = tile / P.tiles_per_matrix;
         const TilePlan tp = plan_tile(P, tile, num_kb);
         const PairTile pt = tp.pt;
+        const int mat = tp.base_mat;
         const int kb_a = tp.kb_a, kb_b = tp.kb_b;
         ok = ptx::mbar_wait(ptx::smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag);
         ok = __all_sync(0xFFFFFFFFu, ok);
@@ -399,7 +447,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       const uint32_t bar = ptx::smem_u32(&my_bars[e]);
       const uint32_t buf = my_base + e * kEntryBytes;
       const int row0 = pre.ib * 128 + q * 32;
-      const int col0 = pre.jb * 128 + pre.qd * 64;
+      const int col0 = pre.col0(pre.quarter());
       if (row0 >= pre.row_limit) {  // this warp's rows lie beyond the matrix: nothing to fetch
         ptx::mbar_arrive(bar);
       } else if (P.last) {
@@ -416,7 +464,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         ptx::mbar_arrive(bar);
       }
       ++pre_g;
-      ++pre.qd;
+      pre.pop_quarter();
       pre_seek();
     };
     if (lane == 0) {
@@ -445,12 +493,13 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * kAccCols) +
                                (static_cast<uint32_t>(q * 32) << 16);
 
-        for (int qd = cur.qd; qd < cur.q_end && ok; ++qd, ++gq) {
+        for (; cur.has_quarter() && ok; cur.pop_quarter(), ++gq) {
+          const int qd = cur.quarter();
           const uint32_t e = gq % ring_len;
           const uint32_t buf = my_base + e * kEntryBytes;  // in / out (W on the last iteration)
-          const int col0 = cur.jb * 128 + qd * 64;
+          const int col0 = cur.col0(qd);
           // column of this lane's row that lies on the matrix diagonal, if the quarter holds it
-          const bool diag_quarter = P.diag_add != 0.f && cur.jb + (qd >> 1) == cur.ib;
+          const bool diag_quarter = P.diag_add != 0.f && cur.col_block(qd) == cur.ib;
           const int dcol = q * 32 + lane - (qd & 1) * 64;
 
           uint32_t v[64];
@@ -710,7 +759,8 @@ cudaError_t gemm_max_clusters(int* out) {
 
 // acc_cols: 128 when every tile of the launch is one column block wide, else 256.
 cudaError_t launch_ns_gemm(const GemmParams& P, int acc_cols, int max_clusters, cudaStream_t stream) {
-  const long long total = static_cast<long long>(P.count) * P.tiles_per_matrix;
+  const long long total = static_cast<long long>(P.count / P.unit_mats) * P.tiles_per_unit +
+                          (P.count % P.unit_mats ? P.tiles_per_tail : 0);
   if (total <= 0) return cudaSuccess;
   const unsigned clusters = static_cast<unsigned>(total < max_clusters ? total : max_clusters);
   const bool deep_ring = !P.has_in && !P.last;  // no epilogue input tiles: the Gram product

@@ -1,0 +1,132 @@
+"""The tile tables of the Newton-Schulz products, checked on the host (no GPU):
+every output block that has to be stored is stored exactly once, nothing
+outside the matrix is stored, and every tile obeys the rules the kernel's
+operand layouts impose.
+
+A tile is a CTA pair's work: 128 rows from each CTA (row blocks i[0], i[1] of
+matrices dm[0], dm[1] of the unit) against one or two column blocks j.  One
+instruction reads the operand tiles of both CTAs in one layout, and a symmetric
+operand kept as its upper blocks changes layout at the diagonal, so for such
+operands the two row blocks (and the two column blocks) of a tile must be equal
+or neighbours.  A tile whose CTAs work on different matrices computes two cross
+blocks that mean nothing; they must not be stored.
+"""
+
+import pytest
+
+from paper_2502_16982_b200 import binding as b
+
+SHAPES = [(1408, 2048), (2048, 1408), (2048, 2048), (128, 256), (100, 300), (129, 257), (640, 256), (1536, 1536),
+          (1792, 4608), (2304, 6016), (6656, 2560), (576, 2048), (512, 4096), (16, 65536), (384, 384), (3200, 3300)]
+
+
+def blocks(v):
+    return -(-v // 128)
+
+
+@pytest.mark.parametrize("rows,cols", SHAPES)
+def test_symmetric_product_tables_cover_the_upper_triangle_once(rows, cols):
+    m = min(rows, cols)
+    nb = blocks(m)
+    for which in (0, 1):
+        tiles, unit = b.muon_debug_tile_table(rows, cols, which)
+        if which == 1:
+            assert unit == 1
+            if not tiles:  # single-matrix units need no table for a last matrix alone
+                assert b.muon_debug_tile_table(rows, cols, 0)[1] == 1
+                continue
+            unit_here = 1
+        else:
+            assert unit in (1, 2) and tiles
+            unit_here = unit
+        seen = {}
+        for t in tiles:
+            assert t["nbw"] in (1, 2)
+            # layout rule for symmetric operands: neighbours or equal, on both sides
+            assert abs(t["i"][0] - t["i"][1]) <= 1
+            if t["nbw"] == 2:
+                assert abs(t["j"][0] - t["j"][1]) <= 1
+            for rank in (0, 1):
+                assert 0 <= t["dm"][rank] < unit_here
+                i = t["i"][rank]
+                for h in range(t["nbw"]):
+                    if not (t["keep"][rank] >> h) & 1:
+                        continue
+                    j = t["j"][h]
+                    # a stored block is computed from this CTA's matrix on both sides: with the full
+                    # width the B rows of half h come from CTA h's matrix
+                    if t["nbw"] == 2:
+                        assert t["dm"][h] == t["dm"][rank], t
+                    if i >= nb:
+                        continue  # rows beyond the matrix: the kernel stores nothing for them
+                    assert j < nb and i <= j, t  # on or above the diagonal, inside the matrix
+                    key = (t["dm"][rank], i, j)
+                    seen[key] = seen.get(key, 0) + 1
+                if t["keep"][rank] >> t["nbw"]:
+                    raise AssertionError("keep bit beyond the tile's width: %r" % (t,))
+        want = {(d, i, j) for d in range(unit_here) for i in range(nb) for j in range(i, nb)}
+        assert set(seen) == want
+        assert all(c == 1 for c in seen.values())
+
+
+@pytest.mark.parametrize("rows,cols", SHAPES)
+def test_combine_tables_cover_the_output_once(rows, cols):
+    m, n = min(rows, cols), max(rows, cols)
+    for which, out_rows, out_cols in ((2, m, n), (3, n, m)):
+        tiles, unit = b.muon_debug_tile_table(rows, cols, which)
+        assert unit == 1
+        rb, cb = blocks(out_rows), blocks(out_cols)
+        seen = {}
+        for t in tiles:
+            assert t["dm"] == (0, 0)
+            assert t["i"][1] == t["i"][0] + 1  # the symmetric operand's rows (or X^T's): neighbours
+            for rank in (0, 1):
+                i = t["i"][rank]
+                for h in range(t["nbw"]):
+                    assert (t["keep"][rank] >> h) & 1
+                    j = t["j"][h]
+                    assert j < cb
+                    if i < rb:
+                        seen[(i, j)] = seen.get((i, j), 0) + 1
+        assert set(seen) == {(i, j) for i in range(rb) for j in range(cb)}
+        assert all(c == 1 for c in seen.values())
+    assert len(b.muon_debug_tile_table(rows, cols, 2)[0]) == len(b.muon_debug_tile_table(rows, cols, 3)[0])
+
+
+def test_executed_work_follows_the_tables():
+    """muon_plan_work: planned FLOPs add up to muon_plan_flops' figure, executed
+    FLOPs are the tiles' (256 rows x 128 or 256 columns x the contraction length
+    in whole 64-element stages)."""
+    shapes = [(1408, 2048, 7), (2048, 2048, 3), (100, 300, 5)]
+    for ns in (1, 5, 10):
+        planned, executed = b.muon_plan_work(shapes, ns)
+        alg, planned_total = b.muon_plan_flops(shapes, ns)
+        assert abs(sum(planned.values()) - planned_total) <= 1e-9 * planned_total
+        for kind in ("gram", "poly", "comb"):
+            assert executed[kind] >= planned[kind] > 0
+        assert executed["momentum"] == executed["norm"] == executed["update"] == 0
+    # one expert-shaped bucket of 7 matrices, by hand: three units of two matrices and one alone
+    planned, executed = b.muon_plan_work([(1408, 2048, 7)], 1)
+    unit, _ = b.muon_debug_tile_table(1408, 2048, 0)
+    tail, _ = b.muon_debug_tile_table(1408, 2048, 1)
+    comb, _ = b.muon_debug_tile_table(1408, 2048, 2)
+    per = lambda tiles, k: sum(2.0 * 256 * 128 * t["nbw"] * k for t in tiles)
+    assert executed["gram"] == 3 * per(unit, 2048) + per(tail, 2048)
+    assert executed["poly"] == 3 * per(unit, 1408) + per(tail, 1408)
+    assert executed["comb"] == 7 * per(comb, 1408)
+    assert planned["gram"] == 7 * 1408.0 ** 2 * 2048 and planned["comb"] == 2 * planned["gram"]
+
+
+def test_expert_shape_tables_have_the_expected_sizes():
+    """1408 rows are 11 row blocks: 15 full tiles per matrix plus six diagonal
+    blocks that pair up with the neighbour matrix's (36 tiles per two matrices);
+    a matrix alone takes them as six half-width tiles."""
+    unit, mats = b.muon_debug_tile_table(2048, 1408, 0)
+    assert mats == 2 and len(unit) == 36 and all(t["nbw"] == 2 for t in unit)
+    shared = [t for t in unit if t["dm"] == (0, 1)]
+    assert len(shared) == 6 and all(t["i"][0] == t["i"][1] == t["j"][0] == t["j"][1] for t in shared)
+    assert all(t["keep"] == (1, 2) for t in shared)
+    tail, _ = b.muon_debug_tile_table(2048, 1408, 1)
+    assert len(tail) == 21 and sum(1 for t in tail if t["nbw"] == 1) == 6
+    even, mats = b.muon_debug_tile_table(2048, 2048, 0)
+    assert mats == 1 and len(even) == 36
