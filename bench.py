@@ -18,8 +18,12 @@ host inside the timed region.
 --impl reference times the CPU fp64 oracle on a bounded sample of the same
 workload (it is the only reference this method has; a baseline, not a target).
 
-With N > 1 (torchrun) every rank owns its own shard of matrices of the same
-size (matrices are independent units; no data-path collective): weak scaling.
+With N > 1 (torchrun) the SAME parameter set is partitioned over the ranks
+(Sec. 2.3, Distributed Muon: every matrix is stepped by the one rank that owns
+it) and the all-gather of the updated weights over NCCL is inside the timed
+region: strong scaling.  Gradients are taken as already reduced on their owner
+(the reduce-scatter of Algorithm 1's first line belongs to the backward pass
+and is the same as for AdamW); --reduce-grads adds it to the timed region.
 """
 
 from __future__ import annotations
@@ -54,7 +58,7 @@ WORKLOAD_NAMES = {
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/, taken on 64 matrices of the expert-bucket shapes; it scales with the matrix count.
-NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": 7.921e9, "gemm_launches_per_step": 16,
+NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": None, "gemm_launches_per_step": 16,
                "momentum_bytes_per_launch": 2.159e9}
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
@@ -79,8 +83,9 @@ class ClockSampler:
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index):
-        self.gpu_index = gpu_index
+    def __init__(self, gpu_id):
+        # nvidia-smi numbers physical GPUs and ignores CUDA_VISIBLE_DEVICES: the GPU is named by UUID
+        self.gpu_index = gpu_id
         self.proc = None
         self.lines = []  # (arrival time, text)
         self.t_begin = self.t_end = None
@@ -136,7 +141,7 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "gpu": str(self.gpu_index)}
 
 
 def oracle_sample_time(specs, hp_dict, budget_s=20.0, max_mats=4):
@@ -176,12 +181,6 @@ def oracle_sample_time(specs, hp_dict, budget_s=20.0, max_mats=4):
     return flops, secs, "%d oracle steps on single matrices of %s" % (len(done), ", ".join(uniq)), threads
 
 
-def rank_seed(cfg, group_index, rank):
-    """Seed of one group's tensors on one rank: every rank owns its own shard
-    of equally many matrices (weak scaling), drawn from a different stream."""
-    return 1000 * cfg + group_index + 100000 * rank
-
-
 def max_over_ranks(value, dist, device):
     """MAX-reduce of a scalar over the process group (identity without one)."""
     if dist is None:
@@ -191,9 +190,10 @@ def max_over_ranks(value, dist, device):
     return float(t.item())
 
 
-def whole_job_value(flops_per_rank, world, ms_per_step):
-    """Aggregate metric: the work of all ranks over the slowest rank's time."""
-    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+def whole_job_value(job_flops, ms_per_step):
+    """Aggregate metric: the work of the whole job (all ranks together step every
+    matrix of the one parameter set once) over the slowest rank's time."""
+    return job_flops / (ms_per_step * 1e-3) / 1e12
 
 
 def hp_dict_default():
@@ -220,13 +220,190 @@ def run_reference(args, rank):
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": {"workload": WORKLOAD_NAMES[args.config], "sample": desc},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+def gpu_uuid(dev):
+    try:
+        u = str(torch.cuda.get_device_properties(dev).uuid)
+        return u if u.startswith("GPU-") else "GPU-" + u
+    except Exception:
+        return str(dev.index)
+
+
+def gemm_rooflines(prof, steps, alg_flops, dense_flops, planned, executed, peaks, clocks):
+    """Roofline of the Newton-Schulz GEMM launches from per-kind event times.
+    `prof`: {kind: (ms, launches)} over `steps` steps; `planned` / `executed`:
+    FLOPs per step by kind (muon_plan_work)."""
+    kinds = ("gram", "poly", "comb")
+    gemm_ms = sum(prof[k][0] for k in kinds)
+    gemm_launches = sum(prof[k][1] for k in kinds)
+    if not gemm_launches:
+        return None, {}
+    peak = float(peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops")))
+    burst = float(peaks.get("bf16_tflops", peak))
+    tf = lambda flops, ms: flops * steps / (ms * 1e-3) / 1e12
+    per_kind = {}
+    for k in kinds:
+        if prof[k][1]:
+            per_kind[k] = {"planned_tflops": tf(planned[k], prof[k][0]), "executed_tflops": tf(executed[k], prof[k][0]),
+                           "planned_frac_of_sustained": tf(planned[k], prof[k][0]) / peak,
+                           "executed_over_planned": executed[k] / planned[k]}
+    planned_all = sum(planned[k] for k in kinds)
+    executed_all = sum(executed[k] for k in kinds)
+    achieved = tf(alg_flops, gemm_ms)
+    roof = {
+        "kernel": "ns_gemm_kernel (gram + poly + comb launches)", "bound": "tensor",
+        "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+        "peak_source": "%s bf16_tflops_sustained" % peaks["_source"],
+        "frac_of_measured_burst": achieved / burst, "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
+        "numerator": "algorithmic FLOPs of Eq. 2, ns_steps * (3 m^2 n + m^3) per matrix",
+        "dense_equivalent_tflops": tf(dense_flops, gemm_ms),
+        "avg_launch_ms": gemm_ms / gemm_launches, "flops_per_launch": alg_flops * steps / gemm_launches,
+        # what the launch sequence asks of the tensor cores (less than algorithmic where two
+        # iterations share a pass over X) and what they execute (whole tiles: padding, dropped blocks)
+        "planned_tflops": tf(planned_all, gemm_ms), "frac_planned": tf(planned_all, gemm_ms) / peak,
+        "planned_over_algorithmic_flops": planned_all / alg_flops,
+        "executed_tflops": tf(executed_all, gemm_ms), "executed_over_planned_flops": executed_all / planned_all,
+        "by_kind": per_kind, "traffic": None,
+    }
+    if clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+        # tensor-pipe utilisation implied by the executed FLOPs at the clock sampled during the run:
+        # against the nominal dense rate scaled by clock / maximum clock, and as FLOPs per clock per SM
+        # against the 8192 a B200 SM retires (2.25 PFLOP/s / 148 SMs / 1.856 GHz)
+        roof["tensor_util_at_sampled_clock"] = tf(executed_all, gemm_ms) / (
+            NOMINAL_BF16_TFLOPS * clocks["sm_mhz"] / clocks["sm_max_mhz"])
+        roof["executed_flops_per_clock_per_sm"] = tf(executed_all, gemm_ms) * 1e12 / (148 * clocks["sm_mhz"] * 1e6)
+    return roof, per_kind
+
+
+def run_distributed(args, rank, world, local_rank):
+    """N > 1: one parameter set, partitioned over the ranks (Sec. 2.3)."""
+    import torch.distributed as dist
+    from paper_2502_16982_b200 import binding
+    from paper_2502_16982_b200.distributed import DistributedMuon
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world == 1 and "RANK" not in os.environ:  # --distributed without torchrun: a one-rank group
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29517")
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+    else:
+        dist.init_process_group("nccl", device_id=dev)
+    specs = wl.config_groups(args.config, args.layers)
+    if args.max_count is not None:
+        import dataclasses
+        specs = [dataclasses.replace(s, count=min(s.count, args.max_count)) for s in specs]
+    hpd = hp_dict_default()
+    hpd["ns_steps"] = args.ns_steps
+    hp = binding.Hyper(**hpd)
+    dm = DistributedMuon([(s.rows, s.cols, s.count, s.w_dtype, s.g_dtype) for s in specs], dev, dist=dist)
+    # the same weights and (already reduced) gradients on every rank: same seeds everywhere
+    for gi, sp in enumerate(specs):
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1000 * args.config + gi)
+        for j in range(sp.count):
+            dm.weights[gi][j].copy_((torch.randn(sp.rows, sp.cols, generator=gen, device=dev) * sp.w_std).to(sp.w_dtype))
+            dm.grads[gi][j].copy_((torch.randn(sp.rows, sp.cols, generator=gen, device=dev) * sp.g_std).to(sp.g_dtype))
+    stream = torch.cuda.current_stream(dev)
+    alg_flops, _ = wl.ns_flops(specs, hp.ns_steps)
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        dm.step(hp, reduce_grads=args.reduce_grads)
+    status, which = dm.status()
+    if status != 0:
+        raise SystemExit("device status %d at matrix %d during warm-up" % (status, which))
+    sampler = ClockSampler(gpu_uuid(dev))
+    sampler.start()
+    barrier()
+    sampler.begin()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    timings = []
+    e0.record(stream)
+    for _ in range(args.steps):
+        t = {}
+        dm.step(hp, reduce_grads=args.reduce_grads, timing=t)
+        timings.append(t)
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    status, which = dm.status()
+    if status != 0:
+        raise SystemExit("device status %d at matrix %d in the timed region" % (status, which))
+    compute_ms = sum(t["start"].elapsed_time(t["compute_end"]) for t in timings) / args.steps
+    total_ms = sum(t["start"].elapsed_time(t["end"]) for t in timings) / args.steps
+    exch_ms = sum(a.elapsed_time(b) for t in timings for a, b in t["exchanges"]) / args.steps
+    exposed = max(0.0, total_ms - compute_ms)
+    dist_info = {
+        "ranks": world, "owned_matrices_this_rank": len(dm.owned), "matrices": sum(s.count for s in specs),
+        "compute_ms_per_step": max_over_ranks(compute_ms, dist, dev),
+        "exchange_ms_per_step": max_over_ranks(exch_ms, dist, dev),
+        "exposed_exchange_ms_per_step": max_over_ranks(exposed, dist, dev),
+        "overlapped_fraction": (1.0 - exposed / exch_ms) if exch_ms > 0 else None,
+        "gather_bytes_received_per_rank": dm.gather_bytes_per_rank,
+        "gather_gbs_per_rank": dm.gather_bytes_per_rank / (exch_ms * 1e-3) / 1e9 if exch_ms > 0 else None,
+        "gradients": "reduce-scatter inside the timed region" if args.reduce_grads
+                     else "assumed already reduced on the owner (reduce-scatter left to the backward pass)",
+        "load_imbalance": max(dm.loads) / (sum(dm.loads) / world),
+    }
+    # end to end: this rank's gradients from pinned host memory, its updated weights back
+    e2e = None
+    if not args.no_e2e:
+        slots = [(u, dm._slot(dm.g_flat[u], u, rank), dm._slot(dm.w_flat[u], u, rank)) for u in range(dm.n_units)]
+        g_host = [g.cpu().pin_memory() for _, g, _ in slots]
+        w_host = [torch.empty(w.shape, dtype=w.dtype).pin_memory() for _, _, w in slots]
+        h2d = sum(t.numel() * t.element_size() for t in g_host)
+        d2h = sum(t.numel() * t.element_size() for t in w_host)
+        e2e_steps = max(3, min(args.steps, 5))
+
+        def one():
+            for (u, g, w), gh in zip(slots, g_host):
+                g.copy_(gh, non_blocking=True)
+            dm.step(hp)
+            for (u, g, w), wh in zip(slots, w_host):
+                wh.copy_(w, non_blocking=True)
+
+        one()
+        barrier()
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            one()
+        e1.record(stream)
+        barrier()
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), dist, dev) / e2e_steps
+        h2d_all = max_over_ranks(h2d, dist, dev)
+        e2e = {"value": whole_job_value(alg_flops, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "note": "bytes of rank 0; every rank moves its own slots (largest: %d B up)" % int(h2d_all)}
+    launches = dm._ctx.muon_last_launch_count() * len([b for b in dm.local_bucket if b is not None]) if dm._ctx else 0
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": whole_job_value(alg_flops, ms_step), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD_NAMES[args.config], "matrices": sum(s.count for s in specs),
+                       "params": wl.group_params(specs), "ns_steps": hp.ns_steps,
+                       "parallelism": "owner-computes dp%d, in-place NCCL all-gather of W per shape bucket" % world,
+                       "l2": "inputs exceed L2", "algorithmic_tflop_per_step": alg_flops / 1e12},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches * args.steps, "distributed": dist_info,
+            "roofline": None, "cpu_baseline": None,
+        }
+        print(json.dumps(line))
+    dm.close()
+    dist.destroy_process_group()
 
 
 def main():
@@ -244,6 +421,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-adamw", action="store_true", help="skip the AdamW (non-Muon parameters) leg")
+    ap.add_argument("--reduce-grads", action="store_true",
+                    help="N > 1: sum the gradients over the ranks (reduce-scatter) inside the timed region")
+    ap.add_argument("--distributed", action="store_true",
+                    help="take the partitioned (N > 1) path even with one rank")
     ap.add_argument("--max-count", type=int, default=None,
                     help="cap the matrices per group (small cases for profiler captures)")
     ap.add_argument("--ref-budget", type=float, default=12.0)
@@ -262,15 +443,13 @@ def main():
         args.warmup = 3
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the Muon step has no CPU path")
+    if world > 1 or args.distributed:
+        run_distributed(args, rank, world, local_rank)
+        return
     from paper_2502_16982_b200 import binding
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
 
     specs = wl.config_groups(args.config, args.layers)
     if args.max_count is not None:
@@ -283,10 +462,10 @@ def main():
     hpd["ns_steps"] = args.ns_steps
     hp = binding.Hyper(**hpd)
 
-    # Inputs: seeded, drawn on the device (each rank its own shard of equal size).
+    # Inputs: seeded, drawn on the device.
     groups, state = [], []
     for gi, sp in enumerate(specs):
-        W, G, M = wl.make_group(sp, rank_seed(args.config, gi, rank), dev)
+        W, G, M = wl.make_group(sp, 1000 * args.config + gi, dev)
         state.append((W, G, M))
         if args.weights == "fp32+bf16copy":
             copy = torch.zeros(W.shape, dtype=torch.bfloat16, device=dev)
@@ -298,25 +477,21 @@ def main():
     stream = torch.cuda.current_stream(dev)
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
         torch.cuda.synchronize(dev)
 
     alg_flops, dense_flops = wl.ns_flops(specs, hp.ns_steps)
-    # what the launch sequence asks of the tensor cores: less than the algorithmic count
-    # where the library takes two iterations per pass over X (wide matrices)
-    _, planned_flops = binding.muon_plan_flops([(s.rows, s.cols, s.count) for s in specs], hp.ns_steps)
+    shape_list = [(s.rows, s.cols, s.count) for s in specs]
+    planned, executed = binding.muon_plan_work(shape_list, hp.ns_steps)
     sbytes = wl.stream_bytes(specs)
 
-    # ---- device-resident timing ------------------------------------------------
+    # ---- device-resident timing: the headline, with no per-launch events -------------
     for _ in range(args.warmup):
         ctx.muon_step(hp)
     status, which = ctx.muon_status()
     if status != 0:
         raise SystemExit("device status %d at matrix %d during warm-up" % (status, which))
     launches_per_step = ctx.muon_last_launch_count()
-    ctx.muon_profile_enable(True)
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(gpu_uuid(dev))
     sampler.start()
     barrier()
     sampler.begin()
@@ -328,15 +503,23 @@ def main():
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
-    prof = ctx.muon_profile_read()
-    ctx.muon_profile_enable(False)
+    ms_step = e0.elapsed_time(e1) / args.steps
     status, which = ctx.muon_status()
     if status != 0:
         raise SystemExit("device status %d at matrix %d in the timed region" % (status, which))
-    ms_total = max_over_ranks(ms_total, dist, dev)
-    ms_step = ms_total / args.steps
-    value = whole_job_value(alg_flops, world, ms_step)
+    value = whole_job_value(alg_flops, ms_step)
+
+    # ---- the same steps again with an event pair around every launch: time per kernel kind --------
+    ctx.muon_profile_enable(True)
+    prof_steps = args.steps
+    e0.record(stream)
+    for _ in range(prof_steps):
+        ctx.muon_step(hp)
+    e1.record(stream)
+    barrier()
+    ms_step_profiled = e0.elapsed_time(e1) / prof_steps
+    prof = ctx.muon_profile_read()
+    ctx.muon_profile_enable(False)
 
     # ---- end to end through muon_step_host --------------------------------------
     e2e = None
@@ -358,85 +541,93 @@ def main():
             ctx.muon_step_host(hp, g_host, w_host)
         e1.record(stream)
         barrier()
-        ms_e2e = e0.elapsed_time(e1)
-        ms_e2e = max_over_ranks(ms_e2e, dist, dev) / e2e_steps
-        e2e = {"value": whole_job_value(alg_flops, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
-
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
+        ms_e2e = e0.elapsed_time(e1) / e2e_steps
+        # the copies alone, one direction at a time: what the host link of this machine gives
+        n_copy = 3
+        e0.record(stream)
+        for _ in range(n_copy):
+            for (W, G, M), gh in zip([st for st in state if len(st) == 3], g_host):
+                for i, t in enumerate(gh):
+                    G[i].copy_(t, non_blocking=True)
+        e1.record(stream)
+        barrier()
+        ms_up = e0.elapsed_time(e1) / n_copy
+        e0.record(stream)
+        for _ in range(n_copy):
+            for (W, G, M), wh in zip([st for st in state if len(st) == 3], w_host):
+                for i, t in enumerate(wh):
+                    t.copy_(W[i], non_blocking=True)
+        e1.record(stream)
+        barrier()
+        ms_down = e0.elapsed_time(e1) / n_copy
+        floor = max(ms_step, ms_up, ms_down)
+        e2e = {"value": whole_job_value(alg_flops, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "h2d_gbs_in_step": h2d / (ms_e2e * 1e-3) / 1e9, "d2h_gbs_in_step": d2h / (ms_e2e * 1e-3) / 1e9,
+               "h2d_alone_ms": ms_up, "h2d_alone_gbs": h2d / (ms_up * 1e-3) / 1e9,
+               "d2h_alone_ms": ms_down, "d2h_alone_gbs": d2h / (ms_down * 1e-3) / 1e9,
+               "over_floor": ms_e2e / floor,
+               "floor": "max(device-resident step, upload alone, download alone) = %.2f ms" % floor}
 
     # ---- roofline of the dominant kernel -----------------------------------------
     peaks = load_peaks()
-    gemm_ms = sum(prof[k][0] for k in ("gram", "poly", "comb"))
-    gemm_launches = sum(prof[k][1] for k in ("gram", "poly", "comb"))
+    roofline, per_kind = gemm_rooflines(prof, prof_steps, alg_flops, dense_flops, planned, executed, peaks, clocks)
     mom_ms, mom_launches = prof["momentum"]
-    per_kernel = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
+    per_kernel = {k: {"ms_per_step": v[0] / prof_steps, "launches_per_step": v[1] / prof_steps}
                   for k, v in prof.items() if v[1]}
-    roofline = None
-    if gemm_launches:
-        achieved = alg_flops * args.steps / (gemm_ms * 1e-3) / 1e12
-        peak = float(peaks.get("bf16_tflops_sustained", peaks.get("bf16_tflops")))
-        roofline = {
-            "kernel": "ns_gemm_kernel (gram + poly + comb launches)", "bound": "tensor",
-            "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-            "peak_source": "%s bf16_tflops_sustained" % peaks["_source"],
-            "frac_of_measured_burst": achieved / float(peaks.get("bf16_tflops", peak)),
-            "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
-            "dense_equivalent_tflops": dense_flops * args.steps / (gemm_ms * 1e-3) / 1e12,
-            "avg_launch_ms": gemm_ms / gemm_launches,
-            "flops_per_launch": alg_flops * args.steps / gemm_launches,
-            "planned_tflops": planned_flops * args.steps / (gemm_ms * 1e-3) / 1e12,
-            "frac_planned": planned_flops * args.steps / (gemm_ms * 1e-3) / 1e12 / peak,
-            "planned_over_algorithmic_flops": planned_flops / alg_flops,
-            "traffic": None,
-        }
-        if args.config == 3 and hp.ns_steps == 5:
+    for k, extra in per_kind.items():
+        per_kernel[k].update(extra)
+    if roofline is not None:
+        roofline["timed"] = "CUDA event pairs around every launch, %d steps after the headline loop (%.3f ms per step with the events, %.3f without)" % (prof_steps, ms_step_profiled, ms_step)
+        if args.config == 3 and hp.ns_steps == 5 and NCU_CAPTURE.get("gemm_bytes_per_step"):
             scale = sum(s.count for s in specs) / NCU_CAPTURE["matrices"]
             roofline["traffic"] = NCU_CAPTURE["gemm_bytes_per_step"] * scale / NCU_CAPTURE["gemm_launches_per_step"]
             roofline["traffic_note"] = "DRAM bytes per launch (average of the 16 launches of a step), scaled from a 64-matrix ncu capture"
     stream_roof = None
     if mom_launches:
-        gbs = sbytes * args.steps / (mom_ms * 1e-3) / 1e9
+        gbs = sbytes * prof_steps / (mom_ms * 1e-3) / 1e9
         stream_roof = {"kernel": "momentum_tma_kernel", "bound": "hbm", "achieved": gbs,
                        "peak": float(peaks["hbm_gbs"]), "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]),
                        "peak_source": "%s hbm_gbs" % peaks["_source"], "frac_of_nominal": gbs / NOMINAL_HBM_GBS,
                        "bytes_per_element": sbytes / wl.group_params(specs), "traffic": None,
-                       "algorithmic_bytes_per_launch": sbytes / max(1, mom_launches // args.steps)}
-        if args.config == 3:
+                       "algorithmic_bytes_per_launch": sbytes / max(1, mom_launches // prof_steps)}
+        if args.config == 3 and NCU_CAPTURE.get("momentum_bytes_per_launch"):
             stream_roof["traffic"] = NCU_CAPTURE["momentum_bytes_per_launch"] * sum(s.count for s in specs) / NCU_CAPTURE["matrices"]
 
     # ---- shape sweep: every shape of the configuration on its own ---------------------
     shapes = None
-    if args.config == 4 and world == 1:
+    if args.config == 4:
         shapes = []
         ctx.muon_destroy()
         for gi, sp in enumerate(specs):
             one = binding.MuonContext([groups[gi]])
             for _ in range(args.warmup):
                 one.muon_step(hp)
-            one.muon_profile_enable(True)
             torch.cuda.synchronize(dev)
             e0.record(stream)
             for _ in range(args.steps):
                 one.muon_step(hp)
             e1.record(stream)
             torch.cuda.synchronize(dev)
+            ms = e0.elapsed_time(e1) / args.steps
+            one.muon_profile_enable(True)
+            for _ in range(args.steps):
+                one.muon_step(hp)
             pr = one.muon_profile_read()
             one.muon_profile_enable(False)
-            ms = e0.elapsed_time(e1) / args.steps
             g_ms = sum(pr[k][0] for k in ("gram", "poly", "comb")) / args.steps
             fl, _ = wl.ns_flops([sp], hp.ns_steps)
-            _, fl_planned = binding.muon_plan_flops([(sp.rows, sp.cols, sp.count)], hp.ns_steps)
+            pl, ex = binding.muon_plan_work([(sp.rows, sp.cols, sp.count)], hp.ns_steps)
+            fl_planned, fl_executed = sum(pl.values()), sum(ex.values())
             m_, n_ = min(sp.rows, sp.cols), max(sp.rows, sp.cols)
             blocks, pairs = -(-m_ // 128), -(-(-(-m_ // 128)) // 2)
             shapes.append({"shape": "%dx%d" % (sp.rows, sp.cols), "ms_per_step": ms,
+                           "launches_per_step": one.muon_last_launch_count(),
                            "step_tflops": fl / (ms * 1e-3) / 1e12,
                            "gemm_tflops": fl / (g_ms * 1e-3) / 1e12,
                            "gemm_frac_of_measured_sustained": fl / (g_ms * 1e-3) / 1e12 / float(peaks.get("bf16_tflops_sustained", 1400.0)),
                            "gemm_planned_tflops": fl_planned / (g_ms * 1e-3) / 1e12,
+                           "gemm_executed_tflops": fl_executed / (g_ms * 1e-3) / 1e12,
                            "iterations_in_pairs": fl_planned < fl,
                            "row_blocks": blocks, "cta_pairs_per_column_tile": pairs})
             one.muon_destroy()
@@ -444,7 +635,7 @@ def main():
 
     # ---- AdamW for the parameters Muon does not handle: embedding-sized tensors -------
     adamw = None
-    if not args.no_adamw and world == 1:
+    if not args.no_adamw:
         torch.cuda.empty_cache()
         shape = (163840, 2048)  # Moonlight's embedding / LM head
         ps = [torch.zeros(shape, dtype=torch.bfloat16, device=dev) for _ in range(2)]
@@ -469,21 +660,21 @@ def main():
         del ps, gs, ms_, vs
 
     cpu_baseline = None
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline:
         fl, secs, desc, threads = oracle_sample_time(specs, hpd, budget_s=args.ref_budget, max_mats=args.ref_mats)
         cpu_baseline = {"value": fl / secs / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": desc, "seconds": secs}
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD_NAMES[args.config], "matrices": sum(s.count for s in specs),
                    "params": wl.group_params(specs), "ns_steps": hp.ns_steps, "weights": args.weights,
                    "l2": "inputs exceed L2" if wl.group_params(specs) * 8 > 126e6 else "inputs fit L2",
                    "algorithmic_tflop_per_step": alg_flops / 1e12},
-        "pct_bf16_peak_measured_sustained": 100.0 * value / world / float(peaks.get("bf16_tflops_sustained", 1400.0)),
-        "pct_bf16_peak_nominal": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
+        "pct_bf16_peak_measured_sustained": 100.0 * value / float(peaks.get("bf16_tflops_sustained", 1400.0)),
+        "pct_bf16_peak_nominal": 100.0 * value / NOMINAL_BF16_TFLOPS,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline, "roofline_stream": stream_roof, "kernels": per_kernel,
         "cpu_baseline": cpu_baseline,
@@ -494,8 +685,6 @@ def main():
         line["roofline_adamw"] = adamw
     print(json.dumps(line))
     ctx.muon_destroy()
-    if dist is not None:
-        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -161,6 +161,28 @@ int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_byt
 int muon_partition(const muon_group* groups, int n_groups, int world, int* owner_out, double* load_out);
 
 /*
+ * The same ownership question answered for storage that can be gathered in
+ * place.  Every shape bucket (numbering of muon_plan_buckets) is cut into
+ * `world` slots of share_out[bucket] = ceil(count / world) matrices; rank r owns
+ * the matrices of slot r, which fill it from the front (a slot may hold one
+ * matrix fewer than its capacity, or none when the bucket has fewer matrices
+ * than ranks).  If a bucket's weights are stored slot after slot - matrix i at
+ * index owner_out[i] * share + pos_out[i] of a [world * share] array of
+ * matrices - the all-gather of the updated weights (Algorithm 1, last exchange)
+ * writes every rank's slot where it already lives, and a reduce-scatter of
+ * gradients stored the same way (Algorithm 1, first line) leaves every owner
+ * with the reduced gradients of exactly its matrices; neither needs a staging
+ * copy.  Within a bucket the matrices go to the ranks in consecutive runs,
+ * groups in order; which ranks get the longer runs is decided by the
+ * Newton-Schulz work (3 m^2 n + m^3 per matrix) accumulated over the earlier
+ * buckets, so that the load stays balanced to within one matrix per bucket.
+ * Pure host computation; owner_out, pos_out: one int per matrix (HOST);
+ * share_out: one int per bucket (HOST); load_out: world doubles or NULL.
+ */
+int muon_partition_slots(const muon_group* groups, int n_groups, int world, int* owner_out, int* pos_out,
+                         int* share_out, double* load_out);
+
+/*
  * Build a context: validate the descriptors, form shape buckets, carve the
  * caller's workspace (DEVICE memory, 1024-byte aligned, at least
  * muon_workspace_bytes() long, owned by the caller, alive until destroy),

@@ -30,7 +30,7 @@ MUON_TAP_X0, MUON_TAP_A, MUON_TAP_B, MUON_TAP_X = 0, 1, 2, 3
 MUON_SCALE_ADJUSTED_LR, MUON_SCALE_FIXED_DIM, MUON_SCALE_UPDATE_NORM = 0, 1, 2
 
 EXPORTED = [
-    "muon_workspace_bytes", "muon_partition", "muon_plan_buckets", "muon_plan_flops", "muon_plan_work", "muon_debug_tile_table", "muon_init", "muon_step", "muon_step_bucket",
+    "muon_workspace_bytes", "muon_partition", "muon_partition_slots", "muon_plan_buckets", "muon_plan_flops", "muon_plan_work", "muon_debug_tile_table", "muon_init", "muon_step", "muon_step_bucket",
     "muon_step_host", "muon_status",
     "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
     "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes", "muon_debug_set_pair_fold",
@@ -94,6 +94,8 @@ def lib():
     L = C.CDLL(LIB_PATH)
     L.muon_workspace_bytes.argtypes = [C.POINTER(muon_group), C.c_int, C.POINTER(C.c_size_t)]
     L.muon_partition.argtypes = [C.POINTER(muon_group), C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_double)]
+    L.muon_partition_slots.argtypes = [C.POINTER(muon_group), C.c_int, C.c_int, C.POINTER(C.c_int),
+                                       C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_double)]
     L.muon_init.argtypes = [C.POINTER(C.c_void_p), C.POINTER(muon_group), C.c_int, C.c_void_p, C.c_size_t, C.c_int]
     L.muon_step.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_void_p]
     L.muon_plan_buckets.argtypes = [C.POINTER(muon_group), C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
@@ -285,6 +287,21 @@ def muon_partition(shapes, world: int):
     loads = (C.c_double * world)()
     _check(lib().muon_partition(arr, len(shapes), int(world), owners, loads))
     return list(owners), list(loads)
+
+
+def muon_partition_slots(shapes, world: int):
+    """Slot partition for in-place collectives.  ``shapes`` is a list of (rows,
+    cols, count, w_dtype code, g_dtype code); returns (owner per matrix, position
+    in the owner's slot per matrix, slot capacity per bucket, load per rank)."""
+    arr = shape_only_groups(shapes)
+    total = sum(sh[2] for sh in shapes)
+    _, n_buckets = muon_plan_buckets(shapes)
+    owners = (C.c_int * total)()
+    pos = (C.c_int * total)()
+    share = (C.c_int * n_buckets)()
+    loads = (C.c_double * world)()
+    _check(lib().muon_partition_slots(arr, len(shapes), int(world), owners, pos, share, loads))
+    return list(owners), list(pos), list(share), list(loads)
 
 
 def muon_plan_flops(shapes, ns_steps: int = 5):

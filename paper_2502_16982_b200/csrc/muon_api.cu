@@ -586,6 +586,46 @@ int muon_partition(const muon_group* groups, int n_groups, int world, int* owner
   return MUON_OK;
 }
 
+int muon_partition_slots(const muon_group* groups, int n_groups, int world, int* owner_out, int* pos_out,
+                         int* share_out, double* load_out) {
+  if (!owner_out || !pos_out || !share_out || world <= 0)
+    return fail(MUON_ERR_INVALID_ARG, "an output pointer is null or world <= 0");
+  int rc = validate_groups(groups, n_groups, false);
+  if (rc) return rc;
+  std::vector<Bucket> buckets;
+  PlanSizes sizes;
+  int total;
+  rc = make_plan(groups, n_groups, &buckets, &sizes, &total);
+  if (rc) return rc;
+  std::vector<double> load(world, 0.0);
+  std::vector<int> order(world);
+  for (size_t b = 0; b < buckets.size(); ++b) {
+    const Bucket& B = buckets[b];
+    const int cnt = static_cast<int>(B.mats.size());
+    const double m = B.m, n = B.n, cost = 3.0 * m * m * n + m * m * m;
+    const int base = cnt / world, extra = cnt % world;
+    share_out[b] = base + (extra ? 1 : 0);
+    // the `extra` ranks with one matrix more are the least loaded so far (ties: lower rank)
+    for (int r = 0; r < world; ++r) order[r] = r;
+    std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return load[x] < load[y]; });
+    std::vector<int> mine(world, base);
+    for (int k = 0; k < extra; ++k) mine[order[k]] += 1;
+    // consecutive runs of the bucket's matrices, rank by rank
+    int next = 0;
+    for (int r = 0; r < world; ++r) {
+      for (int k = 0; k < mine[r]; ++k) {
+        const int g = B.mats[next++].global;
+        owner_out[g] = r;
+        pos_out[g] = k;
+      }
+      load[r] += mine[r] * cost;
+    }
+  }
+  if (load_out)
+    for (int r = 0; r < world; ++r) load_out[r] = load[r];
+  return MUON_OK;
+}
+
 int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_bytes) {
   if (!out_bytes) return fail(MUON_ERR_INVALID_ARG, "out_bytes is null");
   int rc = validate_groups(groups, n_groups, false);

@@ -665,7 +665,8 @@ def test_bucket_by_bucket_step_gives_muon_step_bits():
 
 def test_distributed_wrapper_single_rank_steps_bucket_by_bucket():
     """The data-parallel wrapper with one rank owns every matrix and must give
-    the plain context's bits (its momentum starts at zero like the plain one's)."""
+    the plain context's bits (its momentum starts at zero like the plain one's);
+    its matrices are views into the flat per-bucket storage."""
     b = _binding()
     from paper_2502_16982_b200.distributed import DistributedMuon
     specs = [wl.GroupSpec(328, 200, 3, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
@@ -673,21 +674,23 @@ def test_distributed_wrapper_single_rank_steps_bucket_by_bucket():
              wl.GroupSpec(128, 384, 2, torch.float32, torch.float32, 0.02, 1.0)]
     hp = default_hp(lr=1e-2)
     plain = Case(specs, seed=73)
-    other = Case(specs, seed=73)
-    dm = DistributedMuon([([W[i] for i in range(sp.count)], [G[i] for i in range(sp.count)])
-                          for sp, (W, G, M) in zip(specs, other.dev)])
+    dm = DistributedMuon([(sp.rows, sp.cols, sp.count, sp.w_dtype, sp.g_dtype) for sp in specs], "cuda")
     try:
         assert dm.n_units == 2
+        for gi, sp in enumerate(specs):
+            for i in range(sp.count):
+                dm.weights[gi][i].copy_(plain.dev[gi][0][i])
+                dm.grads[gi][i].copy_(plain.dev[gi][1][i])
         for _ in range(2):
             assert plain.step(hp)[0] == 0
             dm.step(hp)
-        torch.cuda.synchronize()
-        for gi in range(len(specs)):
-            assert torch.equal(plain.dev[gi][0], other.dev[gi][0])
+        assert dm.status()[0] == 0
+        for gi, sp in enumerate(specs):
+            for i in range(sp.count):
+                assert torch.equal(plain.dev[gi][0][i], dm.weights[gi][i])
     finally:
         dm.close()
         plain.close()
-        other.close()
 
 
 def test_step_captured_in_a_cuda_graph_replays_the_eager_bits():
