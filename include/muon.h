@@ -372,6 +372,21 @@ int muon_debug_wait_expiry(muon_ctx* ctx, void* stream, int matrix_index, unsign
 size_t muon_debug_set_chunk_bytes(size_t bytes);
 
 /*
+ * Knob: how tiles are cut where row blocks of 128 do not pair up.  Bit 0: a row
+ * block without a partner (an odd number of row blocks in the combine) is a
+ * half-height tile - UMMA M = 128, 64 rows per CTA, half a full tile's time -
+ * instead of a full tile whose second CTA works on rows beyond the matrix.
+ * Bit 1: the diagonal blocks of a symmetric product that no full tile can hold
+ * without waste are half-height, half-width tiles, instead of sharing a
+ * full-width tile with the neighbour matrix's (cross blocks dropped).  Default
+ * 1 (bit 1 computes nothing in vain but measured slower).  Process-wide, read where muon_debug_set_pair_fold is.  Returns the
+ * previous mode; a value outside 0..3 only queries.  The modes agree to
+ * rounding, not bit for bit (instructions of different heights round their
+ * sums differently); within one mode results are reproducible bit for bit.
+ */
+int muon_debug_set_tile_mode(int mode);
+
+/*
  * Knob: where the planner takes two iterations per pass over X (Eq. 2 gives
  * X_{k+1} = P_k X_k with P_k = a*I + b*A_k + c*A_k^2, so A_{k+1} = P_k^2 A_k and
  * X_{k+2} = P_{k+1} P_k X_k need no Gram product and no combine for the second
@@ -393,11 +408,12 @@ int muon_debug_set_pair_fold(int mode);
  * of a rows x cols matrix use.  which = 0: products with a symmetric result,
  * table of one unit of *unit_mats matrices; 1: the same for a last matrix
  * without a partner (empty when units are single matrices); 2: the combine;
- * 3: the combine formed transposed.  Every tile is nine int16 in `out` (room
+ * 3: the combine formed transposed.  Every tile is ten int16 in `out` (room
  * for cap_tiles tiles; NULL only queries the count): row block of CTA 0 and of
  * CTA 1, column block of the first and of the second 128 accumulator columns,
  * width in column blocks (1 or 2), matrix of CTA 0 and of CTA 1 within the unit,
- * and per CTA a mask of the column halves whose 128 x 128 block is stored.
+ * per CTA a mask of the column halves whose 128 x 128 block is stored, and 1 for
+ * a half-height tile (one row block, 64 rows per CTA; its mask is the first).
  */
 int muon_debug_tile_table(int rows, int cols, int which, int16_t* out, int cap_tiles, int* n_tiles, int* unit_mats);
 

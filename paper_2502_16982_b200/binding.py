@@ -33,7 +33,7 @@ EXPORTED = [
     "muon_workspace_bytes", "muon_partition", "muon_partition_slots", "muon_plan_buckets", "muon_plan_flops", "muon_plan_work", "muon_debug_tile_table", "muon_init", "muon_step", "muon_step_bucket",
     "muon_step_host", "muon_status",
     "muon_get_norms", "muon_get_update_rms", "muon_destroy", "muon_last_error", "muon_last_launch_count",
-    "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes", "muon_debug_set_pair_fold",
+    "muon_debug_keep", "muon_debug_read", "muon_debug_set_chunk_bytes", "muon_debug_set_pair_fold", "muon_debug_set_tile_mode",
     "muon_debug_wait_expiry",
     "muon_profile_enable", "muon_profile_read", "muon_debug_tmem_bases",
     "muon_momentum_norm_static", "muon_adamw_step",
@@ -123,6 +123,7 @@ def lib():
                                             C.c_int, C.c_float, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
     L.muon_debug_set_chunk_bytes.argtypes = [C.c_size_t]
     L.muon_debug_set_pair_fold.argtypes = [C.c_int]
+    L.muon_debug_set_tile_mode.argtypes = [C.c_int]
     L.muon_debug_wait_expiry.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_uint]
     L.muon_adamw_step.argtypes = [C.POINTER(muon_adamw_tensor), C.c_int, C.POINTER(muon_adamw_hparams), C.c_int,
                                   C.c_void_p]
@@ -331,13 +332,21 @@ def muon_debug_tile_table(rows: int, cols: int, which: int):
     two accumulator halves, the width ``nbw`` and the ``keep`` masks."""
     n, unit = C.c_int(0), C.c_int(0)
     _check(lib().muon_debug_tile_table(rows, cols, which, None, 0, C.byref(n), C.byref(unit)))
-    buf = (C.c_int16 * (9 * max(1, n.value)))()
+    buf = (C.c_int16 * (10 * max(1, n.value)))()
     _check(lib().muon_debug_tile_table(rows, cols, which, buf, n.value, C.byref(n), C.byref(unit)))
     tiles = []
     for k in range(n.value):
-        v = buf[9 * k:9 * k + 9]
-        tiles.append({"i": (v[0], v[1]), "j": (v[2], v[3]), "nbw": v[4], "dm": (v[5], v[6]), "keep": (v[7], v[8])})
+        v = buf[10 * k:10 * k + 10]
+        tiles.append({"i": (v[0], v[1]), "j": (v[2], v[3]), "nbw": v[4], "dm": (v[5], v[6]), "keep": (v[7], v[8]),
+                      "half": v[9]})
     return tiles, unit.value
+
+
+def muon_debug_set_tile_mode(mode: int) -> int:
+    """How tiles are cut where row blocks do not pair up (bit 0: half-height
+    tiles for a row block without a partner, bit 1: for lone diagonal blocks of
+    symmetric products; default 1).  Returns the previous mode."""
+    return lib().muon_debug_set_tile_mode(int(mode))
 
 
 def muon_debug_set_pair_fold(mode: int) -> int:

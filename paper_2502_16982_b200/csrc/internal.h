@@ -55,8 +55,13 @@ struct DevStatus {
 //             column block j[1]; CTA r stages the operand-B rows of block j[r],
 //             taken from ITS matrix;
 //   nbw == 1: the columns are block j[0]; each CTA stages 64 of its rows.
+// half != 0: a half-height tile (UMMA M = 128 over the pair instead of 256).  The
+// pair computes ONE row block, i[0], its upper 64 rows in CTA 0 and its lower 64
+// in CTA 1, against the same columns; dm[0] names the matrix.  It costs half a
+// full tile's tensor-core time, so a row block that has no partner (an odd
+// number of row blocks, a lone diagonal block) wastes nothing.
 // keep[r] bit h set: the 128 x 128 block (rows of CTA r, column half h) is
-// stored.  The other blocks of the product are computed and dropped: a block
+// stored (half-height tiles: keep[0] bit h for column half h of the row block).  The other blocks of the product are computed and dropped: a block
 // below the diagonal of a symmetric result, or the cross terms of a tile whose
 // two CTAs work on different matrices.
 // The row blocks (and, for a symmetric operand B, the column blocks) of one
@@ -68,7 +73,8 @@ struct PairTile {
   unsigned char nbw;
   unsigned char dm[2];
   unsigned char keep[2];
-  unsigned char pad_[3];
+  unsigned char half;
+  unsigned char pad_[2];
 };
 static_assert(sizeof(PairTile) == 16, "PairTile is read as one 16-byte entry");
 

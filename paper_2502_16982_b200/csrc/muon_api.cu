@@ -64,6 +64,11 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 constexpr size_t kChunkBytesDefault = size_t(8) << 30;
 size_t g_chunk_bytes_max = kChunkBytesDefault;  // process-wide; see muon_debug_set_chunk_bytes
 constexpr int kChunkCountMax = 4096;
+// Gradient bytes per slice of the host-buffer step (muon_step_host).
+#ifndef MUON_HOST_SLICE_BYTES
+#define MUON_HOST_SLICE_BYTES (size_t(32) << 20)
+#endif
+constexpr size_t kHostSliceBytes = MUON_HOST_SLICE_BYTES;
 
 // Two iterations per pass over X.  With P_k = a*I + b*A_k + c*A_k^2 (symmetric, a
 // polynomial in A_k = X_k X_k^T) Eq. 2 reads X_{k+1} = P_k X_k, hence
@@ -280,75 +285,89 @@ PairTile make_tile(int i0, int i1, int j0, int j1, int nbw, int dm0, int dm1, un
   return t;
 }
 
-// Tiles of the symmetric products (only the 128-blocks on or above the diagonal
-// are produced) for matrix `dm` of a unit, nb row blocks.  A tile is two
-// neighbouring row blocks times two neighbouring column blocks.
-//  * nb even: row pair (r, r+1), r even, takes columns r, r+1, then r+2, r+3, ...:
-//    every tile is full width; the first one holds the block (r+1, r) below the
-//    diagonal, which is computed and dropped (nb/2 blocks of nb(nb+1)/2 + nb/2).
-//  * nb odd: row pair (r, r+1) takes columns r+1, r+2, then r+3, r+4, ...: an even
-//    number of columns, every block of every tile is kept.  That leaves the
-//    diagonal blocks (r, r), r even, which no full tile can hold (the block
-//    below it in the pair lies under the diagonal).  `lone` receives them.
-void sym_tiles_of_matrix(int nb, int dm, std::vector<PairTile>* tiles, std::vector<int>* lone) {
-  if (nb % 2 == 0) {
-    for (int r = 0; r < nb; r += 2)
-      for (int c = r; c < nb; c += 2)
-        tiles->push_back(make_tile(r, r + 1, c, c + 1, 2, dm, dm, 3u, c == r ? 2u : 3u));
-    return;
-  }
-  for (int r = 0; r + 1 < nb; r += 2)
-    for (int c = r + 1; c + 1 < nb; c += 2) tiles->push_back(make_tile(r, r + 1, c, c + 1, 2, dm, dm, 3u, 3u));
-  for (int r = 0; r < nb; r += 2) lone->push_back(r);
+// A half-height tile: row block i alone (64 rows in each CTA) against column blocks j0 (, j1).
+PairTile make_half_tile(int i, int j0, int j1, int nbw, int dm, unsigned keep) {
+  PairTile t = make_tile(i, i, j0, j1, nbw, dm, dm, keep, 0u);
+  t.half = 1;
+  return t;
 }
 
-// Tile tables of a bucket.  Symmetric products with an odd number of row blocks
-// work on units of two matrices: the lone diagonal blocks (r, r) of the two
-// share a full-width tile, one CTA per matrix, whose two cross blocks are
-// dropped; a matrix alone takes them as half-width tiles instead.
+// How tiles are cut where the row blocks do not pair up; see muon_debug_set_tile_mode.
+// bit 0: a row block without a partner is taken at half height; bit 1: so is a lone diagonal block.
+// Measured on the expert bucket (1408 rows = 11 row blocks): mode 1 13.49 ms per step, mode 0 13.67,
+// mode 3 13.67, mode 2 13.83: the half-height, half-width tiles of bit 1 run too far below the
+// tensor cores' rate to pay, although they compute nothing in vain.
+int g_tile_mode = 1;
+
+// Tiles of the symmetric products (only the 128-blocks on or above the diagonal
+// are produced) for matrix `dm` of a unit, nb row blocks.  A full tile is two
+// neighbouring row blocks times two neighbouring column blocks.  Row pair
+// (r, r+1), r even, takes the columns from r+1 on two at a time (a last single
+// column as a tile of half the width); every block of these tiles is kept.  That
+// leaves the diagonal blocks (r, r), r even, which no full tile can hold without
+// waste (the block below it in the pair lies under the diagonal): with
+// `half_lone` each becomes a half-height, half-width tile, otherwise `lone`
+// receives them.
+void sym_tiles_of_matrix(int nb, int dm, bool half_lone, std::vector<PairTile>* tiles, std::vector<int>* lone) {
+  for (int r = 0; r < nb; r += 2) {
+    if (half_lone) tiles->push_back(make_half_tile(r, r, r, 1, dm, 1u));
+    else lone->push_back(r);
+    if (r + 1 >= nb) break;
+    for (int c = r + 1; c < nb; c += 2) {
+      const int w = std::min(2, nb - c);
+      tiles->push_back(make_tile(r, r + 1, c, c + 1, w, dm, dm, w == 2 ? 3u : 1u, w == 2 ? 3u : 1u));
+    }
+  }
+}
+
+// Tile tables of a bucket.
 void build_tile_tables(Bucket* Bp) {
   Bucket& B = *Bp;
   const int nb = ceil_div(B.m, 128), ncb = ceil_div(B.n, 128), np = ceil_div(nb, 2);
+  const bool half_rows = (g_tile_mode & 1) != 0, half_lone = (g_tile_mode & 2) != 0;
   B.sym_tiles.clear();
   B.sym_tiles_tail.clear();
   B.comb_tiles.clear();
   B.comb_tiles_t.clear();
   B.sym_acc_cols = B.comb_acc_cols = 128;
   std::vector<int> lone;
-  if (nb % 2 == 0) {
+  if (half_lone) {
     B.sym_unit_mats = 1;
-    sym_tiles_of_matrix(nb, 0, &B.sym_tiles, &lone);
+    sym_tiles_of_matrix(nb, 0, true, &B.sym_tiles, &lone);
   } else {
+    // Without half-height tiles the lone diagonal blocks (r, r) of two matrices share a
+    // full-width tile, one CTA per matrix, whose two cross blocks are dropped; a matrix
+    // alone takes each with the block below it, which lies under the diagonal and is dropped.
     B.sym_unit_mats = 2;
-    sym_tiles_of_matrix(nb, 0, &B.sym_tiles, &lone);
+    sym_tiles_of_matrix(nb, 0, false, &B.sym_tiles, &lone);
     lone.clear();
-    sym_tiles_of_matrix(nb, 1, &B.sym_tiles, &lone);
+    sym_tiles_of_matrix(nb, 1, false, &B.sym_tiles, &lone);
     for (int r : lone) B.sym_tiles.push_back(make_tile(r, r, r, r, 2, 0, 1, 1u, 2u));
     lone.clear();
-    sym_tiles_of_matrix(nb, 0, &B.sym_tiles_tail, &lone);
-    // half width: rows (r, r+1) against column block r; the second CTA's block is under the diagonal
+    sym_tiles_of_matrix(nb, 0, false, &B.sym_tiles_tail, &lone);
     for (int r : lone) B.sym_tiles_tail.push_back(make_tile(r, r + 1, r, r, 1, 0, 0, 1u, 0u));
   }
   for (const PairTile& t : B.sym_tiles)
     if (t.nbw == 2) B.sym_acc_cols = 256;
-  // combine: row pair p covers row blocks 2p, 2p+1; column tiles are two 128-blocks
-  // wide, with one single block at the end of an odd run
-  for (int p = 0; p < np; ++p) {
-    for (int jb = 0; jb < ncb;) {
-      const int w = std::min(2, ncb - jb);
-      B.comb_tiles.push_back(make_tile(2 * p, 2 * p + 1, jb, jb + 1, w, 0, 0, w == 2 ? 3u : 1u, w == 2 ? 3u : 1u));
-      if (w == 2) B.comb_acc_cols = 256;
-      jb += w;
+  // combine: row pair p covers row blocks 2p, 2p+1 (a last row block without a partner
+  // at half height); column tiles are two 128-blocks wide, with one single block at the
+  // end of an odd run
+  auto rows_by_cols = [&](int row_blocks, int col_blocks, std::vector<PairTile>* out) {
+    for (int p = 0; p < ceil_div(row_blocks, 2); ++p) {
+      const bool single = 2 * p + 1 >= row_blocks && half_rows;
+      for (int jb = 0; jb < col_blocks;) {
+        const int w = std::min(2, col_blocks - jb);
+        if (single) out->push_back(make_half_tile(2 * p, jb, jb + 1, w, 0, w == 2 ? 3u : 1u));
+        else out->push_back(make_tile(2 * p, 2 * p + 1, jb, jb + 1, w, 0, 0, w == 2 ? 3u : 1u, w == 2 ? 3u : 1u));
+        jb += w;
+      }
     }
-  }
+  };
+  rows_by_cols(nb, ncb, &B.comb_tiles);
+  if (ncb >= 2) B.comb_acc_cols = 256;
   // the same product with the roles of the sides exchanged (as many tiles)
-  for (int p = 0; p < ceil_div(ncb, 2); ++p) {
-    for (int jb = 0; jb < nb;) {
-      const int w = std::min(2, nb - jb);
-      B.comb_tiles_t.push_back(make_tile(2 * p, 2 * p + 1, jb, jb + 1, w, 0, 0, w == 2 ? 3u : 1u, w == 2 ? 3u : 1u));
-      jb += w;
-    }
-  }
+  rows_by_cols(ncb, nb, &B.comb_tiles_t);
+  (void)np;
 }
 
 // Forms the shape buckets and lays out the workspace.  Deterministic in the
@@ -639,6 +658,12 @@ int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_byt
   return MUON_OK;
 }
 
+int muon_debug_set_tile_mode(int mode) {
+  const int prev = g_tile_mode;
+  if (mode >= 0 && mode <= 3) g_tile_mode = mode;
+  return prev;
+}
+
 int muon_debug_set_pair_fold(int mode) {
   const int prev = g_pair_fold_mode;
   if (mode >= 0 && mode <= 4) g_pair_fold_mode = mode;
@@ -697,7 +722,8 @@ int muon_plan_work(const muon_group* groups, int n_groups, int ns_steps, double*
   // contraction length in whole 64-element pipeline stages
   auto table_flops = [](const std::vector<PairTile>& t, int k) {
     double f = 0.0;
-    for (const PairTile& e : t) f += 2.0 * 256.0 * (128.0 * e.nbw) * (static_cast<double>(ceil_div(k, kBK)) * kBK);
+    for (const PairTile& e : t)
+      f += 2.0 * (e.half ? 128.0 : 256.0) * (128.0 * e.nbw) * (static_cast<double>(ceil_div(k, kBK)) * kBK);
     return f;
   };
   for (const Bucket& B : buckets) {
@@ -736,9 +762,9 @@ int muon_debug_tile_table(int rows, int cols, int which, int16_t* out, int cap_t
   if (out) {
     if (cap_tiles < *n_tiles) return fail(MUON_ERR_INVALID_ARG, "table has %d tiles, room for %d", *n_tiles, cap_tiles);
     for (size_t k = 0; k < t.size(); ++k) {
-      int16_t* o = out + 9 * k;
+      int16_t* o = out + 10 * k;
       o[0] = t[k].i[0]; o[1] = t[k].i[1]; o[2] = t[k].j[0]; o[3] = t[k].j[1]; o[4] = t[k].nbw;
-      o[5] = t[k].dm[0]; o[6] = t[k].dm[1]; o[7] = t[k].keep[0]; o[8] = t[k].keep[1];
+      o[5] = t[k].dm[0]; o[6] = t[k].dm[1]; o[7] = t[k].keep[0]; o[8] = t[k].keep[1]; o[9] = t[k].half;
     }
   }
   return MUON_OK;
@@ -1256,15 +1282,22 @@ int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* con
   for (size_t b = 0; b < ctx->buckets.size(); ++b) {
     const Bucket& B = ctx->buckets[b];
     const int total = static_cast<int>(B.mats.size());
-    const int slice = std::max(1, std::min(B.chunk, (total + 7) / 8));  // eight slices per bucket measured best
+    // Slices of about kHostSliceBytes of gradients: short enough that the first upload and the last
+    // download, which nothing overlaps, are a small part of the step, long enough to keep the launches few.
+    const size_t g_bytes_per_mat = static_cast<size_t>(B.m) * B.n * (B.g_dtype == MUON_DTYPE_FP32 ? 4 : 2);
+    const int slice = static_cast<int>(std::max<size_t>(1, std::min<size_t>(B.chunk, std::max<size_t>(1, kHostSliceBytes / g_bytes_per_mat))));
     for (int first = 0; first < total; first += slice) {
       const int count = std::min(slice, total - first);
       for (int i = first; i < first + count && ce == cudaSuccess; ++i) {
         const MatRef& r = B.mats[i];
         const muon_group& G = ctx->groups[r.group];
         const size_t es = G.g_dtype == MUON_DTYPE_FP32 ? 4 : 2;
-        ce = cudaMemcpy2DAsync(const_cast<void*>(G.g[r.index]), G.ld_g * es, g_host[r.group][r.index], G.cols * es,
-                               G.cols * es, G.rows, cudaMemcpyHostToDevice, ctx->s_in);
+        if (G.ld_g == G.cols)  // dense on both sides: one linear copy
+          ce = cudaMemcpyAsync(const_cast<void*>(G.g[r.index]), g_host[r.group][r.index],
+                               static_cast<size_t>(G.rows) * G.cols * es, cudaMemcpyHostToDevice, ctx->s_in);
+        else
+          ce = cudaMemcpy2DAsync(const_cast<void*>(G.g[r.index]), G.ld_g * es, g_host[r.group][r.index], G.cols * es,
+                                 G.cols * es, G.rows, cudaMemcpyHostToDevice, ctx->s_in);
       }
       if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gradient upload: %s", cudaGetErrorString(ce));
       ce = next_event(&ev);
@@ -1281,8 +1314,12 @@ int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* con
           const MatRef& r = B.mats[i];
           const muon_group& G = ctx->groups[r.group];
           const size_t es = G.w_dtype == MUON_DTYPE_FP32 ? 4 : 2;
-          ce = cudaMemcpy2DAsync(w_host[r.group][r.index], G.cols * es, G.w[r.index], G.ld_w * es, G.cols * es,
-                                 G.rows, cudaMemcpyDeviceToHost, ctx->s_out);
+          if (G.ld_w == G.cols)
+            ce = cudaMemcpyAsync(w_host[r.group][r.index], G.w[r.index], static_cast<size_t>(G.rows) * G.cols * es,
+                                 cudaMemcpyDeviceToHost, ctx->s_out);
+          else
+            ce = cudaMemcpy2DAsync(w_host[r.group][r.index], G.cols * es, G.w[r.index], G.ld_w * es, G.cols * es,
+                                   G.rows, cudaMemcpyDeviceToHost, ctx->s_out);
         }
         if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "weight download: %s", cudaGetErrorString(ce));
       }

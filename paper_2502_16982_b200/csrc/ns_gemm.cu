@@ -24,6 +24,12 @@
 //               rounding) and written back by a TMA store issued by the warp
 //               itself; the warps never wait for one another.
 //
+// A tile may also be half height (M = 128: 64 rows per CTA, both halves of one
+// row block).  The accumulator then lies differently in TMEM: lanes 0-63 of a
+// CTA hold its 64 rows against the first half of the N columns, lanes 64-127 the
+// same rows against the second half (both in TMEM columns [0, N/2)), so epilogue
+// warp q owns rows 32 (q & 1) .. + 31 of the CTA and column half q >> 1.
+//
 // Symmetric matrices (A and B) are kept as their 128x128 blocks on or above
 // the diagonal only.  The products that produce them visit only column blocks
 // j >= 2p of row pair p and drop the one below-diagonal block (2p+1, 2p) the
@@ -176,19 +182,21 @@ __device__ __forceinline__ TilePlan plan_tile(const GemmParams& P, int tile, int
   return t;
 }
 
-// Walks the stream of 64-column quarters one CTA's epilogue processes: tiles in
-// the CTA pair's order, within a tile the quarters that hold output of this CTA
-// (`qmask`: bit qd set = quarter qd, accumulator columns [64 qd, 64 qd + 64),
-// is still to be stored).
+// Walks the stream of 64-column quarters one epilogue warp processes: tiles in
+// the CTA pair's order, within a tile the quarters that hold output of this warp
+// (`qmask`: bit s set = the 32 rows x 64 columns at TMEM columns [64 s, 64 s + 64)
+// of the warp's lanes are still to be stored).
 struct QuarterCursor {
   int tile, mat;
   unsigned qmask;
-  int ib;
-  int jb0, jb1;   // column blocks of the two accumulator halves
+  int ib;         // row block of the output
+  int row0;       // first of this warp's 32 output rows
+  int cb0, cb1;   // column block of quarters {0, 1} and of quarters {2, 3}
+  int cofs;       // column offset inside the block on top of 64 (s & 1)
   int row_limit;  // output rows of the matrix in this tile's orientation
 
-  // Quarters of tile `t` for CTA `rank`; returns false past the last tile.
-  __device__ __forceinline__ bool open_tile(const GemmParams& P, int t, int total_tiles, int rank) {
+  // Quarters of tile `t` for warp `q` of CTA `rank`; returns false past the last tile.
+  __device__ __forceinline__ bool open_tile(const GemmParams& P, int t, int total_tiles, int rank, int q) {
     tile = t;
     if (t >= total_tiles) {
       qmask = 0;
@@ -198,20 +206,44 @@ struct QuarterCursor {
     int base_mat;
     bool swapped;
     locate_tile(P, t, pt, base_mat, swapped);
-    mat = base_mat + of_rank(pt.dm, rank);
     row_limit = swapped ? P.n_long : P.m;
     const int col_limit = swapped ? P.m : P.out_cols;
-    ib = of_rank(pt.i, rank);
-    jb0 = pt.j[0];
-    jb1 = pt.j[1];
+    unsigned keep, slots;
+    if (pt.half) {
+      // half height: lanes 0-63 of the CTA (warps 0, 1) hold its 64 rows against the first half of the
+      // N columns, lanes 64-127 (warps 2, 3) against the second half, both in TMEM columns [0, N/2)
+      const int ch = q >> 1;
+      mat = base_mat + pt.dm[0];
+      ib = pt.i[0];
+      row0 = ib * 128 + rank * 64 + (q & 1) * 32;
+      if (pt.nbw == 2) {
+        cb0 = cb1 = ch ? pt.j[1] : pt.j[0];
+        cofs = 0;
+        slots = 3u;
+        keep = ((static_cast<unsigned>(pt.keep[0]) >> ch) & 1u) ? 3u : 0u;
+      } else {
+        cb0 = cb1 = pt.j[0];
+        cofs = ch * 64;
+        slots = 1u;
+        keep = (pt.keep[0] & 1u) ? 1u : 0u;
+      }
+    } else {
+      mat = base_mat + of_rank(pt.dm, rank);
+      ib = of_rank(pt.i, rank);
+      row0 = ib * 128 + q * 32;
+      cb0 = pt.j[0];
+      cb1 = pt.j[1];
+      cofs = 0;
+      slots = pt.nbw == 2 ? 15u : 3u;
+      const unsigned k2 = static_cast<unsigned>(of_rank(pt.keep, rank));
+      keep = ((k2 & 1u) ? 3u : 0u) | ((k2 & 2u) ? 12u : 0u);
+    }
     qmask = 0;
     if (ib * 128 < row_limit) {  // else a ragged pair: nothing of ours
-      const unsigned keep = static_cast<unsigned>(of_rank(pt.keep, rank));
 #pragma unroll
-      for (int qd = 0; qd < 4; ++qd) {
-        const int h = qd >> 1;
-        const bool on = qd < 2 * pt.nbw && ((keep >> h) & 1u) && (h ? jb1 : jb0) * 128 + (qd & 1) * 64 < col_limit;
-        qmask |= on ? (1u << qd) : 0u;
+      for (int sl = 0; sl < 4; ++sl) {
+        const bool on = ((slots & keep) >> sl & 1u) && col0(sl) < col_limit;
+        qmask |= on ? (1u << sl) : 0u;
       }
     }
     return true;
@@ -219,9 +251,10 @@ struct QuarterCursor {
   __device__ __forceinline__ bool has_quarter() const { return qmask != 0; }
   __device__ __forceinline__ int quarter() const { return __ffs(qmask) - 1; }
   __device__ __forceinline__ void pop_quarter() { qmask &= qmask - 1; }
-  // first output column of quarter qd
-  __device__ __forceinline__ int col_block(int qd) const { return (qd >> 1) ? jb1 : jb0; }
-  __device__ __forceinline__ int col0(int qd) const { return col_block(qd) * 128 + (qd & 1) * 64; }
+  __device__ __forceinline__ int col_block(int sl) const { return (sl >> 1) ? cb1 : cb0; }
+  // offset of quarter sl's first column inside its column block, and that column itself
+  __device__ __forceinline__ int col_in_block(int sl) const { return (sl & 1) * 64 + cofs; }
+  __device__ __forceinline__ int col0(int sl) const { return col_block(sl) * 128 + col_in_block(sl); }
 };
 
 // kAccCols: fp32 TMEM columns per accumulator stage = widest N (128 or 256).
@@ -293,10 +326,11 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
         const PairTile pt = tp.pt;
         const int r = static_cast<int>(rank);
         const int mat = tp.base_mat + of_rank(pt.dm, r);  // this CTA's matrix (its own A rows and B rows)
-        const int row0 = of_rank(pt.i, r) * 128;
+        const bool hh = pt.half != 0;  // half height: this CTA stages 64 A rows of row block i[0]
+        const int row0 = hh ? pt.i[0] * 128 + r * 64 : of_rank(pt.i, r) * 128;
         const int half = 64 * pt.nbw;  // B rows (N columns) staged by each CTA
         const int b0 = pt.nbw == 2 ? of_rank(pt.j, r) * 128 : pt.j[0] * 128 + r * 64;
-        const uint32_t stage_tx = 2u * static_cast<uint32_t>(kTileABytes + half * 128);
+        const uint32_t stage_tx = 2u * static_cast<uint32_t>((hh ? kTileABytes / 2 : kTileABytes) + half * 128);
         const int kb_a = tp.kb_a, kb_b = tp.kb_b;
         // a transposed-formulation tile takes its operands from the other two 64 x 64 maps
         const CUtensorMap* map_a64 = tp.swapped ? &P.map_b : &P.map_a64;
@@ -315,10 +349,12 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
             const int k0 = kb * kBK;
             if (rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, stage_tx);
             if (kb >= kb_a) {
-              ptx::tma_load_3d_pair(sa, &P.map_a, k0, row0, mat, leader_full);
+              // K-major; the 64 x 64 box gives the first 64 rows of the 128-row tile's layout
+              if (hh) ptx::tma_load_3d_pair(sa, map_a64, k0, row0, mat, leader_full);
+              else ptx::tma_load_3d_pair(sa, &P.map_a, k0, row0, mat, leader_full);
             } else {
               ptx::tma_load_3d_pair(sa, map_a64, row0, k0, mat, leader_full);
-              ptx::tma_load_3d_pair(sa + 8192, map_a64, row0 + 64, k0, mat, leader_full);
+              if (!hh) ptx::tma_load_3d_pair(sa + 8192, map_a64, row0 + 64, k0, mat, leader_full);
             }
             if (kb >= kb_b) {
               ptx::tma_load_3d_pair(sb, map_b, k0, b0, mat, leader_full);
@@ -380,7 +416,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           const int seg_end = seg == 0 ? cut1 : (seg == 1 ? cut2 : num_kb);
           if (kb >= seg_end) continue;
           const bool a_mn = kb < kb_a, b_mn = kb < kb_b;
-          const uint32_t idesc = ptx::make_idesc_bf16(256, 128 * pt.nbw, a_mn ? 1 : 0, b_mn ? 1 : 0);
+          const uint32_t idesc = ptx::make_idesc_bf16(pt.half ? 128 : 256, 128 * pt.nbw, a_mn ? 1 : 0, b_mn ? 1 : 0);
           const uint32_t a_fix = a_mn ? kLboMN : kLboK, b_fix = (b_mn ? kLboMN : kLboK) + (kTileABytes >> 4);
           const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
 #pragma unroll 1
@@ -436,7 +472,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
     int loads_in_flight = 0;
     auto pre_seek = [&]() {  // moves `pre` to a quarter, opening tiles as needed
       while (pre_valid && !pre.has_quarter()) {
-        pre_valid = pre.open_tile(P, pre.tile + num_clusters, total_tiles, static_cast<int>(rank));
+        pre_valid = pre.open_tile(P, pre.tile + num_clusters, total_tiles, static_cast<int>(rank), q);
       }
     };
     // Arms ring entry pre_g % ring_len for quarter pre_g: starts the TMA loads of
@@ -446,7 +482,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       const uint32_t e = pre_g % ring_len;
       const uint32_t bar = ptx::smem_u32(&my_bars[e]);
       const uint32_t buf = my_base + e * kEntryBytes;
-      const int row0 = pre.ib * 128 + q * 32;
+      const int row0 = pre.row0;
       const int col0 = pre.col0(pre.quarter());
       if (row0 >= pre.row_limit) {  // this warp's rows lie beyond the matrix: nothing to fetch
         ptx::mbar_arrive(bar);
@@ -468,7 +504,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       pre_seek();
     };
     if (lane == 0) {
-      pre_valid = pre.open_tile(P, cluster, total_tiles, static_cast<int>(rank));
+      pre_valid = pre.open_tile(P, cluster, total_tiles, static_cast<int>(rank), q);
       pre_seek();
       for (uint32_t i = 0; i + 1 < ring_len; ++i) arm_next();
     }
@@ -476,7 +512,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
     QuarterCursor cur;
     bool ok = true;
     for (int tile = cluster; tile < total_tiles && ok; tile += num_clusters) {
-      cur.open_tile(P, tile, total_tiles, static_cast<int>(rank));
+      cur.open_tile(P, tile, total_tiles, static_cast<int>(rank), q);
       const int mat = cur.mat;
       ok = ptx::mbar_wait_relaxed(ptx::smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag);
       ok = __all_sync(0xFFFFFFFFu, ok);  // the warp goes on or gives up as one
@@ -489,7 +525,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
       if (cur.has_quarter()) {
         const MatScal sc = P.scal[mat];
         const float scale = P.scale_kind == 1 ? sc.inv_norm_sq : (P.scale_kind == 2 ? sc.inv_norm : 1.0f);
-        const int row0 = cur.ib * 128 + q * 32;  // first of this warp's rows
+        const int row0 = cur.row0;  // first of this warp's rows
         const uint32_t taddr = tmem_base + static_cast<uint32_t>(acc * kAccCols) +
                                (static_cast<uint32_t>(q * 32) << 16);
 
@@ -500,7 +536,7 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
           const int col0 = cur.col0(qd);
           // column of this lane's row that lies on the matrix diagonal, if the quarter holds it
           const bool diag_quarter = P.diag_add != 0.f && cur.col_block(qd) == cur.ib;
-          const int dcol = q * 32 + lane - (qd & 1) * 64;
+          const int dcol = row0 - cur.ib * 128 + lane - cur.col_in_block(qd);
 
           uint32_t v[64];
           ptx::tmem_ld_32x64(taddr + qd * 64, v);

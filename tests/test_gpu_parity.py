@@ -631,6 +631,42 @@ def test_paired_and_plain_sequences_agree_within_tolerance(pair_fold_knob):
     assert 0 < rel(outs[1], outs[0]) <= 2 * TOL_NS
 
 
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+def test_every_tile_mode_matches_the_oracle(mode):
+    """Half-height tiles, tiles shared by two matrices, and full tiles whose
+    second CTA works beyond the matrix are different ways of cutting the same
+    products (muon_debug_set_tile_mode; 1 is the default every other test runs).
+    Each must meet the oracle on its own: odd and even numbers of row blocks,
+    both orientations, an odd number of matrices (one is left without a partner
+    in the modes that pair matrices), bf16 and fp32 weights, two steps, with the
+    tap on O and with the update fused into the last epilogue."""
+    b = _binding()
+    specs = [wl.GroupSpec(328, 704, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3, lognormal_scale=True),
+             wl.GroupSpec(704, 328, 1, torch.bfloat16, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(256, 640, 3, torch.float32, torch.bfloat16, 0.02, 1e-3),
+             wl.GroupSpec(100, 72, 2, torch.bfloat16, torch.bfloat16, 0.02, 1e-3)]
+    hp = default_hp(lr=1e-2, wd=0.1)
+    prev = b.muon_debug_set_tile_mode(mode)
+    try:
+        for one in specs:  # the tap needs a context with a single bucket
+            case = Case([one], seed=19)
+            try:
+                check_step(case, hp, check_o=True)
+            finally:
+                case.close()
+        case = Case(specs, seed=19)
+        try:
+            check_step(case, hp)
+            gen = torch.Generator().manual_seed(20)
+            for gi, sp in enumerate(specs):
+                case.dev[gi][1].copy_(wl.make_grads(sp, gen, "cpu"))
+            check_step(case, hp)
+        finally:
+            case.close()
+    finally:
+        b.muon_debug_set_tile_mode(prev)
+
+
 def test_bucket_by_bucket_step_gives_muon_step_bits():
     """muon_step_bucket over every bucket, in reverse order, is one muon_step:
     buckets are independent, and the numbering is muon_plan_buckets' (the two

@@ -9,7 +9,9 @@ instruction reads the operand tiles of both CTAs in one layout, and a symmetric
 operand kept as its upper blocks changes layout at the diagonal, so for such
 operands the two row blocks (and the two column blocks) of a tile must be equal
 or neighbours.  A tile whose CTAs work on different matrices computes two cross
-blocks that mean nothing; they must not be stored.
+blocks that mean nothing; they must not be stored.  A half-height tile is one
+row block, 64 rows per CTA.  The tables exist in four modes
+(muon_debug_set_tile_mode); all are checked.
 """
 
 import pytest
@@ -24,8 +26,34 @@ def blocks(v):
     return -(-v // 128)
 
 
+@pytest.fixture(params=[0, 1, 2, 3])
+def tile_mode(request):
+    prev = b.muon_debug_set_tile_mode(request.param)
+    yield request.param
+    b.muon_debug_set_tile_mode(prev)
+
+
+def stored_blocks(t):
+    """(matrix, row block, column block) of every block a tile stores."""
+    out = []
+    if t["half"]:
+        assert t["i"][0] == t["i"][1] and t["dm"][0] == t["dm"][1] and t["keep"][1] == 0
+        for h in range(t["nbw"]):
+            if (t["keep"][0] >> h) & 1:
+                out.append((t["dm"][0], t["i"][0], t["j"][h]))
+        return out
+    for rank in (0, 1):
+        for h in range(t["nbw"]):
+            if (t["keep"][rank] >> h) & 1:
+                # with the full width the B rows of half h come from CTA h's matrix
+                if t["nbw"] == 2:
+                    assert t["dm"][h] == t["dm"][rank], t
+                out.append((t["dm"][rank], t["i"][rank], t["j"][h]))
+    return out
+
+
 @pytest.mark.parametrize("rows,cols", SHAPES)
-def test_symmetric_product_tables_cover_the_upper_triangle_once(rows, cols):
+def test_symmetric_product_tables_cover_the_upper_triangle_once(rows, cols, tile_mode):
     m = min(rows, cols)
     nb = blocks(m)
     for which in (0, 1):
@@ -37,40 +65,30 @@ def test_symmetric_product_tables_cover_the_upper_triangle_once(rows, cols):
                 continue
             unit_here = 1
         else:
-            assert unit in (1, 2) and tiles
+            assert unit == (1 if tile_mode & 2 else 2) and tiles
             unit_here = unit
         seen = {}
         for t in tiles:
             assert t["nbw"] in (1, 2)
+            assert bool(t["half"]) <= bool(tile_mode & 2)
             # layout rule for symmetric operands: neighbours or equal, on both sides
             assert abs(t["i"][0] - t["i"][1]) <= 1
             if t["nbw"] == 2:
                 assert abs(t["j"][0] - t["j"][1]) <= 1
-            for rank in (0, 1):
-                assert 0 <= t["dm"][rank] < unit_here
-                i = t["i"][rank]
-                for h in range(t["nbw"]):
-                    if not (t["keep"][rank] >> h) & 1:
-                        continue
-                    j = t["j"][h]
-                    # a stored block is computed from this CTA's matrix on both sides: with the full
-                    # width the B rows of half h come from CTA h's matrix
-                    if t["nbw"] == 2:
-                        assert t["dm"][h] == t["dm"][rank], t
-                    if i >= nb:
-                        continue  # rows beyond the matrix: the kernel stores nothing for them
-                    assert j < nb and i <= j, t  # on or above the diagonal, inside the matrix
-                    key = (t["dm"][rank], i, j)
-                    seen[key] = seen.get(key, 0) + 1
-                if t["keep"][rank] >> t["nbw"]:
-                    raise AssertionError("keep bit beyond the tile's width: %r" % (t,))
+            assert all(k >> t["nbw"] == 0 for k in t["keep"]), t
+            for (d, i, j) in stored_blocks(t):
+                assert 0 <= d < unit_here
+                if i >= nb:
+                    continue  # rows beyond the matrix: the kernel stores nothing for them
+                assert j < nb and i <= j, t  # on or above the diagonal, inside the matrix
+                seen[(d, i, j)] = seen.get((d, i, j), 0) + 1
         want = {(d, i, j) for d in range(unit_here) for i in range(nb) for j in range(i, nb)}
         assert set(seen) == want
         assert all(c == 1 for c in seen.values())
 
 
 @pytest.mark.parametrize("rows,cols", SHAPES)
-def test_combine_tables_cover_the_output_once(rows, cols):
+def test_combine_tables_cover_the_output_once(rows, cols, tile_mode):
     m, n = min(rows, cols), max(rows, cols)
     for which, out_rows, out_cols in ((2, m, n), (3, n, m)):
         tiles, unit = b.muon_debug_tile_table(rows, cols, which)
@@ -79,15 +97,16 @@ def test_combine_tables_cover_the_output_once(rows, cols):
         seen = {}
         for t in tiles:
             assert t["dm"] == (0, 0)
-            assert t["i"][1] == t["i"][0] + 1  # the symmetric operand's rows (or X^T's): neighbours
-            for rank in (0, 1):
-                i = t["i"][rank]
-                for h in range(t["nbw"]):
-                    assert (t["keep"][rank] >> h) & 1
-                    j = t["j"][h]
-                    assert j < cb
-                    if i < rb:
-                        seen[(i, j)] = seen.get((i, j), 0) + 1
+            if t["half"]:
+                assert tile_mode & 1 and t["i"][0] == rb - 1 and rb % 2 == 1  # only the row block without a partner
+            else:
+                assert t["i"][1] == t["i"][0] + 1  # the symmetric operand's rows (or X^T's): neighbours
+                assert not (tile_mode & 1 and t["i"][1] >= rb)
+            assert len(stored_blocks(t)) == (1 if t["half"] else 2) * t["nbw"]
+            for (d, i, j) in stored_blocks(t):
+                assert j < cb
+                if i < rb:
+                    seen[(i, j)] = seen.get((i, j), 0) + 1
         assert set(seen) == {(i, j) for i in range(rb) for j in range(cb)}
         assert all(c == 1 for c in seen.values())
     assert len(b.muon_debug_tile_table(rows, cols, 2)[0]) == len(b.muon_debug_tile_table(rows, cols, 3)[0])
@@ -105,28 +124,48 @@ def test_executed_work_follows_the_tables():
         for kind in ("gram", "poly", "comb"):
             assert executed[kind] >= planned[kind] > 0
         assert executed["momentum"] == executed["norm"] == executed["update"] == 0
-    # one expert-shaped bucket of 7 matrices, by hand: three units of two matrices and one alone
-    planned, executed = b.muon_plan_work([(1408, 2048, 7)], 1)
-    unit, _ = b.muon_debug_tile_table(1408, 2048, 0)
-    tail, _ = b.muon_debug_tile_table(1408, 2048, 1)
-    comb, _ = b.muon_debug_tile_table(1408, 2048, 2)
-    per = lambda tiles, k: sum(2.0 * 256 * 128 * t["nbw"] * k for t in tiles)
-    assert executed["gram"] == 3 * per(unit, 2048) + per(tail, 2048)
-    assert executed["poly"] == 3 * per(unit, 1408) + per(tail, 1408)
-    assert executed["comb"] == 7 * per(comb, 1408)
-    assert planned["gram"] == 7 * 1408.0 ** 2 * 2048 and planned["comb"] == 2 * planned["gram"]
+    # one expert-shaped bucket of 7 matrices, by hand from the tables
+    prev = b.muon_debug_set_tile_mode(0)
+    try:
+        for mode in (0, 3):
+            b.muon_debug_set_tile_mode(mode)
+            planned, executed = b.muon_plan_work([(1408, 2048, 7)], 1)
+            unit, mats = b.muon_debug_tile_table(1408, 2048, 0)
+            tail, _ = b.muon_debug_tile_table(1408, 2048, 1)
+            comb, _ = b.muon_debug_tile_table(1408, 2048, 2)
+            per = lambda tiles, k: sum(2.0 * (128 if t["half"] else 256) * 128 * t["nbw"] * k for t in tiles)
+            units, left = divmod(7, mats)
+            assert executed["gram"] == units * per(unit, 2048) + left * per(tail, 2048)
+            assert executed["poly"] == units * per(unit, 1408) + left * per(tail, 1408)
+            assert executed["comb"] == 7 * per(comb, 1408)
+            assert planned["gram"] == 7 * 1408.0 ** 2 * 2048 and planned["comb"] == 2 * planned["gram"]
+            if mode == 3:  # nothing computed in vain but the lower halves of the diagonal blocks
+                assert executed["comb"] == planned["comb"]
+                assert abs(executed["gram"] / planned["gram"] - 66 / 60.5) < 1e-12
+    finally:
+        b.muon_debug_set_tile_mode(prev)
 
 
 def test_expert_shape_tables_have_the_expected_sizes():
-    """1408 rows are 11 row blocks: 15 full tiles per matrix plus six diagonal
-    blocks that pair up with the neighbour matrix's (36 tiles per two matrices);
-    a matrix alone takes them as six half-width tiles."""
+    """1408 rows are 11 row blocks: 15 full tiles per matrix and six diagonal
+    blocks.  Default (mode 1): the six pair up with the neighbour matrix's (36
+    tiles per two matrices; a matrix alone takes them as six half-width tiles),
+    and the combine's eleventh row block is eight half-height tiles.  Mode 3:
+    each of the six is a half-height, half-width tile of its own matrix."""
+    assert b.muon_debug_set_tile_mode(-1) == 1  # query only
     unit, mats = b.muon_debug_tile_table(2048, 1408, 0)
-    assert mats == 2 and len(unit) == 36 and all(t["nbw"] == 2 for t in unit)
+    assert mats == 2 and len(unit) == 36 and all(t["nbw"] == 2 and not t["half"] for t in unit)
     shared = [t for t in unit if t["dm"] == (0, 1)]
     assert len(shared) == 6 and all(t["i"][0] == t["i"][1] == t["j"][0] == t["j"][1] for t in shared)
     assert all(t["keep"] == (1, 2) for t in shared)
     tail, _ = b.muon_debug_tile_table(2048, 1408, 1)
     assert len(tail) == 21 and sum(1 for t in tail if t["nbw"] == 1) == 6
-    even, mats = b.muon_debug_tile_table(2048, 2048, 0)
-    assert mats == 1 and len(even) == 36
+    comb, _ = b.muon_debug_tile_table(2048, 1408, 2)
+    assert len(comb) == 48 and sum(1 for t in comb if t["half"]) == 8
+    prev = b.muon_debug_set_tile_mode(3)
+    try:
+        unit, mats = b.muon_debug_tile_table(2048, 1408, 0)
+        assert mats == 1 and len(unit) == 21
+        assert sum(1 for t in unit if t["half"]) == 6 and all(t["nbw"] == 1 for t in unit if t["half"])
+    finally:
+        b.muon_debug_set_tile_mode(prev)
