@@ -307,6 +307,10 @@ ns_gemm_kernel(const __grid_constant__ GemmParams P) {
   ptx::cluster_sync_all();  // both CTAs' barriers are initialised, both TMEM allocations done
   ptx::tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+  // Everything above touched only this CTA's shared memory, TMEM and the kernel's parameters, so
+  // it may overlap the tail of the previous kernel of the stream; its results are needed from here on.
+  ptx::grid_dependency_wait();
+  ptx::grid_launch_dependents();
   if (P.debug != nullptr && threadIdx.x == 0) P.debug[blockIdx.x] = tmem_base;
 
   if (warp == 0) {
@@ -755,13 +759,17 @@ cudaError_t launch_one(const GemmParams& P, unsigned clusters, cudaStream_t stre
   cfg.blockDim = dim3(kGemmThreads, 1, 1);
   cfg.dynamicSmemBytes = smem_bytes(kStages, kSubs, kWFp32 ? kSubBytesFp32 : kSubBytes);
   cfg.stream = stream;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = 2;
-  attr.val.clusterDim.y = 1;
-  attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  // the kernel's set-up (barriers, TMEM allocation) may start while the previous kernel of the
+  // stream drains; the kernel waits for that kernel's results itself (grid_dependency_wait)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, ns_gemm_kernel<kAccCols, kStages, kSubs, kWFp32>, P);
 }
 

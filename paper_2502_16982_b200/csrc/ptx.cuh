@@ -377,6 +377,22 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask
       : "memory");
 }
 
+// ------------------------------------------- programmatic dependent launch --
+// Blocks until every grid this one depends on has completed and its memory is
+// visible (returns at once for a grid launched without programmatic
+// serialisation).  Nothing that reads or writes memory of an earlier kernel may
+// precede it.
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// Lets the next grid of the stream, if it was launched with programmatic
+// serialisation, be scheduled as this grid's CTAs retire instead of after the
+// whole grid has drained; that grid still waits in grid_dependency_wait().
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ------------------------------------------------------------ descriptors --
 // Shared-memory matrix descriptor (64-bit), 128-byte swizzle, descriptor
 // version 1.  Fields: start address >> 4 (bits 0-13), leading byte offset >> 4
