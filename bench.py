@@ -58,7 +58,7 @@ WORKLOAD_NAMES = {
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/, taken on 64 matrices of the expert-bucket shapes; it scales with the matrix count.
-NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": None, "gemm_launches_per_step": 16,
+NCU_CAPTURE = {"matrices": 64, "gemm_bytes_per_step": 7.915e9, "gemm_launches_per_step": 16,
                "momentum_bytes_per_launch": 2.159e9}
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
@@ -406,6 +406,60 @@ def run_distributed(args, rank, world, local_rank):
     dist.destroy_process_group()
 
 
+def run_aux_kernels(args):
+    """Event figures for the element-wise kernels the default workload does not reach: the ld/st
+    momentum kernel (gradients and momenta that TMA cannot address) and the separate weight update
+    (weights that TMA cannot address, or no iteration).  Matrices of the expert shapes, every tensor
+    starting one element into its buffer so that nothing is 16-byte aligned; ns_steps = 0 keeps the
+    step to momentum, norm, update."""
+    from paper_2502_16982_b200 import binding
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    count = args.max_count or 32
+    groups, keep, elems = [], [], 0
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7)
+    for rows, cols in ((2048, 1408), (1408, 2048)):
+        n = rows * cols
+        ws, gs, ms = [], [], []
+        for _ in range(count):
+            wb = (torch.randn(n + 8, generator=gen, device=dev) * 0.02).to(torch.bfloat16)
+            gb = (torch.randn(n + 8, generator=gen, device=dev) * 1e-3).to(torch.bfloat16)
+            mb = torch.zeros(n + 8, dtype=torch.float32, device=dev)
+            keep += [wb, gb, mb]
+            ws.append(wb[1:1 + n].view(rows, cols))
+            gs.append(gb[1:1 + n].view(rows, cols))
+            ms.append(mb[1:1 + n].view(rows, cols))
+            elems += n
+        groups.append((ws, gs, ms))
+    ctx = binding.MuonContext(groups)
+    hpd = hp_dict_default()
+    hpd["ns_steps"] = 0
+    hp = binding.Hyper(**hpd)
+    for _ in range(3):
+        ctx.muon_step(hp)
+    ctx.muon_profile_enable(True)
+    steps = max(3, args.steps)
+    for _ in range(steps):
+        ctx.muon_step(hp)
+    prof = ctx.muon_profile_read()
+    ctx.muon_profile_enable(False)
+    status, which = ctx.muon_status()
+    if status != 0:
+        raise SystemExit("device status %d at matrix %d" % (status, which))
+    out = {"aux_kernels": True, "matrices": 2 * count, "elements": elems, "steps": steps,
+           "peak_hbm_gbs": float(peaks["hbm_gbs"]), "peak_source": peaks["_source"]}
+    for kind, name, bpe in (("momentum", "momentum_cast_kernel", 12.0), ("update", "update_from_x_kernel", 6.0)):
+        ms, n = prof[kind]
+        gbs = bpe * elems * steps / (ms * 1e-3) / 1e9
+        out[name] = {"ms_per_launch": ms / max(1, n), "launches": n, "bytes_per_element": bpe, "achieved_gbs": gbs,
+                     "frac": gbs / float(peaks["hbm_gbs"])}
+    print(json.dumps(out))
+    ctx.muon_destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -423,6 +477,8 @@ def main():
     ap.add_argument("--no-adamw", action="store_true", help="skip the AdamW (non-Muon parameters) leg")
     ap.add_argument("--reduce-grads", action="store_true",
                     help="N > 1: sum the gradients over the ranks (reduce-scatter) inside the timed region")
+    ap.add_argument("--aux-kernels", action="store_true",
+                    help="time the element-wise kernels of the unaligned path instead (one JSON line of their own)")
     ap.add_argument("--distributed", action="store_true",
                     help="take the partitioned (N > 1) path even with one rank")
     ap.add_argument("--max-count", type=int, default=None,
@@ -443,6 +499,10 @@ def main():
         args.warmup = 3
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the Muon step has no CPU path")
+    if args.aux_kernels:
+        if rank == 0:
+            run_aux_kernels(args)
+        return
     if world > 1 or args.distributed:
         run_distributed(args, rank, world, local_rank)
         return

@@ -378,9 +378,12 @@ size_t muon_debug_set_chunk_bytes(size_t bytes);
  * instead of a full tile whose second CTA works on rows beyond the matrix.
  * Bit 1: the diagonal blocks of a symmetric product that no full tile can hold
  * without waste are half-height, half-width tiles, instead of sharing a
- * full-width tile with the neighbour matrix's (cross blocks dropped).  Default
- * 1 (bit 1 computes nothing in vain but measured slower).  Process-wide, read where muon_debug_set_pair_fold is.  Returns the
- * previous mode; a value outside 0..3 only queries.  The modes agree to
+ * full-width tile with the neighbour matrix's (cross blocks dropped).  Bit 2
+ * switches off the finer cut (every row block on its own at half height, or
+ * block by block) that the symmetric products of a bucket take when full tiles
+ * would be fewer than the CTA pairs of the GPU.  Default 1 (bit 1 computes
+ * nothing in vain but measured slower).  Process-wide, read where muon_debug_set_pair_fold is.  Returns the
+ * previous mode; a value outside 0..7 only queries.  The modes agree to
  * rounding, not bit for bit (instructions of different heights round their
  * sums differently); within one mode results are reproducible bit for bit.
  */
@@ -405,7 +408,8 @@ int muon_debug_set_pair_fold(int mode);
 
 /*
  * Test tap (pure host computation): the tile table the Newton-Schulz products
- * of a rows x cols matrix use.  which = 0: products with a symmetric result,
+ * of a bucket of `count` rows x cols matrices use (the count matters because a
+ * bucket whose launches would leave SMs idle is cut into finer tiles).  which = 0: products with a symmetric result,
  * table of one unit of *unit_mats matrices; 1: the same for a last matrix
  * without a partner (empty when units are single matrices); 2: the combine;
  * 3: the combine formed transposed.  Every tile is ten int16 in `out` (room
@@ -415,7 +419,8 @@ int muon_debug_set_pair_fold(int mode);
  * per CTA a mask of the column halves whose 128 x 128 block is stored, and 1 for
  * a half-height tile (one row block, 64 rows per CTA; its mask is the first).
  */
-int muon_debug_tile_table(int rows, int cols, int which, int16_t* out, int cap_tiles, int* n_tiles, int* unit_mats);
+int muon_debug_tile_table(int rows, int cols, int count, int which, int16_t* out, int cap_tiles, int* n_tiles,
+                          int* unit_mats);
 
 /*
  * Test tap: the TMEM base address each CTA of the last Newton-Schulz GEMM launch

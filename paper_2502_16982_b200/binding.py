@@ -103,7 +103,7 @@ def lib():
                                   C.POINTER(C.c_double)]
     L.muon_plan_work.argtypes = [C.POINTER(muon_group), C.c_int, C.c_int, C.POINTER(C.c_double),
                                  C.POINTER(C.c_double)]
-    L.muon_debug_tile_table.argtypes = [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int16), C.c_int,
+    L.muon_debug_tile_table.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int16), C.c_int,
                                         C.POINTER(C.c_int), C.POINTER(C.c_int)]
     L.muon_step_bucket.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.c_int, C.c_void_p]
     L.muon_step_host.argtypes = [C.c_void_p, C.POINTER(muon_hparams), C.POINTER(C.POINTER(C.c_void_p)),
@@ -326,14 +326,15 @@ def muon_plan_work(shapes, ns_steps: int = 5):
             {k: executed[i] for i, k in enumerate(KERNEL_KINDS)})
 
 
-def muon_debug_tile_table(rows: int, cols: int, which: int):
-    """(tiles, matrices per unit): every tile is a dict with the row blocks
+def muon_debug_tile_table(rows: int, cols: int, which: int, count: int = 4096):
+    """(tiles, matrices per unit) of a bucket of ``count`` matrices (few small
+    matrices are cut into finer tiles): every tile is a dict with the row blocks
     ``i`` and matrices ``dm`` of the two CTAs, the column blocks ``j`` of the
     two accumulator halves, the width ``nbw`` and the ``keep`` masks."""
     n, unit = C.c_int(0), C.c_int(0)
-    _check(lib().muon_debug_tile_table(rows, cols, which, None, 0, C.byref(n), C.byref(unit)))
+    _check(lib().muon_debug_tile_table(rows, cols, count, which, None, 0, C.byref(n), C.byref(unit)))
     buf = (C.c_int16 * (10 * max(1, n.value)))()
-    _check(lib().muon_debug_tile_table(rows, cols, which, buf, n.value, C.byref(n), C.byref(unit)))
+    _check(lib().muon_debug_tile_table(rows, cols, count, which, buf, n.value, C.byref(n), C.byref(unit)))
     tiles = []
     for k in range(n.value):
         v = buf[10 * k:10 * k + 10]

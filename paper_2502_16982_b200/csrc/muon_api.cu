@@ -293,11 +293,13 @@ PairTile make_half_tile(int i, int j0, int j1, int nbw, int dm, unsigned keep) {
 }
 
 // How tiles are cut where the row blocks do not pair up; see muon_debug_set_tile_mode.
-// bit 0: a row block without a partner is taken at half height; bit 1: so is a lone diagonal block.
+// bit 0: a row block without a partner is taken at half height; bit 1: so is a lone diagonal block;
+// bit 2: launches with few tiles are NOT cut finer.
 // Measured on the expert bucket (1408 rows = 11 row blocks): mode 1 13.49 ms per step, mode 0 13.67,
 // mode 3 13.67, mode 2 13.83: the half-height, half-width tiles of bit 1 run too far below the
 // tensor cores' rate to pay, although they compute nothing in vain.
 int g_tile_mode = 1;
+constexpr int kNominalPairs = 74;  // CTA pairs of a B200 (148 SMs); a planning constant, not a device query
 
 // Tiles of the symmetric products (only the 128-blocks on or above the diagonal
 // are produced) for matrix `dm` of a unit, nb row blocks.  A full tile is two
@@ -307,8 +309,17 @@ int g_tile_mode = 1;
 // leaves the diagonal blocks (r, r), r even, which no full tile can hold without
 // waste (the block below it in the pair lies under the diagonal): with
 // `half_lone` each becomes a half-height, half-width tile, otherwise `lone`
-// receives them.
+// receives them (an odd number of row blocks; an even number needs none, see below).
 void sym_tiles_of_matrix(int nb, int dm, bool half_lone, std::vector<PairTile>* tiles, std::vector<int>* lone) {
+  if (nb % 2 == 0 && !half_lone) {
+    // an even number of row blocks: row pair (r, r+1) takes columns r, r+1, then r+2, r+3, ...: every
+    // tile is full width; the first holds the block (r+1, r) under the diagonal, computed and dropped
+    // (nb/2 blocks in nb(nb+1)/2 + nb/2), which is cheaper than half-width tiles at the end of every row pair
+    for (int r = 0; r < nb; r += 2)
+      for (int c = r; c < nb; c += 2)
+        tiles->push_back(make_tile(r, r + 1, c, c + 1, 2, dm, dm, 3u, c == r ? 2u : 3u));
+    return;
+  }
   for (int r = 0; r < nb; r += 2) {
     if (half_lone) tiles->push_back(make_half_tile(r, r, r, 1, dm, 1u));
     else lone->push_back(r);
@@ -331,9 +342,9 @@ void build_tile_tables(Bucket* Bp) {
   B.comb_tiles_t.clear();
   B.sym_acc_cols = B.comb_acc_cols = 128;
   std::vector<int> lone;
-  if (half_lone) {
+  if (half_lone || nb % 2 == 0) {
     B.sym_unit_mats = 1;
-    sym_tiles_of_matrix(nb, 0, true, &B.sym_tiles, &lone);
+    sym_tiles_of_matrix(nb, 0, half_lone, &B.sym_tiles, &lone);
   } else {
     // Without half-height tiles the lone diagonal blocks (r, r) of two matrices share a
     // full-width tile, one CTA per matrix, whose two cross blocks are dropped; a matrix
@@ -346,6 +357,33 @@ void build_tile_tables(Bucket* Bp) {
     lone.clear();
     sym_tiles_of_matrix(nb, 0, false, &B.sym_tiles_tail, &lone);
     for (int r : lone) B.sym_tiles_tail.push_back(make_tile(r, r + 1, r, r, 1, 0, 0, 1u, 0u));
+  }
+  // A launch with fewer tiles than CTA pairs leaves SMs idle: a bucket of few small matrices is then
+  // cut finer, every row block on its own at half height (twice the tiles at about 0.6 of a full tile's
+  // time each), or block by block (four times the tiles at about 0.45).  The estimate is rounds of
+  // kNominalPairs concurrent tiles times the tile's relative time; full tiles win whenever the SMs are busy.
+  {
+    const int count = std::max(1, std::min<int>(B.chunk > 0 ? B.chunk : 1, static_cast<int>(B.mats.size())));
+    const long long t_full = static_cast<long long>(count / B.sym_unit_mats) * static_cast<long long>(B.sym_tiles.size()) +
+                             (count % B.sym_unit_mats) * static_cast<long long>(B.sym_tiles_tail.size());
+    long long t_rows = 0;
+    for (int i = 0; i < nb; ++i) t_rows += ceil_div(nb - i, 2);
+    t_rows *= count;
+    const long long t_blocks = static_cast<long long>(count) * nb * (nb + 1) / 2;
+    auto rounds = [](long long t) { return static_cast<double>((t + kNominalPairs - 1) / kNominalPairs); };
+    const double c_full = rounds(t_full) * 1.0, c_rows = rounds(t_rows) * 0.6, c_blocks = rounds(t_blocks) * 0.45;
+    if ((g_tile_mode & 4) == 0 && t_full < kNominalPairs && (c_rows < c_full || c_blocks < c_full)) {
+      const bool by_block = c_blocks < c_rows;
+      B.sym_tiles.clear();
+      B.sym_tiles_tail.clear();
+      B.sym_unit_mats = 1;
+      for (int i = 0; i < nb; ++i)
+        for (int c = i; c < nb;) {
+          const int w = by_block ? 1 : std::min(2, nb - c);
+          B.sym_tiles.push_back(make_half_tile(i, c, c + 1, w, 0, w == 2 ? 3u : 1u));
+          c += w;
+        }
+    }
   }
   for (const PairTile& t : B.sym_tiles)
     if (t.nbw == 2) B.sym_acc_cols = 256;
@@ -660,7 +698,7 @@ int muon_workspace_bytes(const muon_group* groups, int n_groups, size_t* out_byt
 
 int muon_debug_set_tile_mode(int mode) {
   const int prev = g_tile_mode;
-  if (mode >= 0 && mode <= 3) g_tile_mode = mode;
+  if (mode >= 0 && mode <= 7) g_tile_mode = mode;
   return prev;
 }
 
@@ -749,12 +787,16 @@ int muon_plan_work(const muon_group* groups, int n_groups, int ns_steps, double*
   return MUON_OK;
 }
 
-int muon_debug_tile_table(int rows, int cols, int which, int16_t* out, int cap_tiles, int* n_tiles, int* unit_mats) {
-  if (!n_tiles || !unit_mats || rows <= 0 || cols <= 0 || rows > 65536 || cols > 65536 || which < 0 || which > 3)
+int muon_debug_tile_table(int rows, int cols, int count, int which, int16_t* out, int cap_tiles, int* n_tiles,
+                          int* unit_mats) {
+  if (!n_tiles || !unit_mats || rows <= 0 || cols <= 0 || rows > 65536 || cols > 65536 || which < 0 || which > 3 ||
+      count <= 0)
     return fail(MUON_ERR_INVALID_ARG, "bad arguments");
   Bucket B{};
   B.m = std::min(rows, cols);
   B.n = std::max(rows, cols);
+  B.mats.resize(count);
+  B.chunk = std::min(count, kChunkCountMax);
   build_tile_tables(&B);
   const std::vector<PairTile>& t = which == 0 ? B.sym_tiles : (which == 1 ? B.sym_tiles_tail : (which == 2 ? B.comb_tiles : B.comb_tiles_t));
   *n_tiles = static_cast<int>(t.size());

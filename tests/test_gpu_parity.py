@@ -217,9 +217,18 @@ RAGGED = [(1, 300), (300, 1), (129, 257), (257, 129), (8, 8), (130, 130), (64, 1
 
 @pytest.mark.parametrize("rows,cols", RAGGED)
 @pytest.mark.parametrize("wdt", [torch.float32, torch.bfloat16])
-def test_ragged_shapes(rows, cols, wdt):
-    sp = wl.GroupSpec(rows, cols, 3, wdt, wdt, 0.02, 1.0)
-    case = Case([sp], seed=rows * 7 + cols)
+@pytest.mark.parametrize("tile_mode", [1, 5])
+def test_ragged_shapes(rows, cols, wdt, tile_mode):
+    """Three matrices of an awkward shape.  So small a bucket is cut into finer
+    tiles by default (tile mode 1: every row block on its own); mode 5 switches
+    that off, so that the tiles a large bucket takes - row pairs, tiles shared
+    by two matrices, a dropped block - meet the same ragged edges."""
+    prev = _binding().muon_debug_set_tile_mode(tile_mode)
+    try:
+        sp = wl.GroupSpec(rows, cols, 3, wdt, wdt, 0.02, 1.0)
+        case = Case([sp], seed=rows * 7 + cols)
+    finally:
+        _binding().muon_debug_set_tile_mode(prev)
     try:
         check_step(case, default_hp(lr=4.2e-4, wd=0.05), check_o=True)
         check_step(case, default_hp(lr=4.2e-4, wd=0.05))
@@ -631,11 +640,13 @@ def test_paired_and_plain_sequences_agree_within_tolerance(pair_fold_knob):
     assert 0 < rel(outs[1], outs[0]) <= 2 * TOL_NS
 
 
-@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+@pytest.mark.parametrize("mode", [4, 5, 6, 7, 1, 3])
 def test_every_tile_mode_matches_the_oracle(mode):
     """Half-height tiles, tiles shared by two matrices, and full tiles whose
     second CTA works beyond the matrix are different ways of cutting the same
-    products (muon_debug_set_tile_mode; 1 is the default every other test runs).
+    products (muon_debug_set_tile_mode; 1 is the default).  Modes 4 to 7 are 0 to
+    3 with the finer cut of small buckets switched off, so that these few small
+    matrices take the tiles of a large bucket; modes 1 and 3 cut them finer.
     Each must meet the oracle on its own: odd and even numbers of row blocks,
     both orientations, an odd number of matrices (one is left without a partner
     in the modes that pair matrices), bf16 and fp32 weights, two steps, with the

@@ -65,7 +65,8 @@ def test_symmetric_product_tables_cover_the_upper_triangle_once(rows, cols, tile
                 continue
             unit_here = 1
         else:
-            assert unit == (1 if tile_mode & 2 else 2) and tiles
+            # matrices pair up only to share their lone diagonal blocks: an odd number of row blocks
+            assert unit == (2 if nb % 2 == 1 and not tile_mode & 2 else 1) and tiles
             unit_here = unit
         seen = {}
         for t in tiles:
@@ -167,5 +168,38 @@ def test_expert_shape_tables_have_the_expected_sizes():
         unit, mats = b.muon_debug_tile_table(2048, 1408, 0)
         assert mats == 1 and len(unit) == 21
         assert sum(1 for t in unit if t["half"]) == 6 and all(t["nbw"] == 1 for t in unit if t["half"])
+    finally:
+        b.muon_debug_set_tile_mode(prev)
+
+
+def test_an_even_number_of_row_blocks_needs_no_lone_tiles():
+    """2048 rows = 16 row blocks: 36 full tiles, eight of which hold a block
+    under the diagonal that is dropped; single-matrix units."""
+    tiles, mats = b.muon_debug_tile_table(2048, 2048, 0)
+    assert mats == 1 and len(tiles) == 36 and all(t["nbw"] == 2 and not t["half"] for t in tiles)
+    assert sum(1 for t in tiles if t["keep"] == (3, 2)) == 8
+
+
+@pytest.mark.parametrize("rows,cols,count,expect_tiles,width", [(1024, 1024, 1, 36, 1), (2048, 2048, 1, 72, 2),
+                                                                 (512, 512, 1, 10, 1), (1408, 2048, 1, 66, 1)])
+def test_few_small_matrices_are_cut_into_finer_tiles(rows, cols, count, expect_tiles, width):
+    """A launch with fewer full tiles than the GPU has CTA pairs would leave SMs
+    idle: the symmetric products of such a bucket take every row block on its
+    own at half height, or block by block; coverage stays exact, and the same
+    shapes in a large bucket keep full tiles."""
+    nb = blocks(min(rows, cols))
+    tiles, mats = b.muon_debug_tile_table(rows, cols, 0, count)
+    assert mats == 1 and len(tiles) == expect_tiles and all(t["half"] for t in tiles)
+    assert max(t["nbw"] for t in tiles) == width
+    seen = sorted((i, j) for t in tiles for (_, i, j) in stored_blocks(t))
+    assert seen == [(i, j) for i in range(nb) for j in range(i, nb)]
+    for t in tiles:
+        assert t["nbw"] == 1 or t["j"][1] == t["j"][0] + 1
+    big, _ = b.muon_debug_tile_table(rows, cols, 0, 512)
+    assert not any(t["half"] for t in big)
+    prev = b.muon_debug_set_tile_mode(1 | 4)  # the finer cut switched off
+    try:
+        coarse, _ = b.muon_debug_tile_table(rows, cols, 1 if nb % 2 else 0, count)
+        assert not any(t["half"] for t in coarse)
     finally:
         b.muon_debug_set_tile_mode(prev)
