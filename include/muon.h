@@ -116,6 +116,12 @@ typedef struct muon_group {
  *   coeffs    : NULL, or a HOST array of 3 * ns_steps floats (a_1, b_1, c_1, a_2, ...)
  *               giving every iteration its own quintic; then a, b, c are ignored.
  *               (The paper uses one triple for all iterations.)
+ *   protect_momentum: non-zero adds a pass over the gradients before the
+ *               momentum update (2 or 4 more bytes read per element) that finds
+ *               the matrices holding an Inf or a NaN; such a matrix keeps its M
+ *               as well as its W, so that training can go on after a bad batch
+ *               without repairing anything (the paper is silent on non-finite
+ *               gradients).  0 (default): no such pass, see muon_status.
  */
 enum { MUON_SCALE_ADJUSTED_LR = 0, MUON_SCALE_FIXED_DIM = 1, MUON_SCALE_UPDATE_NORM = 2 };
 typedef struct muon_hparams {
@@ -132,6 +138,7 @@ typedef struct muon_hparams {
   int32_t scale_mode;
   float scale_dim;
   const float* coeffs;
+  int32_t protect_momentum;
 } muon_hparams;
 
 typedef struct muon_ctx muon_ctx;
@@ -280,7 +287,9 @@ int muon_step_host(muon_ctx* ctx, const muon_hparams* hp, const void* const* con
  * the norm is known).  Before the next step the caller must repair that
  * matrix's M - zero it, or restore it from a copy - or every later step of the
  * matrix reports MUON_ERR_NONFINITE again and leaves its W unchanged; the
- * other matrices of the context are not affected.
+ * other matrices of the context are not affected.  With
+ * muon_hparams.protect_momentum the matrix is reported in the same way but its
+ * M is left as it was, and nothing needs repair.
  */
 int muon_status(muon_ctx* ctx, void* stream, int* device_status, int* matrix_index);
 

@@ -66,6 +66,10 @@ class Hyper:
     # Optional list of (a, b, c), one triple per Newton-Schulz step, replacing
     # the single triple above (the paper uses one triple for all steps).
     coeffs: object = None
+    # Non-finite gradients (the paper is silent): False = the momentum is still
+    # M_t as the rule's first line defines it; True = a matrix whose gradient
+    # holds an Inf or a NaN keeps its momentum as well as its weight.
+    protect_momentum: bool = False
 
 
 def _f64(x):
@@ -232,12 +236,16 @@ def muon_step(W, G, M, hp: Hyper, trace=False):
     Non-finite input (a NaN or Inf anywhere in the Newton-Schulz input): the
     paper is silent.  The reading taken: the weight is left unchanged, the
     momentum is still M_t as the first line of the rule defines it, and the
-    result carries ``nonfinite = True``."""
+    result carries ``nonfinite = True``; with ``hp.protect_momentum`` a
+    non-finite gradient leaves the momentum unchanged as well."""
     W = _f64(W)
     G = _f64(G)
     M = _f64(M)
     if not (W.shape == G.shape == M.shape and W.ndim == 2):
         raise ValueError("W, G, M must be 2-D and of one shape")
+    if hp.protect_momentum and not np.all(np.isfinite(G)):
+        return {"M": M.copy(), "nu": float("nan"), "nonfinite": True, "W": W.copy(), "X0": None, "O": None,
+                "rms": float("nan")}
     M_new = momentum_update(M, G, hp.mu)
     U = newton_schulz_input(M_new, G, hp.mu, hp.nesterov)
     nu, X0 = frobenius_normalise(U, hp.eps)

@@ -59,7 +59,7 @@ class muon_hparams(C.Structure):
         ("a", C.c_float), ("b", C.c_float), ("c", C.c_float),
         ("eps", C.c_float), ("rms_scale", C.c_float),
         ("scale_mode", C.c_int32), ("scale_dim", C.c_float),
-        ("coeffs", C.POINTER(C.c_float)),
+        ("coeffs", C.POINTER(C.c_float)), ("protect_momentum", C.c_int32),
     ]
 
 
@@ -161,11 +161,12 @@ class Hyper:
     scale_mode: int = MUON_SCALE_ADJUSTED_LR
     scale_dim: float = 0.0
     coeffs: Optional[Sequence] = None  # one (a, b, c) per Newton-Schulz step
+    protect_momentum: bool = False  # a matrix with a non-finite gradient keeps its momentum too
 
     def to_c(self) -> muon_hparams:
         hp = muon_hparams(self.lr, self.wd, self.mu, int(bool(self.nesterov)), int(self.ns_steps),
                           self.a, self.b, self.c, self.eps, self.rms_scale, int(self.scale_mode),
-                          float(self.scale_dim), None)
+                          float(self.scale_dim), None, int(bool(self.protect_momentum)))
         if self.coeffs is not None:
             flat = [float(v) for triple in self.coeffs for v in triple]
             if len(flat) != 3 * int(self.ns_steps):

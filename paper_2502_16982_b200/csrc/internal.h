@@ -129,6 +129,7 @@ struct StreamParams {
   int tiles_per_matrix;
   float mu;
   int nesterov;
+  const int* g_bad;  // optional: per matrix, non-zero = its gradient is non-finite, leave M as it is
 };
 
 // Parameters of the TMA-pipelined momentum kernel (64 x 64 tiles).
@@ -144,6 +145,7 @@ struct StreamTmaParams {
   int m, n;                  // short and long side of the bucket
   float mu;
   int nesterov;
+  const int* g_bad;          // optional: per matrix, non-zero = its gradient is non-finite, leave M as it is
 };
 
 }  // namespace muon

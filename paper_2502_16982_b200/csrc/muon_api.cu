@@ -22,6 +22,8 @@
 namespace muon {
 
 cudaError_t launch_momentum_cast(const StreamParams& P, bool grad_fp32, cudaStream_t stream);
+cudaError_t launch_grad_finite(const MatDesc* descs, int count, int rows_max, bool grad_fp32, int* bad,
+                               cudaStream_t stream);
 cudaError_t launch_norm_finalise(const float* partials, int tiles_per_matrix, int count, float eps,
                                  const MatDesc* descs, MatScal* scal, float* norms, DevStatus* status,
                                  cudaStream_t stream);
@@ -126,7 +128,7 @@ struct Bucket {
   int pair_mode;              // the pair-fold mode the plan was made with
   // workspace offsets (bytes) of the chunk buffers
   // off_s: the symmetric m x m buffers (A and B; two more when iterations are taken in pairs)
-  size_t off_x[2], off_s[4], off_partials, off_scal, off_rms_partials, off_factors;
+  size_t off_x[2], off_s[4], off_partials, off_scal, off_rms_partials, off_factors, off_bad;
   // workspace offsets of the persistent per-bucket tables
   size_t off_descs, off_wmaps, off_gmaps, off_mmaps, off_sym_tiles, off_sym_tiles_tail, off_comb_tiles, off_comb_tiles_t;
   std::vector<PairTile> sym_tiles;       // symmetric products: table of one unit of sym_unit_mats matrices
@@ -483,6 +485,7 @@ int make_plan(const muon_group* groups, int n_groups, std::vector<Bucket>* bucke
       B.off_rms_partials = take(chunk * comb_tiles * 8 * sizeof(float));
     }
     B.off_factors = take(chunk * sizeof(float));
+    B.off_bad = take(chunk * sizeof(int));
     chunk_region = std::max(chunk_region, off);
   }
   size_t off = align_up(chunk_region, 1024);
@@ -1025,6 +1028,16 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
   float* partials = reinterpret_cast<float*>(ctx->ws + B.off_partials);
 
   const int stream_tiles = B.stream_tma ? B.stream_tiles_tma : B.stream_tiles_generic;
+  const int* g_bad = nullptr;
+  if (hp->protect_momentum) {
+    // find the matrices with a non-finite gradient first, so that their momentum is left alone
+    int* bad = reinterpret_cast<int*>(ctx->ws + B.off_bad);
+    LaunchTimer lt(ctx, stream, MUON_KERNEL_NORM);
+    ce = launch_grad_finite(descs, count, B.n, B.g_dtype == MUON_DTYPE_FP32, bad, stream);
+    if (ce != cudaSuccess) return fail(MUON_ERR_CUDA, "gradient check launch: %s", cudaGetErrorString(ce));
+    ++launches;
+    g_bad = bad;
+  }
   if (B.stream_tma) {
     StreamTmaParams S{};
     S.map_x = B.x_b64[0];
@@ -1039,6 +1052,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     S.n = B.n;
     S.mu = hp->mu;
     S.nesterov = hp->nesterov ? 1 : 0;
+    S.g_bad = g_bad;
     LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM);
     ce = launch_momentum_tma(S, B.g_dtype == MUON_DTYPE_FP32, ctx->num_sms, stream);
   } else {
@@ -1052,6 +1066,7 @@ static int step_chunk(muon_ctx* ctx, const muon_hparams* hp, cudaStream_t stream
     S.tiles_per_matrix = stream_tiles;
     S.mu = hp->mu;
     S.nesterov = hp->nesterov ? 1 : 0;
+    S.g_bad = g_bad;
     LaunchTimer lt(ctx, stream, MUON_KERNEL_MOMENTUM);
     ce = launch_momentum_cast(S, B.g_dtype == MUON_DTYPE_FP32, stream);
   }

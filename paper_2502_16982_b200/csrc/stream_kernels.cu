@@ -83,6 +83,7 @@ momentum_cast_kernel(const StreamParams P) {
   const int col = col0 + cgrp * 8;
   const int valid = min(8, max(0, d.cols - col));
   const bool vec = d.vec_ok != 0;
+  const bool keep_m = P.g_bad != nullptr && P.g_bad[mat] != 0;
 
   float g[kRowsPerThread][8], m[kRowsPerThread][8];
 #pragma unroll
@@ -132,7 +133,9 @@ momentum_cast_kernel(const StreamParams P) {
     for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(u[2 * e], u[2 * e + 1]);
     if (in) {
       float* mp = d.m + static_cast<long long>(row) * d.ld_m + col;
-      if (vec && valid == 8) {
+      if (keep_m) {
+        // a matrix whose gradient was found non-finite keeps its momentum
+      } else if (vec && valid == 8) {
         __stcs(reinterpret_cast<float4*>(mp), make_float4(m[p][0], m[p][1], m[p][2], m[p][3]));
         __stcs(reinterpret_cast<float4*>(mp) + 1, make_float4(m[p][4], m[p][5], m[p][6], m[p][7]));
       } else {
@@ -456,6 +459,56 @@ cudaError_t launch_sumsq_x(const __nv_bfloat16* x, long long x_stride, int ldx, 
   if (count == 0) return cudaSuccess;
   sumsq_x_kernel<<<dim3(static_cast<unsigned>(per_matrix), static_cast<unsigned>(count)), 256, 0, stream>>>(
       x, x_stride, ldx, m, n, partials);
+  return cudaGetLastError();
+}
+
+// Optional pass before the momentum update: bad[mat] = 1 if the gradient of matrix `mat` holds an Inf
+// or a NaN (exponent bits all ones), so that the momentum kernels can leave that matrix's M alone.
+// Grid (row slabs, matrices); `bad` is zeroed before the launch.
+template <bool kGradFp32>
+__global__ void __launch_bounds__(256)
+grad_finite_kernel(const MatDesc* __restrict__ descs, int* __restrict__ bad) {
+  const int mat = blockIdx.y;
+  const MatDesc d = descs[mat];
+  const bool vec = (reinterpret_cast<uintptr_t>(d.g) & 15) == 0 && d.ld_g % 8 == 0;
+  int found = 0;
+  for (int row = blockIdx.x; row < d.rows; row += gridDim.x) {
+    const long long base = static_cast<long long>(row) * d.ld_g;
+    for (int c = threadIdx.x * 8; c < d.cols; c += blockDim.x * 8) {
+      if (kGradFp32) {
+        const uint32_t* p = reinterpret_cast<const uint32_t*>(d.g) + base + c;
+        if (vec && c + 8 <= d.cols) {
+          const uint4 a = *reinterpret_cast<const uint4*>(p), b = *(reinterpret_cast<const uint4*>(p) + 1);
+          const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+          for (int e = 0; e < 8; ++e) found |= (w[e] & 0x7F800000u) == 0x7F800000u;
+        } else {
+          for (int e = 0; e < 8 && c + e < d.cols; ++e) found |= (p[e] & 0x7F800000u) == 0x7F800000u;
+        }
+      } else {
+        const unsigned short* p = reinterpret_cast<const unsigned short*>(d.g) + base + c;
+        if (vec && c + 8 <= d.cols) {
+          const uint4 a = *reinterpret_cast<const uint4*>(p);
+          const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            found |= ((w[e] & 0x7F80u) == 0x7F80u) | ((w[e] & 0x7F800000u) == 0x7F800000u);
+        } else {
+          for (int e = 0; e < 8 && c + e < d.cols; ++e) found |= (p[e] & 0x7F80u) == 0x7F80u;
+        }
+      }
+    }
+  }
+  if (__syncthreads_or(found) && threadIdx.x == 0) bad[mat] = 1;
+}
+
+cudaError_t launch_grad_finite(const MatDesc* descs, int count, int rows_max, bool grad_fp32, int* bad,
+                               cudaStream_t stream) {
+  cudaError_t e = cudaMemsetAsync(bad, 0, static_cast<size_t>(count) * sizeof(int), stream);
+  if (e != cudaSuccess) return e;
+  const dim3 grid(static_cast<unsigned>(rows_max < 64 ? rows_max : 64), static_cast<unsigned>(count));
+  if (grad_fp32) grad_finite_kernel<true><<<grid, 256, 0, stream>>>(descs, bad);
+  else grad_finite_kernel<false><<<grid, 256, 0, stream>>>(descs, bad);
   return cudaGetLastError();
 }
 

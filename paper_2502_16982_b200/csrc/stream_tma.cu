@@ -124,7 +124,9 @@ momentum_tma_kernel(const __grid_constant__ StreamTmaParams P) {
         const long long t = blockIdx.x + static_cast<long long>(i) * gridDim.x;
         P.partials[t] = sum;
         const uint32_t base = ptx::smem_u32(smem + s * C::kStageBytes);
-        ptx::tma_store_3d(P.mmaps + inf.mat, inf.col0, inf.row0, 0, base);
+        // a matrix whose gradient was found non-finite keeps its momentum (its norm comes out
+        // non-finite all the same, so its weight is kept too)
+        if (P.g_bad == nullptr || P.g_bad[inf.mat] == 0) ptx::tma_store_3d(P.mmaps + inf.mat, inf.col0, inf.row0, 0, base);
         if (inf.transposed) {
           ptx::tma_store_3d(&P.map_x, inf.row0, inf.col0, inf.mat, base + kMBytes + C::kGBytes);
         } else {

@@ -270,6 +270,58 @@ def test_canary_margins_stay_intact(wdt, cols):
         ctx.muon_destroy()
 
 
+@pytest.mark.parametrize("gdt,cols,bad", [(torch.float32, 264, float("nan")), (torch.bfloat16, 264, float("inf")),
+                                          (torch.bfloat16, 203, float("-inf"))])
+def test_protected_momentum_survives_a_nonfinite_gradient(gdt, cols, bad):
+    """hparams.protect_momentum: a pass over the gradients finds the matrix with
+    an Inf or a NaN before the momentum update; that matrix keeps its momentum
+    and its weight bit for bit, is reported, and steps normally - from that
+    momentum - on the next finite gradient, with nothing repaired.  The others
+    are not affected.  264 columns take the TMA momentum kernel, 203 the ld/st
+    one (rows that TMA cannot address)."""
+    b = _binding()
+    sp = wl.GroupSpec(136, cols, 3, torch.float32, gdt, 0.02, 1.0)
+    W, G, M = wl.make_group(sp, 81, "cpu", zero_momentum=False)
+    Wd, Gd, Md = W.cuda(), G.cuda(), M.cuda()
+    ctx = b.MuonContext([(wl.views(Wd), wl.views(Gd), wl.views(Md))])
+    try:
+        hp = b.Hyper(lr=1e-2, wd=0.1, protect_momentum=True)
+        ohp = orc.Hyper(lr=1e-2, wd=0.1, eps=hp.eps, protect_momentum=True)
+        # a clean step with the option on is the plain step
+        ctx.muon_step(hp)
+        assert ctx.muon_status()[0] == 0
+        for i in range(3):
+            ref = orc.muon_step(f64(W[i]), f64(G[i]), f64(M[i]), ohp)
+            assert rel(f64(Md[i]), ref["M"]) <= TOL_FP32
+            assert rel(f64(Wd[i]) - f64(W[i]), ref["W"] - f64(W[i])) <= TOL_NS
+        w1, m1 = Wd.cpu().clone(), Md.cpu().clone()
+        # the bad batch: last element of the last row of matrix 1
+        gen = torch.Generator().manual_seed(82)
+        G2 = wl.make_grads(sp, gen, "cpu")
+        G2[1, 135, cols - 1] = bad
+        Gd.copy_(G2)
+        ctx.muon_step(hp)
+        status, which = ctx.muon_status()
+        assert status == b.MUON_ERR_NONFINITE and which == 1
+        assert torch.equal(Wd[1].cpu(), w1[1]) and torch.equal(Md[1].cpu(), m1[1])
+        ref_bad = orc.muon_step(f64(w1[1]), f64(G2[1]), f64(m1[1]), ohp)
+        assert ref_bad["nonfinite"] and np.array_equal(ref_bad["M"], f64(m1[1]))
+        for i in (0, 2):
+            ref = orc.muon_step(f64(w1[i]), f64(G2[i]), f64(m1[i]), ohp)
+            assert rel(f64(Md[i]), ref["M"]) <= TOL_FP32
+            assert rel(f64(Wd[i]) - f64(w1[i]), ref["W"] - f64(w1[i])) <= TOL_NS
+        # the next finite gradient: matrix 1 carries on from the momentum it kept
+        G3 = wl.make_grads(sp, gen, "cpu")
+        Gd.copy_(G3)
+        ctx.muon_step(hp)
+        assert ctx.muon_status()[0] == 0
+        ref = orc.muon_step(f64(w1[1]), f64(G3[1]), f64(m1[1]), ohp)
+        assert rel(f64(Md[1]), ref["M"]) <= TOL_FP32
+        assert rel(f64(Wd[1]) - f64(w1[1]), ref["W"] - f64(w1[1])) <= TOL_NS
+    finally:
+        ctx.muon_destroy()
+
+
 def test_momentum_repaired_after_a_nonfinite_gradient():
     """A non-finite gradient: the matrix keeps its weight and its momentum holds
     the non-finite values (the oracle follows the same rule); the other matrices

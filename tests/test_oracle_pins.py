@@ -263,6 +263,25 @@ def test_nonfinite_input_leaves_weight_unchanged():
     assert out["nonfinite"] and np.array_equal(out["W"], W)
 
 
+def test_protected_momentum_on_a_nonfinite_gradient():
+    """The other reading of a non-finite gradient: weight AND momentum are left as
+    they were; a finite gradient gives exactly the default step."""
+    rng = np.random.default_rng(13)
+    W, M = rng.standard_normal((3, 4)), rng.standard_normal((3, 4))
+    G = rng.standard_normal((3, 4))
+    hp = orc.Hyper(protect_momentum=True)
+    same = orc.muon_step(W, G, M, hp)
+    ref = orc.muon_step(W, G, M, orc.Hyper())
+    assert np.array_equal(same["W"], ref["W"]) and np.array_equal(same["M"], ref["M"]) and not same["nonfinite"]
+    for bad in (np.nan, np.inf, -np.inf):
+        Gb = G.copy()
+        Gb[2, 1] = bad
+        out = orc.muon_step(W, Gb, M, hp)
+        assert out["nonfinite"] and np.array_equal(out["W"], W) and np.array_equal(out["M"], M)
+        plain = orc.muon_step(W, Gb, M, orc.Hyper())
+        assert plain["nonfinite"] and np.array_equal(plain["W"], W) and not np.all(np.isfinite(plain["M"]))
+
+
 def test_multi_step_momentum_chain():
     rng = np.random.default_rng(12)
     W = rng.standard_normal((4, 6))
