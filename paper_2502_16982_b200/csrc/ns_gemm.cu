@@ -5,7 +5,9 @@
 // Two CTAs on neighbouring SMs form a cluster and share one UMMA
 // (tcgen05.mma.cta_group::2): M = 256 (128 rows from each CTA's own A tile),
 // N = 128 or 256 with the B operand split between the two CTAs' shared
-// memories, so each CTA stages only half of B.
+// memories, so each CTA stages only half of B.  Which rows and columns a tile
+// covers comes from a table built on the host (PairTile): the two CTAs' row
+// blocks, even their matrices, need not be the same.
 //
 // Per CTA (192 threads):
 //   warp 0      TMA producer: its 128x64 A tile and its half of the B tile per
@@ -31,11 +33,12 @@
 // warp q owns rows 32 (q & 1) .. + 31 of the CTA and column half q >> 1.
 //
 // Symmetric matrices (A and B) are kept as their 128x128 blocks on or above
-// the diagonal only.  The products that produce them visit only column blocks
-// j >= 2p of row pair p and drop the one below-diagonal block (2p+1, 2p) the
-// pair computes anyway; the products that consume them read a block below the
-// diagonal as the transpose of its mirror image (an MN-major UMMA operand), so
-// both triangles are the same bits by construction.
+// the diagonal only.  The products that produce them follow a tile table that
+// covers exactly those blocks (a table entry says which blocks of a tile are
+// stored: a block under the diagonal, or the cross blocks of a tile shared by
+// two matrices, are computed and dropped); the products that consume them read
+// a block below the diagonal as the transpose of its mirror image (an MN-major
+// UMMA operand), so both triangles are the same bits by construction.
 //
 // The combine is a*X + B X.  For buckets whose short side is at least 16 the
 // polynomial's epilogue adds a to the diagonal of B in fp32 before the one bf16
