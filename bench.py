@@ -620,12 +620,28 @@ def main():
         e1.record(stream)
         barrier()
         ms_down = e0.elapsed_time(e1) / n_copy
+        # both directions at once on two streams, no kernels: what the link gives when gradients go up
+        # while weights come down, which is what every step but its first and last slice does
+        side = torch.cuda.Stream(device=dev)
+        e0.record(stream)
+        side.wait_stream(stream)
+        for _ in range(n_copy):
+            for (W, G, M), gh, wh in zip([st for st in state if len(st) == 3], g_host, w_host):
+                for i in range(len(gh)):
+                    G[i].copy_(gh[i], non_blocking=True)
+                    with torch.cuda.stream(side):
+                        wh[i].copy_(W[i], non_blocking=True)
+        stream.wait_stream(side)
+        e1.record(stream)
+        barrier()
+        ms_both = e0.elapsed_time(e1) / n_copy
         floor = max(ms_step, ms_up, ms_down)
         e2e = {"value": whole_job_value(alg_flops, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "h2d_gbs_in_step": h2d / (ms_e2e * 1e-3) / 1e9, "d2h_gbs_in_step": d2h / (ms_e2e * 1e-3) / 1e9,
                "h2d_alone_ms": ms_up, "h2d_alone_gbs": h2d / (ms_up * 1e-3) / 1e9,
                "d2h_alone_ms": ms_down, "d2h_alone_gbs": d2h / (ms_down * 1e-3) / 1e9,
+               "both_directions_at_once_ms": ms_both, "over_both_directions_at_once": ms_e2e / max(ms_both, ms_step),
                "over_floor": ms_e2e / floor,
                "floor": "max(device-resident step, upload alone, download alone) = %.2f ms" % floor}
 
