@@ -134,6 +134,7 @@ def _fill_grads_only(dm, seed, grad_scale):
             dm.grads[gi][j].copy_(_grad(rows, cols, gen, grad_scale).to(gd))
 
 
+@pytest.mark.timeout(600)
 @pytest.mark.parametrize("reduce_grads", [False, True])
 def test_two_ranks_end_with_the_single_process_weights(tmp_path, reduce_grads):
     out = str(tmp_path / "rank%d.pt")

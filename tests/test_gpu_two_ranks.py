@@ -85,6 +85,7 @@ def _worker(rank, world, port, out):
     dist.destroy_process_group()
 
 
+@pytest.mark.timeout(600)
 def test_two_processes_on_one_gpu_give_the_single_process_bits(tmp_path):
     from paper_2502_16982_b200 import binding, workloads as wl
 

@@ -7,6 +7,7 @@ import os
 import socket
 import sys
 
+import pytest
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -46,6 +47,7 @@ def _worker(rank, world, port, out):
     dist.destroy_process_group()
 
 
+@pytest.mark.timeout(600)
 def test_two_cpu_ranks_shard_and_reduce(tmp_path):
     out = str(tmp_path / "r0.pt")
     mp.spawn(_worker, args=(2, _free_port(), out), nprocs=2, join=True)
