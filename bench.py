@@ -306,12 +306,18 @@ def run_distributed(args, rank, world, local_rank):
     hp = binding.Hyper(**hpd)
     dm = DistributedMuon([(s.rows, s.cols, s.count, s.w_dtype, s.g_dtype) for s in specs], dev, dist=dist)
     # the same weights and (already reduced) gradients on every rank: same seeds everywhere
+    # (the generator calls of workloads.make_group, group by group, so that the values are the N = 1 run's)
     for gi, sp in enumerate(specs):
         gen = torch.Generator(device=dev)
         gen.manual_seed(1000 * args.config + gi)
+        W = wl._randn((sp.count, sp.rows, sp.cols), sp.w_std, gen, dev, sp.w_dtype)
         for j in range(sp.count):
-            dm.weights[gi][j].copy_((torch.randn(sp.rows, sp.cols, generator=gen, device=dev) * sp.w_std).to(sp.w_dtype))
-            dm.grads[gi][j].copy_((torch.randn(sp.rows, sp.cols, generator=gen, device=dev) * sp.g_std).to(sp.g_dtype))
+            dm.weights[gi][j].copy_(W[j])
+        del W
+        G = wl.make_grads(sp, gen, dev)
+        for j in range(sp.count):
+            dm.grads[gi][j].copy_(G[j])
+        del G
     stream = torch.cuda.current_stream(dev)
     alg_flops, _ = wl.ns_flops(specs, hp.ns_steps)
 
